@@ -1,0 +1,663 @@
+// Score-side kernels: everything that works on the per-token score arrays.
+//
+//   head_scores  (Sections 2.3-2.4)  min-max, reliability gaps (exact top/bottom-m sums),
+//                                    softmax weights, surprise, gate, routed score, sink pin
+//   budget       (Section 2.6)       per-head safeguard thresholds, cross-head competition
+//   select       (Section 2.5)       TopB_h as an ordered stream compaction
+//   ranks                            place of every token in its head's order (diagnostic)
+//
+// All order statistics are exact.  The selection primitive finds the rank-th largest
+// element of a multiset of floats by counting into 2048 value-linear bins, refining the
+// chosen bin up to three times (each level splits it 2048 ways again), and finishing on
+// the at most kCap candidates that remain by direct rank counting.  If a bin still holds
+// more than kCap elements after three levels (massive ties), an 8-bit most-significant-
+// digit radix select over the ordered key bits finishes the job.  Only monotonicity of the
+// binning function is needed for exactness, so float rounding inside it is harmless.
+#include "nkv_common.cuh"
+
+namespace nkv {
+
+namespace {
+
+constexpr int kThreads = 1024;
+constexpr int kBins = 2048;
+constexpr int kCap = 2048;
+constexpr int kLevels = 3;
+constexpr int kMaxCorr = 64;   // heads per group supported by the budget kernel
+
+struct SelectShared {
+    int hist[kBins];
+    uint32_t cand[kCap];
+    int cand_n;
+    int bin, above, nbin;
+    uint32_t theta;
+    int gt, eq;
+    int found;
+    float red_f[32];
+    int red_i[32];
+    // elements to remove from the multiset (value, multiplicity)
+    float corr_v[kMaxCorr];
+    int corr_m[kMaxCorr];
+    int ncorr;
+};
+
+struct Levels {
+    float lo[kLevels], sc[kLevels];
+    int bin[kLevels];
+    int n;  // levels fixed so far
+};
+
+__device__ __forceinline__ int bin_of(float v, float lo, float sc) {
+    int b = __float2int_rz((v - lo) * sc);
+    return min(max(b, 0), kBins - 1);
+}
+__device__ __forceinline__ bool matches(const Levels& L, float v) {
+    for (int i = 0; i < L.n; ++i)
+        if (bin_of(v, L.lo[i], L.sc[i]) != L.bin[i]) return false;
+    return true;
+}
+
+// warp 0: the bin holding the `need`-th element counted from the top, and the count above it.
+__device__ __forceinline__ void find_bin_desc(SelectShared& S, int need) {
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x;
+        constexpr int per = kBins / 32;
+        const int top = kBins - 1 - lane * per;  // lane 0 owns the highest bins
+        int sum = 0;
+        for (int j = 0; j < per; ++j) sum += S.hist[top - j];
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        const int excl = incl - sum;
+        if (need > excl && need <= incl) {
+            int run = excl;
+            for (int j = 0; j < per; ++j) {
+                const int c = S.hist[top - j];
+                if (need <= run + c) {
+                    S.bin = top - j;
+                    S.above = run;
+                    S.nbin = c;
+                    break;
+                }
+                run += c;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ int block_sum_int(SelectShared& S, int v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) S.red_i[threadIdx.x >> 5] = v;
+    __syncthreads();
+    int t = (threadIdx.x < (blockDim.x >> 5)) ? S.red_i[threadIdx.x] : 0;
+    if (threadIdx.x < 32) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+        if (threadIdx.x == 0) S.red_i[0] = t;
+    }
+    __syncthreads();
+    return S.red_i[0];
+}
+
+// Exact selection of the rank-th largest (1-based) element of { src(j) : j in [0,n), src.get true }
+// minus the S.corr multiset.  Results in S.theta (ordered key), S.gt (#elements > theta),
+// S.eq (#elements == theta).  lo/scale give the level-0 binning.  Must be called by all threads.
+template <class Src>
+__device__ void block_select_desc(SelectShared& S, const Src& src, int n, int rank, float lo0, float sc0, int* status) {
+    Levels L;
+    L.n = 0;
+    float lo = lo0, sc = sc0;
+    int need = rank, above_total = 0;
+    bool small = false;
+    for (int level = 0; level < kLevels; ++level) {
+        for (int b = threadIdx.x; b < kBins; b += blockDim.x) S.hist[b] = 0;
+        if (threadIdx.x == 0) {
+            S.bin = 0;
+            S.above = 0;
+            S.nbin = 0;
+        }
+        __syncthreads();
+        for (int j = threadIdx.x; j < n; j += blockDim.x) {
+            float v;
+            if (src.get(j, v) && matches(L, v)) atomicAdd(&S.hist[bin_of(v, lo, sc)], 1);
+        }
+        __syncthreads();
+        if (threadIdx.x < S.ncorr) {
+            const float v = S.corr_v[threadIdx.x];
+            if (S.corr_m[threadIdx.x] > 0 && matches(L, v)) atomicSub(&S.hist[bin_of(v, lo, sc)], S.corr_m[threadIdx.x]);
+        }
+        __syncthreads();
+        find_bin_desc(S, need);
+        __syncthreads();
+        above_total += S.above;
+        need -= S.above;
+        L.lo[level] = lo;
+        L.sc[level] = sc;
+        L.bin[level] = S.bin;
+        L.n = level + 1;
+        if (S.nbin <= kCap) {
+            small = true;
+            break;
+        }
+        lo = lo + (float)S.bin / sc;
+        sc = sc * (float)kBins;
+        __syncthreads();
+    }
+
+    if (small) {
+        if (threadIdx.x == 0) {
+            S.cand_n = 0;
+            S.found = 0;
+        }
+        __syncthreads();
+        for (int j = threadIdx.x; j < n; j += blockDim.x) {
+            float v;
+            if (src.get(j, v) && matches(L, v)) {
+                const int pos = atomicAdd(&S.cand_n, 1);
+                if (pos < kCap) S.cand[pos] = ord_key(v);
+            }
+        }
+        __syncthreads();
+        const int cn = min(S.cand_n, kCap);
+        for (int a = threadIdx.x; a < cn; a += blockDim.x) {
+            const uint32_t x = S.cand[a];
+            int gt = 0, eq = 0;
+            for (int b = 0; b < cn; ++b) {
+                const uint32_t y = S.cand[b];
+                gt += (y > x);
+                eq += (y == x);
+            }
+            for (int c = 0; c < S.ncorr; ++c) {
+                if (S.corr_m[c] > 0 && matches(L, S.corr_v[c])) {
+                    const uint32_t y = ord_key(S.corr_v[c]);
+                    if (y > x) gt -= S.corr_m[c];
+                    if (y == x) eq -= S.corr_m[c];
+                }
+            }
+            if (gt < need && need <= gt + eq) {
+                S.theta = x;
+                S.gt = above_total + gt;
+                S.eq = eq;
+                S.found = 1;
+            }
+        }
+        __syncthreads();
+        if (!S.found && threadIdx.x == 0) set_status(status, NKV_ERR_DEVICE_CHECK, 101);
+        __syncthreads();
+        return;
+    }
+
+    // radix fallback over the ordered key bits of the elements of the last chosen bin
+    if (threadIdx.x == 0) atomicAdd(&status[kStatusFallbacks], 1);
+    uint32_t prefix = 0;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        const uint32_t himask = (shift == 24) ? 0u : (0xffffffffu << (shift + 8));
+        for (int b = threadIdx.x; b < 256; b += blockDim.x) S.hist[b] = 0;
+        __syncthreads();
+        for (int j = threadIdx.x; j < n; j += blockDim.x) {
+            float v;
+            if (src.get(j, v) && matches(L, v)) {
+                const uint32_t key = ord_key(v);
+                if (((key ^ prefix) & himask) == 0) atomicAdd(&S.hist[(key >> shift) & 255], 1);
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x < S.ncorr) {
+            const float v = S.corr_v[threadIdx.x];
+            const uint32_t key = ord_key(v);
+            if (S.corr_m[threadIdx.x] > 0 && matches(L, v) && ((key ^ prefix) & himask) == 0)
+                atomicSub(&S.hist[(key >> shift) & 255], S.corr_m[threadIdx.x]);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int run = 0, dsel = 0;
+            for (int dgt = 255; dgt >= 0; --dgt) {
+                const int c = S.hist[dgt];
+                if (need <= run + c) {
+                    dsel = dgt;
+                    S.nbin = c;
+                    break;
+                }
+                run += c;
+            }
+            S.bin = dsel;
+            S.above = run;
+        }
+        __syncthreads();
+        above_total += S.above;
+        need -= S.above;
+        prefix |= ((uint32_t)S.bin) << shift;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        S.theta = prefix;
+        S.gt = above_total;
+        S.eq = S.nbin;
+    }
+    __syncthreads();
+}
+
+// ------------------------------------------------------------------------------------------
+// head_scores: one CTA per head.
+// ------------------------------------------------------------------------------------------
+struct ScaleSrc {      // values of one scale of one head; `flip` turns bottom-m into top-m of the negated values
+    const float* a;
+    float sign;
+    __device__ __forceinline__ bool get(int j, float& v) const {
+        v = sign * a[j];
+        return true;
+    }
+};
+
+__device__ __forceinline__ float norm01(float a, float lo, float range) { return range > 0.f ? (a - lo) / range : 0.f; }
+
+__device__ __forceinline__ float surprise3(float x0, float x1, float x2) {
+    const float mean = (x0 + x1 + x2) / 3.0f;
+    const float d0 = x0 - mean, d1 = x1 - mean, d2 = x2 - mean;
+    return sqrtf((d0 * d0 + d1 * d1 + d2 * d2) / 3.0f);
+}
+
+__device__ __forceinline__ float block_reduce_f(SelectShared& S, float v, int op) {  // 0 sum, 1 min, 2 max
+    if (op == 0) v = warp_sum(v);
+    else if (op == 1) v = warp_min(v);
+    else v = warp_max(v);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) S.red_f[threadIdx.x >> 5] = v;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        const int nw = blockDim.x >> 5;
+        float t = (threadIdx.x < nw) ? S.red_f[threadIdx.x] : (op == 0 ? 0.f : (op == 1 ? INFINITY : -INFINITY));
+        if (op == 0) t = warp_sum(t);
+        else if (op == 1) t = warp_min(t);
+        else t = warp_max(t);
+        if (threadIdx.x == 0) S.red_f[0] = t;
+    }
+    __syncthreads();
+    const float r = S.red_f[0];
+    __syncthreads();
+    return r;
+}
+
+__global__ void __launch_bounds__(kThreads) head_scores_kernel(int N, ScoreParams sp, const float* __restrict__ a_raw,
+                                                               const uint32_t* __restrict__ mm,
+                                                               float* __restrict__ a_star, float* __restrict__ stats_out,
+                                                               int* status) {
+    __shared__ SelectShared S;
+    __shared__ float sh_delta[3], sh_w[3], sh_s[3];
+    const int u = blockIdx.x;
+    const float* a[3] = {a_raw + ((int64_t)u * 3 + 0) * N, a_raw + ((int64_t)u * 3 + 1) * N,
+                         a_raw + ((int64_t)u * 3 + 2) * N};
+    float lo[3], range[3];
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+        lo[k] = ord_float(mm[(int64_t)u * 6 + 2 * k]);
+        range[k] = ord_float(mm[(int64_t)u * 6 + 2 * k + 1]) - lo[k];
+    }
+    if (threadIdx.x == 0) S.ncorr = 0;
+    __syncthreads();
+
+    // reliability gaps: (sum of the m largest - sum of the m smallest) / (m * range)
+    const int m = sp.top_m;
+    for (int k = 0; k < 3; ++k) {
+        float gap = 0.f;
+        if (range[k] > 0.f) {
+            float side_sum[2];
+            for (int side = 0; side < 2; ++side) {
+                ScaleSrc src{a[k], side == 0 ? 1.f : -1.f};
+                const float lo0 = side == 0 ? lo[k] : -(lo[k] + range[k]);
+                block_select_desc(S, src, N, m, lo0, (float)kBins / range[k], status);
+                const uint32_t theta = S.theta;
+                const int gt = S.gt;
+                __syncthreads();
+                float part = 0.f;
+                for (int j = threadIdx.x; j < N; j += blockDim.x) {
+                    const float v = src.sign * a[k][j];
+                    if (ord_key(v) > theta) part += v;
+                }
+                const float above = block_reduce_f(S, part, 0);
+                side_sum[side] = above + (float)(m - gt) * ord_float(theta);
+            }
+            // side 1 summed the negated values: top_sum - bot_sum = side_sum[0] + side_sum[1]
+            gap = (side_sum[0] + side_sum[1]) / ((float)m * range[k]);
+        }
+        if (threadIdx.x == 0) sh_delta[k] = gap;
+    }
+
+    // surprise statistics over the head
+    float smin = INFINITY, smax = -INFINITY, ssum = 0.f;
+    for (int j = threadIdx.x; j < N; j += blockDim.x) {
+        const float s = surprise3(norm01(a[0][j], lo[0], range[0]), norm01(a[1][j], lo[1], range[1]),
+                                  norm01(a[2][j], lo[2], range[2]));
+        smin = fminf(smin, s);
+        smax = fmaxf(smax, s);
+        ssum += s;
+    }
+    smin = block_reduce_f(S, smin, 1);
+    smax = block_reduce_f(S, smax, 2);
+    ssum = block_reduce_f(S, ssum, 0);
+    if (threadIdx.x == 0) {
+        float z[3], zmax = -INFINITY, wsum = 0.f;
+        for (int k = 0; k < 3; ++k) {
+            z[k] = sp.log_prior[k] + sp.beta * sh_delta[k];
+            zmax = fmaxf(zmax, z[k]);
+        }
+        for (int k = 0; k < 3; ++k) {
+            z[k] = expf(z[k] - zmax);
+            wsum += z[k];
+        }
+        for (int k = 0; k < 3; ++k) sh_w[k] = z[k] / wsum;
+        const float srange = smax - smin;
+        sh_s[0] = smin;
+        sh_s[1] = srange;
+        sh_s[2] = srange > 0.f ? (ssum / (float)N - smin) / srange : 0.f;
+    }
+    __syncthreads();
+    const float w0 = sh_w[0], w1 = sh_w[1], w2 = sh_w[2];
+    const float s_lo = sh_s[0], s_range = sh_s[1], s_mean = sh_s[2];
+
+    for (int j = threadIdx.x; j < N; j += blockDim.x) {
+        const float x0 = norm01(a[0][j], lo[0], range[0]);
+        const float x1 = norm01(a[1][j], lo[1], range[1]);
+        const float x2 = norm01(a[2][j], lo[2], range[2]);
+        const float blend = w0 * x0 + w1 * x1 + w2 * x2;
+        const float win = fmaxf(x0, fmaxf(x1, x2));
+        float alpha;
+        if (sp.gate_mode == NKV_GATE_AVERAGE) alpha = 0.f;
+        else if (sp.gate_mode == NKV_GATE_MAX) alpha = 1.f;
+        else {
+            const float sn = norm01(surprise3(x0, x1, x2), s_lo, s_range);
+            const float sprime = fmaxf(0.f, sn - s_mean);
+            alpha = 1.0f / (1.0f + expf(-sp.kappa * (sprime - sp.tau)));
+        }
+        float v = (1.0f - alpha) * blend + alpha * win + 0.f;
+        if (j < sp.n_sink) v = INFINITY;
+        a_star[(int64_t)u * N + j] = v;
+    }
+    if (stats_out && threadIdx.x == 0) {
+        float* o = stats_out + (int64_t)u * NKV_HEAD_STATS;
+        for (int k = 0; k < 3; ++k) {
+            o[k] = lo[k];
+            o[3 + k] = lo[k] + range[k];
+            o[6 + k] = sh_delta[k];
+            o[9 + k] = sh_w[k];
+        }
+        o[12] = s_lo;
+        o[13] = s_lo + s_range;
+        o[14] = s_mean;
+        o[15] = (float)m;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// budget: one CTA per layer group.
+// ------------------------------------------------------------------------------------------
+struct HeadSrc {
+    const float* v;
+    __device__ __forceinline__ bool get(int j, float& x) const {
+        x = v[j];
+        return true;
+    }
+};
+struct PoolSrc {       // all (head, token) pairs of a group whose key does not exceed the head's safeguard threshold
+    const float* v;    // [H, N]
+    const uint32_t* T; // per-head safeguard threshold keys (shared memory)
+    int N;
+    __device__ __forceinline__ bool get(int j, float& x) const {
+        x = v[j];
+        return ord_key(x) <= T[j / N];
+    }
+};
+
+__global__ void __launch_bounds__(kThreads) budget_kernel(int H, int N, int keep, int n_safe,
+                                                          const float* __restrict__ a_star,
+                                                          int32_t* __restrict__ budgets, uint32_t* __restrict__ thr,
+                                                          int* status) {
+    __shared__ SelectShared S;
+    __shared__ uint32_t T[kMaxCorr];
+    __shared__ int c_gt[kMaxCorr], corr[kMaxCorr], cnt_mid[kMaxCorr], cnt_eq[kMaxCorr];
+    const int g = blockIdx.x;
+    const float* v = a_star + (int64_t)g * H * N;
+    if (threadIdx.x == 0) S.ncorr = 0;
+    __syncthreads();
+
+    // per-head safeguard: the n_safe best tokens of each head are kept unconditionally
+    for (int h = 0; h < H; ++h) {
+        if (n_safe > 0) {
+            HeadSrc src{v + (int64_t)h * N};
+            block_select_desc(S, src, N, n_safe, 0.f, (float)kBins, status);
+            if (threadIdx.x == 0) {
+                T[h] = S.theta;
+                c_gt[h] = S.gt;
+                corr[h] = n_safe - S.gt;   // ties at the threshold that belong to the safeguard
+            }
+        } else if (threadIdx.x == 0) {
+            T[h] = 0xffffffffu;
+            c_gt[h] = 0;
+            corr[h] = 0;
+        }
+        __syncthreads();
+    }
+
+    // cross-head competition for the remaining slots
+    const int rest = H * keep - H * n_safe;
+    uint32_t tau = 0xffffffffu;
+    if (rest > 0) {
+        if (threadIdx.x < H) {
+            S.corr_v[threadIdx.x] = ord_float(T[threadIdx.x]);
+            S.corr_m[threadIdx.x] = corr[threadIdx.x];
+        }
+        if (threadIdx.x == 0) S.ncorr = H;
+        __syncthreads();
+        PoolSrc src{v, T, N};
+        block_select_desc(S, src, H * N, rest, 0.f, (float)kBins, status);
+        tau = S.theta;
+        __syncthreads();
+    }
+    for (int h = 0; h < H; ++h) {
+        int mid = 0, eq = 0;
+        const uint32_t Th = T[h];
+        for (int j = threadIdx.x; j < N; j += blockDim.x) {
+            const uint32_t key = ord_key(v[(int64_t)h * N + j]);
+            mid += (key > tau && key <= Th);
+            eq += (key == tau && key <= Th);
+        }
+        mid = block_sum_int(S, mid);
+        __syncthreads();
+        eq = block_sum_int(S, eq);
+        if (threadIdx.x == 0) {
+            cnt_mid[h] = mid;
+            cnt_eq[h] = eq;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        int taken_gt = 0;
+        for (int h = 0; h < H; ++h) taken_gt += cnt_mid[h] - (T[h] > tau ? corr[h] : 0);
+        int remaining = rest - taken_gt;
+        int total = 0;
+        for (int h = 0; h < H; ++h) {
+            const int pool_eq = cnt_eq[h] - (T[h] == tau ? corr[h] : 0);
+            const int t = max(0, min(pool_eq, remaining));
+            remaining -= t;
+            const int B = n_safe + cnt_mid[h] - (T[h] > tau ? corr[h] : 0) + t;
+            budgets[(int64_t)g * H + h] = B;
+            total += B;
+            uint32_t theta, q;
+            if (tau < T[h]) {
+                theta = tau;
+                q = (uint32_t)t;
+            } else {
+                theta = T[h];
+                q = (uint32_t)(corr[h] + t);
+            }
+            thr[((int64_t)g * H + h) * 2] = theta;
+            thr[((int64_t)g * H + h) * 2 + 1] = q;
+        }
+        if (total != H * keep || remaining != 0) set_status(status, NKV_ERR_DEVICE_CHECK, 201);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// select: one CTA per head, ordered compaction of the retained positions.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int* total) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    __syncthreads();
+    if (lane == 31) warp_tot[w] = incl;
+    __syncthreads();
+    if (w == 0) {
+        int t = warp_tot[lane];
+        int ti = t;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int y = __shfl_up_sync(0xffffffffu, ti, o);
+            if (lane >= o) ti += y;
+        }
+        warp_tot[lane] = ti - t;
+        if (lane == 31) *total = ti;
+    }
+    __syncthreads();
+    return warp_tot[w] + incl - v;
+}
+
+__global__ void __launch_bounds__(kThreads) select_kernel(int H, int N, int64_t cap, const float* __restrict__ a_star,
+                                                          const int32_t* __restrict__ budgets,
+                                                          const uint32_t* __restrict__ thr, int32_t* __restrict__ idx,
+                                                          int32_t* __restrict__ head_offsets, int* status) {
+    __shared__ SelectShared S;
+    __shared__ int warp_tot[32];
+    __shared__ int tot;
+    const int u = blockIdx.x, g = u / H, h = u % H;
+    const float* v = a_star + (int64_t)u * N;
+    const int B = budgets[u];
+    int off = 0;
+    for (int hh = 0; hh < h; ++hh) off += budgets[(int64_t)g * H + hh];
+    if (threadIdx.x == 0) {
+        head_offsets[(int64_t)g * (H + 1) + h] = off;
+        if (h == H - 1) head_offsets[(int64_t)g * (H + 1) + H] = off + B;
+        S.ncorr = 0;
+    }
+    __syncthreads();
+    if (B <= 0) return;
+    if (B > N || off + B > cap) {
+        if (threadIdx.x == 0) set_status(status, NKV_ERR_DEVICE_CHECK, 301);
+        return;
+    }
+    uint32_t theta;
+    int q;
+    if (thr) {
+        theta = thr[(int64_t)u * 2];
+        q = (int)thr[(int64_t)u * 2 + 1];
+    } else {
+        HeadSrc src{v};
+        block_select_desc(S, src, N, B, 0.f, (float)kBins, status);
+        theta = S.theta;
+        q = B - S.gt;
+        __syncthreads();
+    }
+    int run_eq = 0, run_sel = 0;
+    for (int base = 0; base < N; base += kThreads * 4) {
+        const int j0 = base + threadIdx.x * 4;
+        uint32_t key[4];
+        int eq_cnt = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            key[e] = (j0 + e < N) ? ord_key(v[j0 + e]) : 0u;
+            eq_cnt += (j0 + e < N && key[e] == theta);
+        }
+        int t_eq;
+        int tie_rank = run_eq + block_exclusive_scan(eq_cnt, warp_tot, &tot);
+        t_eq = tot;
+        __syncthreads();
+        int sel[4], sel_cnt = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const bool in = j0 + e < N;
+            const bool is_eq = in && key[e] == theta;
+            sel[e] = in && (key[e] > theta || (is_eq && tie_rank < q));
+            tie_rank += is_eq;
+            sel_cnt += sel[e];
+        }
+        int pos = run_sel + block_exclusive_scan(sel_cnt, warp_tot, &tot);
+        const int t_sel = tot;
+        __syncthreads();
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (sel[e]) {
+                if (pos < B) idx[(int64_t)g * cap + off + pos] = j0 + e;
+                ++pos;
+            }
+        run_eq += t_eq;
+        run_sel += t_sel;
+    }
+    if (threadIdx.x == 0 && run_sel != B) set_status(status, NKV_ERR_DEVICE_CHECK, 302);
+}
+
+// ranks: place of token i in its head's order (score descending, position ascending).  O(N^2).
+__global__ void __launch_bounds__(256) ranks_kernel(int N, const float* __restrict__ a_star, int32_t* __restrict__ ranks) {
+    __shared__ uint32_t tile[1024];
+    const int u = blockIdx.y;
+    const float* v = a_star + (int64_t)u * N;
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    const uint32_t mine = i < N ? ord_key(v[i]) : 0u;
+    int r = 0;
+    for (int base = 0; base < N; base += 1024) {
+        __syncthreads();
+        for (int t = threadIdx.x; t < 1024; t += 256) tile[t] = (base + t < N) ? ord_key(v[base + t]) : 0u;
+        __syncthreads();
+        const int lim = min(1024, N - base);
+        for (int t = 0; t < lim; ++t) {
+            const uint32_t y = tile[t];
+            r += (y > mine) || (y == mine && base + t < i);
+        }
+    }
+    if (i < N) ranks[(int64_t)u * N + i] = r;
+}
+
+}  // namespace
+
+cudaError_t launch_head_scores(int units, int N, const ScoreParams& sp, const float* a_raw,
+                               const uint32_t* minmax_keys, float* a_star, float* head_stats_opt, int* status,
+                               cudaStream_t stream, int64_t* launches) {
+    head_scores_kernel<<<units, kThreads, 0, stream>>>(N, sp, a_raw, minmax_keys, a_star, head_stats_opt, status);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_budget(int G, int H, int N, int keep, int n_safe, const float* a_star, int32_t* budgets,
+                          uint32_t* sel_thresholds, int* status, cudaStream_t stream, int64_t* launches) {
+    if (H > kMaxCorr) return cudaErrorInvalidValue;
+    budget_kernel<<<G, kThreads, 0, stream>>>(H, N, keep, n_safe, a_star, budgets, sel_thresholds, status);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_select(int G, int H, int N, int64_t idx_capacity, const float* a_star, const int32_t* budgets,
+                          const uint32_t* sel_thresholds_or_null, int32_t* idx, int32_t* head_offsets, int* status,
+                          cudaStream_t stream, int64_t* launches) {
+    select_kernel<<<G * H, kThreads, 0, stream>>>(H, N, idx_capacity, a_star, budgets, sel_thresholds_or_null, idx,
+                                                  head_offsets, status);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_ranks(int units, int N, const float* a_star, int32_t* ranks, cudaStream_t stream,
+                         int64_t* launches) {
+    dim3 grid((N + 255) / 256, units);
+    ranks_kernel<<<grid, 256, 0, stream>>>(N, a_star, ranks);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace nkv

@@ -1,0 +1,242 @@
+"""GPU parity: every stage of the CUDA path against the CPU oracle, through the C ABI.
+
+Stage tests feed each GPU stage the oracle's output of the previous one ("teacher forcing"),
+so integer stages are compared bit for bit.  End-to-end tests run the fused call and account
+for near-tie swaps.  All inputs come from the seeded generator; the oracle reads the bytes the
+GPU read.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_26678_b200 import nkv
+from paper_2605_26678_b200 import workloads as wl
+from tests import parity as pr
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _cache(N, d, dtype, H=2, layers=1, seed=11, seg=(32, 96)):
+    cfg = wl.tiny_config(kv_heads=H, head_dim=d, seq_len=N, dtype=dtype, layers=layers, base_seed=seed,
+                         seg_lo=seg[0], seg_hi=seg[1])
+    K, V = wl.make_cache(cfg)
+    return K.to(DEV), V.to(DEV)
+
+
+SHAPES = [(1, 64, "fp32"), (3, 64, "bf16"), (63, 128, "bf16"), (64, 64, "fp32"), (65, 128, "fp32"),
+          (200, 64, "bf16"), (257, 128, "bf16"), (1000, 128, "fp32"), (4133, 64, "bf16"), (6000, 128, "bf16")]
+
+
+@pytest.mark.parametrize("N,d,dtype", SHAPES)
+def test_anchors_match_oracle(N, d, dtype):
+    K, _ = _cache(N, d, dtype)
+    mu_s, mu_e, inv_norm, mu_c = nkv.nkv_anchors(K, want_mu_c=(N <= 1000))
+    torch.cuda.synchronize()
+    for g in range(K.shape[0]):
+        for h in range(K.shape[1]):
+            ref = oracle.score_head(K[g, h].cpu(), want_mu_c=(N <= 1000))
+            pr.assert_close(inv_norm[g, h].cpu().numpy(), ref.inv_norm, "inv_norm", 1e-5)
+            pr.assert_close(mu_s[g, h].cpu().numpy(), ref.mu_s, "mu_s", 1e-5)
+            pr.assert_close(mu_e[g, h].cpu().numpy(), ref.mu_e, "mu_e", 1e-5)
+            if mu_c is not None:
+                pr.assert_close(mu_c[g, h].cpu().numpy(), ref.mu_c, "mu_c", 1e-5)
+
+
+@pytest.mark.parametrize("N,d,dtype", SHAPES)
+def test_scores_match_oracle(N, d, dtype):
+    K, _ = _cache(N, d, dtype)
+    mu_s, mu_e, inv_norm, _ = nkv.nkv_anchors(K)
+    a_star, a_raw, stats = nkv.nkv_score(K, mu_s, mu_e, inv_norm, want_raw=True, want_stats=True)
+    torch.cuda.synchronize()
+    for h in range(K.shape[1]):
+        ref = oracle.score_head(K[0, h].cpu())
+        pr.assert_close(a_raw[0, h].cpu().numpy(), ref.a_raw, "a_raw")
+        st = stats[0, h].cpu().numpy()
+        if N >= 8:   # with a handful of tokens the min-max range can be rounding noise in both precisions
+            pr.assert_close(st[0:3], ref.lo, "lo")
+            pr.assert_close(st[3:6], ref.hi, "hi")
+            pr.assert_close(st[6:9], ref.delta, "delta")
+            pr.assert_close(st[9:12], ref.w, "w")
+            pr.assert_close(st[12:15], [ref.s_min, ref.s_max, ref.s_mean], "surprise stats")
+            pr.assert_close(a_star[0, h].cpu().numpy(), ref.a_star, "a_star")
+        assert st[15] == ref.m
+        assert torch.isinf(a_star[0, h, :min(4, N)]).all()
+
+
+@pytest.mark.parametrize("gate,window,n_sink,prior", [
+    (nkv.NKV_GATE_AVERAGE, 64, 4, (0.4, 0.4, 0.2)), (nkv.NKV_GATE_MAX, 64, 0, (0.4, 0.4, 0.2)),
+    (nkv.NKV_GATE_SURPRISE, 1, 4, (0.2, 0.3, 0.5)), (nkv.NKV_GATE_SURPRISE, 17, 8, (0.4, 0.4, 0.2)),
+    (nkv.NKV_GATE_SURPRISE, 40, 16, (0.6, 0.3, 0.1))])
+def test_score_parameter_switches(gate, window, n_sink, prior):
+    K, _ = _cache(777, 128, "bf16")
+    p = nkv.nkv_default_params()
+    p.gate_mode, p.window, p.n_sink = gate, window, n_sink
+    p.block_div, p.block_min, p.block_max = 64, 64, 128
+    p.beta, p.tau, p.kappa = 2.0, 0.3, 6.0
+    for k in range(3):
+        p.prior[k] = prior[k]
+    mu_s, mu_e, inv_norm, _ = nkv.nkv_anchors(K, p)
+    a_star, a_raw, _ = nkv.nkv_score(K, mu_s, mu_e, inv_norm, p, want_raw=True)
+    torch.cuda.synchronize()
+    for h in range(K.shape[1]):
+        ref = oracle.score_head(K[0, h].cpu(), pr.oracle_params(p))
+        pr.assert_close(a_raw[0, h].cpu().numpy(), ref.a_raw, "a_raw")
+        pr.assert_close(a_star[0, h].cpu().numpy(), ref.a_star, "a_star")
+
+
+def _random_scores(G, H, N, seed, ties):
+    rng = np.random.default_rng(seed)
+    s = rng.random((G, H, N)).astype(np.float32) ** 3
+    s *= rng.uniform(0.05, 1.0, size=(G, H, 1)).astype(np.float32)
+    if ties == "many":
+        s = np.round(s * 16) / 16
+    elif ties == "all":
+        s[:] = 0.25
+    elif ties == "dense":          # bulk packed into a sliver of [0,1], like real scores
+        s = (0.05 + 0.001 * s).astype(np.float32)
+    s[:, :, :4] = np.inf
+    return s
+
+
+@pytest.mark.parametrize("G,H,N,r,ties", [
+    (1, 1, 10, 0.5, "none"), (2, 3, 100, 0.75, "none"), (1, 8, 1000, 0.75, "many"), (2, 4, 5000, 0.95, "dense"),
+    (1, 8, 3000, 0.5, "all"), (1, 2, 4097, 0.0, "none"), (3, 8, 2048, 0.9, "dense"), (1, 5, 40, 0.95, "none")])
+def test_budget_and_select_bit_exact_on_oracle_scores(G, H, N, r, ties):
+    s = _random_scores(G, H, N, seed=N + H, ties=ties)
+    a_star = torch.from_numpy(s).to(DEV)
+    budgets = nkv.nkv_budget(a_star, r)
+    k = nkv.nkv_keep_per_head(N, r)
+    idx, offs, ranks = nkv.nkv_select(a_star, budgets, H * k, want_ranks=(N <= 5000))
+    torch.cuda.synchronize()
+    for g in range(G):
+        ref = oracle.budget_select(s[g], r, want_ranks=True)
+        assert np.array_equal(budgets[g].cpu().numpy(), ref.budgets)
+        assert np.array_equal(offs[g].cpu().numpy(), ref.offsets)
+        assert np.array_equal(idx[g].cpu().numpy(), ref.idx)
+        if ranks is not None:
+            assert np.array_equal(ranks[g].cpu().numpy(), ref.ranks)
+
+
+def test_safeguard_one_gives_uniform_budgets():
+    s = _random_scores(2, 4, 600, seed=3, ties="none")
+    p = nkv.nkv_default_params()
+    p.safeguard = 1.0
+    budgets = nkv.nkv_budget(torch.from_numpy(s).to(DEV), 0.75, p)
+    assert budgets.cpu().tolist() == [[150] * 4] * 2
+
+
+@pytest.mark.parametrize("d,dv,dtype,mode", [(128, 128, "bf16", "out"), (64, 64, "fp32", "out"),
+                                             (128, 128, "fp32", "in"), (64, 64, "bf16", "in")])
+def test_compaction_copies_rows_verbatim(d, dv, dtype, mode):
+    K, V = _cache(900, d, dtype, H=3, layers=2)
+    s = _random_scores(2, 3, 900, seed=5, ties="none")
+    sel = [oracle.budget_select(s[g], 0.6) for g in range(2)]
+    idx = torch.from_numpy(np.stack([x.idx for x in sel])).to(DEV)
+    offs = torch.from_numpy(np.stack([x.offsets for x in sel])).to(DEV)
+    Kr, Vr = pr.raw_rows(K), pr.raw_rows(V)
+    if mode == "out":
+        K_out, V_out = nkv.nkv_compact(K, V, idx, offs)
+        torch.cuda.synchronize()
+        for g in range(2):
+            assert np.array_equal(pr.raw_rows(K_out[g]), oracle.compact(K[g].cpu(), sel[g].idx, sel[g].offsets))
+            assert np.array_equal(pr.raw_rows(V_out[g]), oracle.compact(V[g].cpu(), sel[g].idx, sel[g].offsets))
+    else:
+        Kc, Vc = K.clone(), V.clone()
+        nkv.nkv_compact(Kc, Vc, idx, offs, mode=nkv.NKV_IN_PLACE)
+        torch.cuda.synchronize()
+        Kg, Vg = pr.raw_rows(Kc), pr.raw_rows(Vc)
+        for g in range(2):
+            for h in range(3):
+                rows = sel[g].idx[sel[g].offsets[h]:sel[g].offsets[h + 1]]
+                assert np.array_equal(Kg[g, h, :len(rows)], Kr[g, h][rows])
+                assert np.array_equal(Vg[g, h, :len(rows)], Vr[g, h][rows])
+
+
+@pytest.mark.parametrize("N,d,dtype,H,layers,r", [
+    (5, 64, "fp32", 2, 1, 0.5), (300, 64, "bf16", 4, 2, 0.75), (1000, 128, "fp32", 8, 1, 0.5),
+    (2500, 128, "bf16", 8, 2, 0.95), (4133, 64, "bf16", 3, 1, 0.0), (777, 128, "bf16", 1, 3, 0.9)])
+def test_fused_compress_end_to_end(N, d, dtype, H, layers, r):
+    K, V = _cache(N, d, dtype, H=H, layers=layers)
+    p = nkv.nkv_default_params()
+    ws = nkv.alloc_workspace(K, p)
+    res = nkv.nkv_compress(K, V, r, p, ws=ws, want_a_star=True)
+    assert nkv.nkv_last_device_status(ws) == nkv.NKV_OK
+    rep = pr.SwapReport()
+    for g in range(K.shape[0]):
+        pr.check_group_against_oracle(K, V, res, g, r, p, rep)
+    assert rep.swapped_tokens <= max(2, rep.heads)   # near-tie swaps are rare at fp32 accuracy
+
+
+def test_identical_keys_take_the_tie_path():
+    """All keys equal: every score is 0 and every selection is decided by position alone."""
+    K = torch.ones((1, 2, 3000, 64), dtype=torch.bfloat16, device=DEV)
+    V = torch.randn((1, 2, 3000, 64), device=DEV).to(torch.bfloat16)
+    ws = nkv.alloc_workspace(K)
+    res = nkv.nkv_compress(K, V, 0.75, ws=ws, want_a_star=True)
+    assert nkv.nkv_last_device_status(ws) == nkv.NKV_OK
+    a = res.a_star.cpu().numpy()
+    assert np.isinf(a[0, :, :4]).all() and (a[0, :, 4:] == 0).all()
+    ref = oracle.budget_select(a[0], 0.75)
+    assert np.array_equal(res.budgets[0].cpu().numpy(), ref.budgets)
+    assert np.array_equal(res.idx[0].cpu().numpy(), ref.idx)
+
+
+def test_strided_heads_outermost_layout():
+    """A [H, G, N, d] allocation viewed as [G, H, N, d]: strides, not copies."""
+    K, V = _cache(600, 128, "bf16", H=3, layers=2)
+    Kt = K.permute(1, 0, 2, 3).contiguous().permute(1, 0, 2, 3)
+    Vt = V.permute(1, 0, 2, 3).contiguous().permute(1, 0, 2, 3)
+    assert not Kt.is_contiguous()
+    a = nkv.nkv_compress(K, V, 0.75, want_a_star=True)
+    b = nkv.nkv_compress(Kt, Vt, 0.75, want_a_star=True)
+    torch.cuda.synchronize()
+    assert torch.equal(a.idx, b.idx) and torch.equal(a.k_out, b.k_out) and torch.equal(a.v_out, b.v_out)
+    assert torch.equal(a.a_star, b.a_star)
+
+
+def test_argument_errors_are_reported_not_thrown():
+    K, V = _cache(100, 64, "fp32")
+    with pytest.raises(nkv.NkvError) as e:
+        nkv.nkv_compress(K, V, 1.0)
+    assert e.value.status == nkv.NKV_ERR_INVALID_ARG
+    with pytest.raises(nkv.NkvError) as e:
+        nkv.nkv_compress(K, V, 0.999)      # k = 0
+    assert e.value.status == nkv.NKV_ERR_INVALID_ARG
+    with pytest.raises(nkv.NkvError) as e:
+        nkv.nkv_compress(K[..., :48].contiguous(), V[..., :48].contiguous(), 0.5)
+    assert e.value.status == nkv.NKV_ERR_UNSUPPORTED
+    p = nkv.nkv_default_params()
+    p.window = 65
+    with pytest.raises(nkv.NkvError) as e:
+        nkv.nkv_compress(K, V, 0.5, p)
+    assert e.value.status == nkv.NKV_ERR_UNSUPPORTED
+    with pytest.raises(nkv.NkvError) as e:
+        nkv.nkv_compress(K, V, 0.5, ws=torch.empty(1024, dtype=torch.uint8, device=DEV))
+    assert e.value.status == nkv.NKV_ERR_WORKSPACE
+    with pytest.raises(nkv.NkvError) as e:
+        nkv.nkv_compress(K.half(), V.half(), 0.5)
+    assert e.value.status == nkv.NKV_ERR_UNSUPPORTED
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    K, V = _cache(1500, 128, "bf16", H=4, layers=5)
+    dev = nkv.nkv_compress(K, V, 0.75)
+    torch.cuda.synchronize()
+    Kh, Vh = K.cpu().pin_memory(), V.cpu().pin_memory()
+    G, H, N, d = K.shape
+    k = nkv.nkv_keep_per_head(N, 0.75)
+    out = nkv.Compressed(torch.empty((G, H * k, d), dtype=K.dtype).pin_memory(),
+                         torch.empty((G, H * k, d), dtype=K.dtype).pin_memory(),
+                         torch.empty((G, H * k), dtype=torch.int32).pin_memory(),
+                         torch.empty((G, H + 1), dtype=torch.int32).pin_memory(),
+                         torch.empty((G, H), dtype=torch.int32).pin_memory(), None)
+    nbytes = nkv.nkv_host_staging_bytes(H, N, d, nkv.NKV_BF16, 0.75, 2)
+    staging = torch.empty(nbytes, dtype=torch.uint8, device=DEV)
+    nkv.nkv_compress_host(Kh, Vh, 0.75, out, staging, 2)
+    assert torch.equal(out.idx, dev.idx.cpu()) and torch.equal(out.budgets, dev.budgets.cpu())
+    assert torch.equal(out.head_offsets, dev.head_offsets.cpu())
+    assert torch.equal(out.k_out, dev.k_out.cpu()) and torch.equal(out.v_out, dev.v_out.cpu())
