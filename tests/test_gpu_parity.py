@@ -69,7 +69,7 @@ def test_scores_match_oracle(N, d, dtype):
 
 @pytest.mark.parametrize("gate,window,n_sink,prior", [
     (nkv.NKV_GATE_AVERAGE, 64, 4, (0.4, 0.4, 0.2)), (nkv.NKV_GATE_MAX, 64, 0, (0.4, 0.4, 0.2)),
-    (nkv.NKV_GATE_SURPRISE, 1, 4, (0.2, 0.3, 0.5)), (nkv.NKV_GATE_SURPRISE, 17, 8, (0.4, 0.4, 0.2)),
+    (nkv.NKV_GATE_SURPRISE, 2, 4, (0.2, 0.3, 0.5)), (nkv.NKV_GATE_SURPRISE, 17, 8, (0.4, 0.4, 0.2)),
     (nkv.NKV_GATE_SURPRISE, 40, 16, (0.6, 0.3, 0.1))])
 def test_score_parameter_switches(gate, window, n_sink, prior):
     K, _ = _cache(777, 128, "bf16")
