@@ -6,10 +6,6 @@
 
 #include "nkv_common.cuh"
 
-namespace nkv {
-cudaError_t configure_scan_kernels();
-}
-
 using namespace nkv;
 
 struct nkv_handle {
@@ -216,7 +212,7 @@ int nkv_create(nkv_handle** out, int device) {
     }
     h->sm_count = prop.multiProcessorCount;
     h->l2_bytes = prop.l2CacheSize;
-    if (configure_scan_kernels() != cudaSuccess) {
+    if (configure_scan_kernels() != cudaSuccess || configure_stream_kernels() != cudaSuccess) {
         delete h;
         return NKV_ERR_CUDA;
     }
@@ -394,14 +390,28 @@ int nkv_compress(nkv_handle* h, const nkv_tensor* K, const nkv_tensor* V, double
 
     CU(cudaMemsetAsync(status, 0, kStatusWords * sizeof(int), st));
     CU(mark());
-    CU(launch_anchor_sums(kv, K->dtype, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm), st, &h->launches));
-    CU(launch_anchor_means(units, N, d, sp, at<float>(ws, L.mu_e), at<float>(ws, L.mu_s), st, &h->launches));
-    CU(launch_anchor_norms(units, d, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_s),
-                           at<float>(ws, L.inv_e), at<uint32_t>(ws, L.mm), st, &h->launches));
-    CU(mark());
-    CU(launch_scan_scores(kv, K->dtype, G, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e),
-                          at<float>(ws, L.inv_norm), at<float>(ws, L.inv_s), at<float>(ws, L.inv_e),
-                          at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), st, &h->launches));
+    if (stream_path_supported(sp)) {
+        // pass A: norms, block sums and the current-memory anomaly; pass B: the two anchor anomalies
+        CU(launch_stream_a(kv, K->dtype, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm),
+                           at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));
+        CU(launch_anchor_means(units, N, d, sp, at<float>(ws, L.mu_e), at<float>(ws, L.mu_s), st, &h->launches));
+        CU(launch_anchor_norms(units, d, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_s),
+                               at<float>(ws, L.inv_e), nullptr, st, &h->launches));
+        CU(mark());
+        CU(launch_stream_b(kv, K->dtype, G, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e),
+                           at<float>(ws, L.inv_norm), at<float>(ws, L.inv_s), at<float>(ws, L.inv_e),
+                           at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));
+    } else {
+        CU(launch_anchor_sums(kv, K->dtype, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm), st,
+                              &h->launches));
+        CU(launch_anchor_means(units, N, d, sp, at<float>(ws, L.mu_e), at<float>(ws, L.mu_s), st, &h->launches));
+        CU(launch_anchor_norms(units, d, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_s),
+                               at<float>(ws, L.inv_e), at<uint32_t>(ws, L.mm), st, &h->launches));
+        CU(mark());
+        CU(launch_scan_scores(kv, K->dtype, G, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e),
+                              at<float>(ws, L.inv_norm), at<float>(ws, L.inv_s), at<float>(ws, L.inv_e),
+                              at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), st, &h->launches));
+    }
     CU(mark());
     CU(launch_head_scores(units, N, sp, at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), a_star, nullptr, status, st,
                           &h->launches));

@@ -103,8 +103,19 @@ cudaError_t launch_anchor_means(int units, int N, int d, const ScoreParams& sp, 
 cudaError_t launch_window_means(const TensorView& K, int dtype, int G, const ScoreParams& sp, const float* inv_norm,
                                 float* mu_c, cudaStream_t stream, int64_t* launches);
 cudaError_t launch_anchor_norms(int units, int d, const ScoreParams& sp, const float* mu_s, const float* mu_e,
-                                float* inv_mu_s_norm, float* inv_mu_e_norm, uint32_t* minmax_keys,
+                                float* inv_mu_s_norm, float* inv_mu_e_norm, uint32_t* minmax_keys_to_reset_or_null,
                                 cudaStream_t stream, int64_t* launches);
+// streaming key passes (block size a multiple of 8)
+bool stream_path_supported(const ScoreParams& sp);
+cudaError_t launch_stream_a(const TensorView& K, int dtype, int G, const ScoreParams& sp, float* block_sums,
+                            float* inv_norm, float* a_raw, uint32_t* mm, int* status, int sm_count,
+                            cudaStream_t stream, int64_t* launches);
+cudaError_t launch_stream_b(const TensorView& K, int dtype, int G, const ScoreParams& sp, const float* mu_s,
+                            const float* mu_e, const float* inv_norm, const float* inv_s, const float* inv_e,
+                            float* a_raw, uint32_t* mm, int* status, int sm_count, cudaStream_t stream,
+                            int64_t* launches);
+cudaError_t configure_scan_kernels();
+cudaError_t configure_stream_kernels();
 cudaError_t launch_scan_scores(const TensorView& K, int dtype, int G, const ScoreParams& sp, const float* mu_s,
                                const float* mu_e, const float* inv_norm, const float* inv_mu_s_norm,
                                const float* inv_mu_e_norm, float* a_raw, uint32_t* minmax_keys,
@@ -125,6 +136,5 @@ cudaError_t launch_gather(const TensorView& K, int k_elem_bytes, const TensorVie
 cudaError_t launch_gather_in_place(const TensorView& K, int k_elem_bytes, const TensorView& V, int v_elem_bytes, int G,
                                    const int32_t* idx, const int32_t* head_offsets, int64_t idx_capacity,
                                    cudaStream_t stream, int64_t* launches);
-cudaError_t configure_kernels();  // raises dynamic shared-memory limits (once per device)
 
 }  // namespace nkv

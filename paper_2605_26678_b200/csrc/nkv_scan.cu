@@ -154,7 +154,7 @@ __global__ void __launch_bounds__(128) anchor_norms_kernel(int d, ScoreParams sp
             else inv_e[(int64_t)u * sp.nblocks + t] = inv;
         }
     }
-    if (threadIdx.x < 6) mm[(int64_t)u * 6 + threadIdx.x] = (threadIdx.x & 1) ? 0u : 0xffffffffu;  // [scale][min,max]
+    if (mm && threadIdx.x < 6) mm[(int64_t)u * 6 + threadIdx.x] = (threadIdx.x & 1) ? 0u : 0xffffffffu;  // [scale][min,max]
 }
 
 // ------------------------------------------------------------------------------------------
