@@ -124,6 +124,22 @@ def physical_gpu_index(local: int) -> int:
     return local
 
 
+def replica_config(cfg, rank):
+    """The cache a rank owns: same shape on every rank, different sequences (independent replicas)."""
+    if rank == 0:
+        return cfg
+    return wl.CacheConfig(**{**cfg.__dict__, "base_seed": cfg.base_seed + 977 * rank})
+
+
+def whole_job_throughput(ms_local, steps, keys_per_rank, world, dist=None, device="cpu"):
+    """(keys/s over all ranks, ms per step): the slowest rank's time bounds the job."""
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    if dist is not None and world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_per_step = float(t.item()) / steps
+    return keys_per_rank * world / (ms_per_step * 1e-3), ms_per_step
+
+
 def algorithmic_bytes(cfg, r):
     """Bytes the method must move through HBM for one step (per GPU)."""
     from paper_2605_26678_b200 import nkv
@@ -220,7 +236,7 @@ def run_nkv(args, cfg, r):
         torch.cuda.synchronize()
 
     # every rank owns an independent cache of the same shape (different sequences)
-    my_cfg = cfg if rank == 0 else wl.CacheConfig(**{**cfg.__dict__, "base_seed": cfg.base_seed + 977 * rank})
+    my_cfg = replica_config(cfg, rank)
     K, V = wl.make_cache(my_cfg, dev, groups_per_call=4)
     params = nkv.nkv_default_params()
     ws = nkv.alloc_workspace(K, params)
@@ -250,13 +266,7 @@ def run_nkv(args, cfg, r):
     status = nkv.nkv_last_device_status(ws, h)
     if status != nkv.NKV_OK:
         raise SystemExit("device status %d after the timed region" % status)
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
-    ms_per_step = ms_total / args.steps
-    keys_per_step = cfg.keys * world
-    value = keys_per_step / (ms_per_step * 1e-3)
+    value, ms_per_step = whole_job_throughput(ms_total, args.steps, cfg.keys, world, dist, dev)
 
     # ---- per-stage device time (events recorded on the launching stream inside the library) --
     nkv.nkv_set_timing(True, h)
