@@ -247,6 +247,33 @@ NKV_API int nkv_get_stage_ms(nkv_handle* h, float* ms_out);
 /* Number of kernels this handle has launched since creation. */
 NKV_API int64_t nkv_launch_count(const nkv_handle* h);
 
+/*
+ * nkv_budget for callers that cannot allocate device memory (the paper has no
+ * counterpart: this is a packaging variant of nkv_budget, same arithmetic,
+ * same kernel).  A host that runs inside a memory pool fixed at start-up, a
+ * plugin that receives nothing but its inputs and outputs, or a step that runs
+ * while the process may not grow its footprint has no scratch buffer to hand
+ * to nkv_budget.  Here the scratch (status words and the per-head selection
+ * thresholds, 256 + 8 * NKV_STATIC_MAX_UNITS bytes) is a fixed array inside
+ * the library image; every GPU that loads the library holds it until the
+ * process exits.  No handle and no workspace are needed, and the call makes no
+ * cudaMalloc, cudaFree or other allocating call.
+ *   a_star, r, params, budgets, stream   exactly as in nkv_budget
+ *   G * H <= NKV_STATIC_MAX_UNITS, otherwise NKV_ERR_WORKSPACE is returned and
+ *   nothing is launched (use nkv_budget with your own workspace instead).
+ * The first call made with a given device current looks up the array's device
+ * address (once per device); make that first call before any stream capture.
+ * All calls on a device share the one array, which still holds what the last
+ * call left: the status words are cleared on the stream at the start of each
+ * call, the threshold slots of the call's G * H heads are all rewritten.  Two
+ * calls whose work overlaps on the GPU (different streams) race on the array:
+ * keep calls on one device ordered.  Device-side self-check results are not
+ * readable through this entry point.
+ */
+#define NKV_STATIC_MAX_UNITS 4096
+NKV_API int nkv_budget_static(const float* a_star, int64_t G, int64_t H, int64_t N, double r,
+                              const nkv_params* params, int32_t* budgets, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

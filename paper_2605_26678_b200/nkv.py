@@ -28,6 +28,7 @@ NKV_GATE_SURPRISE, NKV_GATE_AVERAGE, NKV_GATE_MAX = 0, 1, 2
 NKV_OUT_OF_PLACE, NKV_IN_PLACE = 0, 1
 NKV_HEAD_STATS = 16
 NKV_NUM_STAGES = 6
+NKV_STATIC_MAX_UNITS = 4096
 STAGE_NAMES = ("anchors", "score", "head", "budget", "select", "compact")
 
 EXPORTS = (
@@ -35,7 +36,7 @@ EXPORTS = (
     "nkv_keep_per_head", "nkv_safeguard_count", "nkv_top_count", "nkv_create", "nkv_destroy",
     "nkv_workspace_bytes", "nkv_anchors", "nkv_score", "nkv_budget", "nkv_select", "nkv_compact",
     "nkv_compress", "nkv_host_staging_bytes", "nkv_compress_host", "nkv_last_device_status",
-    "nkv_set_timing", "nkv_get_stage_ms", "nkv_launch_count",
+    "nkv_set_timing", "nkv_get_stage_ms", "nkv_launch_count", "nkv_budget_static",
 )
 
 
@@ -110,6 +111,7 @@ def load_library():
     L.nkv_get_stage_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     L.nkv_launch_count.argtypes = [vp]
     L.nkv_launch_count.restype = i64
+    L.nkv_budget_static.argtypes = [vp, i64, i64, i64, dbl, pp, vp, vp]
     _lib = L
     return L
 
@@ -280,6 +282,24 @@ def nkv_budget(a_star: torch.Tensor, r: float, params: Optional[Params] = None,
     ws = ws if ws is not None else torch.empty(4096 + 16 * G * H, dtype=torch.uint8, device=a_star.device)
     _check(h.lib.nkv_budget(h.h, _p(a_star), G, H, N, float(r), ctypes.byref(params), _p(budgets), _p(ws),
                             ws.numel(), _stream()), "nkv_budget")
+    return budgets
+
+
+def nkv_budget_static(a_star: torch.Tensor, r: float, params: Optional[Params] = None,
+                      out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """a_star [G,H,N] f32 -> budgets [G,H] i32, for callers that cannot allocate device memory.
+
+    The C call takes no handle and no workspace: its scratch is a fixed array inside the library
+    (at most NKV_STATIC_MAX_UNITS heads per call).  Pass `out` (an int32 [G,H] CUDA tensor you
+    already own) and this wrapper allocates nothing either; without `out` it creates the result
+    tensor for convenience.  Calls on one device share that scratch, so keep them stream-ordered."""
+    params = params or nkv_default_params()
+    if not a_star.is_contiguous():
+        raise NkvError(NKV_ERR_INVALID_ARG, "nkv_budget_static: a_star must be contiguous")
+    G, H, N = a_star.shape
+    budgets = out if out is not None else torch.empty((G, H), dtype=torch.int32, device=a_star.device)
+    _check(load_library().nkv_budget_static(_p(a_star), G, H, N, float(r), ctypes.byref(params), _p(budgets),
+                                            _stream()), "nkv_budget_static")
     return budgets
 
 
