@@ -1,0 +1,412 @@
+// Fused key scan of the compression path (Sections 2.1-2.3): one persistent kernel that makes both
+// passes over the keys, interleaved head by head so that the second pass finds the keys in L2.
+//
+//   pass A (needs no anchor)   1/||k_i||, sums of normalised keys per 8-row segment and per episodic
+//                              block, the current-memory anomaly a_c(i) and its per-head min/max
+//   finalize (once per head)   stable mean, block means, reciprocal norms of the anchors; done by the
+//                              CTA that finishes the head's last pass-A tile
+//   pass B (needs the anchors) a_s(i), a_e(i) and their per-head min/max
+//
+// Work items are handed out in ticket order: for every step s, the tiles of A(head s), then the tiles
+// of B(head s - lag).  A pass-B item waits (bounded) for its head's anchors; every pass-A item it
+// depends on carries an earlier ticket and never waits, and a CTA pays the anchors it owes before it
+// waits itself, so the order cannot deadlock.
+//
+// A row of d elements is split over 8 lanes (16-byte chunks l, l+8, ...), so a quarter warp reads 128
+// contiguous bytes of shared memory.  Each 8-lane group owns one 8-row segment; per-token partial
+// sums are combined with a transposed shuffle reduction that leaves token l with lane l, which then
+// writes its result straight to global memory (32 contiguous bytes per group).  The sliding-window
+// sum is a running sum over the 8 tokens of a group, seeded from exact segment sums, so no long
+// prefix is ever differenced.  Key tiles are staged with bulk asynchronous copies, double buffered,
+// issued by a control warp that also does the per-item bookkeeping (tickets, tile counters, min/max
+// publication) so that the compute threads never wait for a global atomic.
+#include "nkv_common.cuh"
+
+namespace nkv {
+
+namespace {
+
+constexpr int kHalo = kMaxWindow;
+constexpr uint32_t kSpinLimit = 1u << 24;
+constexpr unsigned long long kWaitLimitNs = 2000000000ULL;   // every device-side wait gives up after 2 s
+constexpr int kLanes = 8;
+
+// control words (ints) in the workspace: [0..1] 64-bit ticket counter, [8 + u] tiles of head u
+// finished by pass A, [8 + units + u] anchors of head u published
+constexpr int kCtrlHeader = 8;
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_keep() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_normal() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_stream() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_global, uint32_t bytes, uint64_t* bar,
+                                          uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+            smem_addr(dst_smem)),
+        "l"(src_global), "r"(bytes), "r"(smem_addr(bar)), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long now_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait for a bulk copy; gives up at once when the CTA has already recorded a failure.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = now_ns();
+    for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 63u) == 63u &&
+            (*reinterpret_cast<const volatile int*>(abort_flag) != 0 || now_ns() - t0 > kWaitLimitNs))
+            return false;
+    }
+    return false;
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ int ld_acquire(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release(int* p, int v) {
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void bar_sync(int id, int count) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+constexpr int kBarCompute = 1;   // the compute threads only
+constexpr int kBarEnd = 2;       // compute threads + control warp, once per item
+
+// ---------------------------------------------------------------------------- packed fp32 helpers
+struct F2 {
+    unsigned long long v;
+};
+__device__ __forceinline__ F2 pack2(float a, float b) {
+    F2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r.v) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack2(F2 x, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(x.v)); }
+__device__ __forceinline__ F2 fma2(F2 a, F2 b, F2 c) {
+    F2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r.v) : "l"(a.v), "l"(b.v), "l"(c.v));
+    return r;
+}
+__device__ __forceinline__ F2 add2(F2 a, F2 b) {
+    F2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v));
+    return r;
+}
+__device__ __forceinline__ float hsum2(F2 x) {
+    float a, b;
+    unpack2(x, a, b);
+    return a + b;
+}
+
+template <typename T> struct Pairs;
+template <> struct Pairs<__nv_bfloat16> {
+    static constexpr int kPairs = 4;   // per 16-byte chunk
+    __device__ __forceinline__ static void unpack(const uint4& q, F2* p) {
+        p[0] = pack2(__uint_as_float(q.x << 16), __uint_as_float(q.x & 0xffff0000u));
+        p[1] = pack2(__uint_as_float(q.y << 16), __uint_as_float(q.y & 0xffff0000u));
+        p[2] = pack2(__uint_as_float(q.z << 16), __uint_as_float(q.z & 0xffff0000u));
+        p[3] = pack2(__uint_as_float(q.w << 16), __uint_as_float(q.w & 0xffff0000u));
+    }
+};
+template <> struct Pairs<float> {
+    static constexpr int kPairs = 2;
+    __device__ __forceinline__ static void unpack(const uint4& q, F2* p) {
+        p[0] = pack2(__uint_as_float(q.x), __uint_as_float(q.y));
+        p[1] = pack2(__uint_as_float(q.z), __uint_as_float(q.w));
+    }
+};
+
+// Geometry for element type T and head dimension D with 8 lanes per row.
+template <typename T, int D>
+struct Geo {
+    static constexpr int kRowBytes = D * (int)sizeof(T);
+    static constexpr int kChunks = kRowBytes / 128;            // 16-byte chunks per lane
+    static constexpr int kPerChunk = 16 / (int)sizeof(T);      // elements per chunk
+    static constexpr int kCols = D / kLanes;                   // columns per lane
+    static constexpr int kNP = kCols / 2;                      // packed pairs per lane
+    static constexpr int kTile = 65536 / kRowBytes;            // rows per tile (64 KB of keys)
+    static constexpr int kRows = kTile + kHalo;
+    static constexpr int kSegs = kRows / kSeg;
+    static constexpr int kThreads = kSegs * kLanes;            // compute threads (== kRows)
+    static constexpr size_t kTileBytes = (size_t)kRows * kRowBytes;
+    static constexpr size_t kSmem = 2 * kTileBytes + (size_t)kSegs * D * 4 + (size_t)kRows * 4 + 128;
+    static_assert(kChunks >= 1 && kThreads % 32 == 0 && kThreads + 32 <= 1024, "bad geometry");
+
+    __device__ __forceinline__ static int col0(int l, int j) { return (l + kLanes * j) * kPerChunk; }
+    __device__ __forceinline__ static void load_row(const unsigned char* row, int l, F2* p) {
+#pragma unroll
+        for (int j = 0; j < kChunks; ++j) {
+            const uint4 q = *reinterpret_cast<const uint4*>(row + (l + kLanes * j) * 16);
+            Pairs<T>::unpack(q, p + j * Pairs<T>::kPairs);
+        }
+    }
+    // the lane's columns of an fp32 vector laid out by column
+    __device__ __forceinline__ static void load_vec(const float* vec, int l, F2* p) {
+#pragma unroll
+        for (int j = 0; j < kChunks; ++j)
+#pragma unroll
+            for (int e = 0; e < kPerChunk; e += 4) {
+                const float4 f = *reinterpret_cast<const float4*>(vec + col0(l, j) + e);
+                p[(j * kPerChunk + e) / 2] = pack2(f.x, f.y);
+                p[(j * kPerChunk + e) / 2 + 1] = pack2(f.z, f.w);
+            }
+    }
+    __device__ __forceinline__ static void store_vec(float* vec, int l, const F2* p) {
+#pragma unroll
+        for (int j = 0; j < kChunks; ++j)
+#pragma unroll
+            for (int e = 0; e < kPerChunk; e += 4) {
+                float4 f;
+                unpack2(p[(j * kPerChunk + e) / 2], f.x, f.y);
+                unpack2(p[(j * kPerChunk + e) / 2 + 1], f.z, f.w);
+                *reinterpret_cast<float4*>(vec + col0(l, j) + e) = f;
+            }
+    }
+};
+
+// Transposed reduction of V per-lane partial values over the 8 lanes of a group (V a power of two).
+// Afterwards, with V >= 8, lane l holds the complete sums of values l*(V/8) .. l*(V/8)+V/8-1 in
+// v[0 .. V/8); with V == 4, v[0] of lane l is the complete sum of value l/2.
+template <int V>
+__device__ __forceinline__ void treduce8(float* v, int l) {
+    int n = V;
+#pragma unroll
+    for (int o = kLanes / 2; o >= 1; o >>= 1) {
+        if (n > 1) {
+            const int half = n / 2;
+            const bool up = (l & o) != 0;
+#pragma unroll
+            for (int j = 0; j < V / 2; ++j) {
+                if (j < half) {
+                    const float send = up ? v[j] : v[j + half];
+                    const float keep = up ? v[j + half] : v[j];
+                    v[j] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+                }
+            }
+            n = half;
+        } else {
+            v[0] += __shfl_xor_sync(0xffffffffu, v[0], o);
+        }
+    }
+}
+
+struct FusedArgs {
+    TensorView K;
+    ScoreParams sp;
+    int units, lag, hints;
+    float* block_sums;   // [units, nb, d]: block sums, turned into block means (mu_e) by finalize
+    float* mu_s;         // [units, d]
+    float* inv_s;        // [units]
+    float* inv_e;        // [units, nb]
+    float* inv_norm;     // [units, N]
+    float* a_raw;        // [units, 3, N]
+    uint32_t* mm;        // [units, 6] ordered keys: min/max of a_s, a_e, a_c
+    int* ctrl;           // control words, see kCtrlHeader
+    int* status;
+};
+
+// item descriptor written by the control warp: kind 0 = pass A, 1 = pass B, 2 = no more work
+struct Item {
+    int kind, unit, tile, pad;
+};
+
+// sum over staged segments [s0, s1) of the per-segment sums, from inclusive prefixes within 64-row chunks
+template <typename T, int D>
+__device__ __forceinline__ void range_sum(const float* pp, int l, int s0, int s1, F2* out) {
+    using G = Geo<T, D>;
+#pragma unroll
+    for (int p = 0; p < G::kNP; ++p) out[p] = pack2(0.f, 0.f);
+    if (s1 <= s0) return;
+    for (int c = s0 >> 3; c <= (s1 - 1) >> 3; ++c) {
+        const int lo = max(s0, c * 8), hi = min(s1, c * 8 + 8);
+        F2 a[G::kNP];
+        G::load_vec(pp + (size_t)(hi - 1) * D, l, a);
+#pragma unroll
+        for (int p = 0; p < G::kNP; ++p) out[p] = add2(out[p], a[p]);
+        if (lo > c * 8) {
+            G::load_vec(pp + (size_t)(lo - 1) * D, l, a);
+            const F2 m1 = pack2(-1.f, -1.f);
+#pragma unroll
+            for (int p = 0; p < G::kNP; ++p) out[p] = fma2(a[p], m1, out[p]);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------- pass A on one tile
+template <typename T, int D>
+__device__ __forceinline__ void pass_a(const FusedArgs& A, int u, int tile_idx, unsigned char* tile, float* pp,
+                                       float* invs, uint32_t* mmk, uint64_t* full, uint32_t parity, int* abort_flag) {
+    using G = Geo<T, D>;
+    constexpr int NP = G::kNP;
+    const int N = A.K.N, W = A.sp.window;
+    const int tid = threadIdx.x, grp = tid >> 3, l = tid & 7;
+    const int i0 = tile_idx * G::kTile;
+
+    // rows outside [0, N) are not copied: zero them (disjoint from the bytes in flight)
+    const int r0 = max(0, i0 - kHalo), r1 = min(N, i0 + G::kTile);
+    const bool fill = (r0 != i0 - kHalo) || (r1 != i0 + G::kTile);
+    if (fill) {
+        const int head_rows = r0 - (i0 - kHalo), tail_row0 = r1 - (i0 - kHalo);
+        constexpr int cpr = G::kRowBytes / 16;
+        const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+        for (int c = tid; c < head_rows * cpr; c += G::kThreads) reinterpret_cast<uint4*>(tile)[c] = z;
+        for (int c = tail_row0 * cpr + tid; c < G::kRows * cpr; c += G::kThreads) reinterpret_cast<uint4*>(tile)[c] = z;
+    }
+    if (!mbar_wait(full, parity, abort_flag)) {
+        set_status(A.status, NKV_ERR_TIMEOUT, 501);
+        *abort_flag = 1;
+    }
+    if (fill) bar_sync(kBarCompute, G::kThreads);
+
+    // ---- S1: reciprocal norms and the sum of normalised keys of every staged 8-row segment
+    {
+        F2 acc[NP];
+#pragma unroll
+        for (int p = 0; p < NP; ++p) acc[p] = pack2(0.f, 0.f);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            F2 x[4][NP];
+            float n2[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                G::load_row(tile + (size_t)(grp * kSeg + half * 4 + r) * G::kRowBytes, l, x[r]);
+                F2 s = pack2(0.f, 0.f);
+#pragma unroll
+                for (int p = 0; p < NP; ++p) s = fma2(x[r][p], x[r][p], s);
+                n2[r] = hsum2(s);
+            }
+            treduce8<4>(n2, l);   // lane l: squared norm of row l/2 of this half
+            const float inv = 1.0f / fmaxf(sqrtf(n2[0]), kEps);
+            if ((l & 1) == 0) {
+                const int sr = grp * kSeg + half * 4 + (l >> 1);
+                invs[sr] = inv;
+                const int gi = i0 - kHalo + sr;
+                if (sr >= kHalo && gi < N) A.inv_norm[(int64_t)u * N + gi] = inv;
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const float ir = __shfl_sync(0xffffffffu, inv, 2 * r, kLanes);
+                const F2 ir2 = pack2(ir, ir);
+#pragma unroll
+                for (int p = 0; p < NP; ++p) acc[p] = fma2(x[r][p], ir2, acc[p]);
+            }
+        }
+        G::store_vec(pp + (size_t)grp * D, l, acc);
+    }
+    bar_sync(kBarCompute, G::kThreads);
+    // ---- S1b: inclusive prefix of the segment sums inside every 64-row chunk (one column per task)
+    for (int task = tid; task < (G::kRows / 64) * D; task += G::kThreads) {
+        const int c64 = task / D, col = task - c64 * D;
+        float run = 0.f;
+#pragma unroll
+        for (int p = 0; p < 8; ++p) {
+            float* q = pp + (size_t)(c64 * 8 + p) * D + col;
+            run += *q;
+            *q = run;
+        }
+    }
+    bar_sync(kBarCompute, G::kThreads);
+
+    // ---- S2: sliding-window anomaly of the tile's tokens
+    constexpr int kHaloSegs = kHalo / kSeg;
+    if (grp >= kHaloSegs) {
+        const int s = grp;
+        F2 Sw[NP];
+        range_sum<T, D>(pp, l, s - W / kSeg, s, Sw);
+        for (int sr = s * kSeg - W; sr < (s - W / kSeg) * kSeg; ++sr) {   // the W % 8 oldest rows
+            F2 x[NP];
+            G::load_row(tile + (size_t)sr * G::kRowBytes, l, x);
+            const float iv = invs[sr];
+            const F2 iv2 = pack2(iv, iv);
+#pragma unroll
+            for (int p = 0; p < NP; ++p) Sw[p] = fma2(x[p], iv2, Sw[p]);
+        }
+        float part[16];
+#pragma unroll
+        for (int o = 0; o < kSeg; ++o) {
+            const int sr = s * kSeg + o;
+            F2 kn[NP], ko[NP];
+            G::load_row(tile + (size_t)sr * G::kRowBytes, l, kn);
+            G::load_row(tile + (size_t)(sr - W) * G::kRowBytes, l, ko);
+            const float in = invs[sr], io = -invs[sr - W];
+            const F2 in2 = pack2(in, in), io2 = pack2(io, io);
+            F2 dc = pack2(0.f, 0.f), nc = pack2(0.f, 0.f);
+#pragma unroll
+            for (int p = 0; p < NP; ++p) {
+                F2 w = fma2(in2, kn[p], Sw[p]);
+                w = fma2(io2, ko[p], w);
+                Sw[p] = w;
+                dc = fma2(kn[p], w, dc);
+                nc = fma2(w, w, nc);
+            }
+            part[2 * o] = hsum2(dc);
+            part[2 * o + 1] = hsum2(nc);
+        }
+        treduce8<16>(part, l);   // lane l: (dc, nc) of token l
+        const int j = (s - kHaloSegs) * kSeg + l;
+        const float a_c = -(part[0] * invs[s * kSeg + l]) / fmaxf(sqrtf(part[1]), kEps) + 0.f;
+        float lo = INFINITY, hi = -INFINITY;
+        if (i0 + j < N) {
+            A.a_raw[((int64_t)u * 3 + 2) * N + i0 + j] = a_c;
+            lo = hi = a_c;
+        }
+        lo = warp_min(lo);
+        hi = warp_max(hi);
+        if ((tid & 31) == 0 && lo <= hi) {
+            atomicMin(&mmk[4], ord_key(lo));
+            atomicMax(&mmk[5], ord_key(hi));
+        }
+    }
+    // ---- sums of normalised keys of the episodic blocks inside this tile (one column per thread);
+    //      the tile size is a multiple of the block size, so every block is written by one tile
+    if (tid < D) {
+        const int b = A.sp.block;
+        const int row_end = min(N, i0 + G::kTile);
+        for (int blk = i0 / b; blk * b < row_end; ++blk) {
+            const int rlo = blk * b, rhi = min((blk + 1) * b, ((N + 7) / 8) * 8);
+            const int s0 = kHaloSegs + (rlo - i0) / kSeg, s1 = kHaloSegs + (rhi - i0 + kSeg - 1) / kSeg;
+            float sum = 0.f;
+            for (int c = s0 >> 3; c <= (s1 - 1) >> 3; ++c) {
+                const int a = max(s0, c * 8), e = min(s1, c * 8 + 8);
+                sum += pp[(size_t)(e - 1) * D + tid];
+                if (a > c * 8) sum -= pp[(size_t)(a - 1) * D + tid];
+            }
+            A.block_sums[((int64_t)u * A.sp.nblocks + blk) * D + tid] = sum;
+        }
+        __threadfence();   // the block sums must be visible before this tile is counted as finished
+    }
+}
