@@ -410,3 +410,162 @@ __device__ __forceinline__ void pass_a(const FusedArgs& A, int u, int tile_idx, 
         __threadfence();   // the block sums must be visible before this tile is counted as finished
     }
 }
+
+// ---------------------------------------------------------------------------- pass B on one tile
+// The first D threads stage the anchors in shared memory: `pp` = mu_s [D], then the block means of
+// the tile's blocks [nblk][D]; `invs` = 1/||mu_s|| at [0], 1/||mu_e|| of the tile's blocks at [1 ..].
+template <typename T, int D>
+__device__ __forceinline__ void pass_b(const FusedArgs& A, int u, int tile_idx, const unsigned char* tile, float* pp,
+                                       float* invs, uint32_t* mmk, uint64_t* full, uint32_t parity, int* abort_flag) {
+    using G = Geo<T, D>;
+    constexpr int NP = G::kNP;
+    const int N = A.K.N, b = A.sp.block, nb = A.sp.nblocks;
+    const int tid = threadIdx.x, grp = tid >> 3, l = tid & 7;
+    const int i0 = tile_idx * G::kTile;
+    const int blk0 = i0 / b;
+    const int nblk = min(nb - blk0, G::kTile / b);
+
+    if (tid < D) {
+        // wait (bounded) until the head's anchors have been published
+        const int* ready = A.ctrl + kCtrlHeader + A.units + u;
+        bool ok = ld_acquire(ready) != 0;
+        if (!ok && *reinterpret_cast<volatile int*>(abort_flag) == 0) {
+            const unsigned long long t0 = now_ns();
+            for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+                if (ld_acquire(ready) != 0) {
+                    ok = true;
+                    break;
+                }
+                __nanosleep(64);
+                if ((spin & 63u) == 63u && now_ns() - t0 > kWaitLimitNs) break;
+            }
+        }
+        if (!ok) {
+            set_status(A.status, NKV_ERR_TIMEOUT, 502);
+            *abort_flag = 1;
+        }
+        pp[tid] = __ldcg(A.mu_s + (int64_t)u * D + tid);
+        for (int q = 0; q < nblk; ++q) pp[(1 + q) * D + tid] = __ldcg(A.block_sums + ((int64_t)u * nb + blk0 + q) * D + tid);
+        if (tid == 0) invs[0] = __ldcg(A.inv_s + u);
+        if (tid >= 1 && tid <= nblk) invs[tid] = __ldcg(A.inv_e + (int64_t)u * nb + blk0 + tid - 1);
+    }
+    bar_sync(kBarCompute, G::kThreads);
+
+    const int gi0 = i0 + grp * kSeg;
+    const bool active = grp < G::kTile / kSeg && gi0 < N;
+    float inv_mine = 0.f;
+    F2 ms[NP], me[NP];
+    float rs = 0.f, re = 0.f;
+    if (active) {
+        const int q = min(gi0 / b, nb - 1) - blk0;
+        G::load_vec(pp, l, ms);
+        G::load_vec(pp + (1 + q) * D, l, me);
+        rs = invs[0];
+        re = invs[1 + q];
+        if (gi0 + l < N) inv_mine = __ldcg(A.inv_norm + (int64_t)u * N + gi0 + l);
+    }
+    if (!mbar_wait(full, parity, abort_flag)) {
+        set_status(A.status, NKV_ERR_TIMEOUT, 503);
+        *abort_flag = 1;
+    }
+    if (active) {
+        float part[16];
+#pragma unroll
+        for (int o = 0; o < kSeg; ++o) {
+            F2 kn[NP];
+            G::load_row(tile + (size_t)(grp * kSeg + o) * G::kRowBytes, l, kn);
+            F2 ds = pack2(0.f, 0.f), de = pack2(0.f, 0.f);
+#pragma unroll
+            for (int p = 0; p < NP; ++p) {
+                ds = fma2(kn[p], ms[p], ds);
+                de = fma2(kn[p], me[p], de);
+            }
+            part[2 * o] = hsum2(ds);
+            part[2 * o + 1] = hsum2(de);
+        }
+        treduce8<16>(part, l);   // lane l: (k_l . mu_s, k_l . mu_e)
+        const float a_s = -(part[0] * inv_mine) * rs + 0.f;
+        const float a_e = -(part[1] * inv_mine) * re + 0.f;
+        float lo_s = INFINITY, hi_s = -INFINITY, lo_e = INFINITY, hi_e = -INFINITY;
+        if (gi0 + l < N) {
+            A.a_raw[((int64_t)u * 3 + 0) * N + gi0 + l] = a_s;
+            A.a_raw[((int64_t)u * 3 + 1) * N + gi0 + l] = a_e;
+            lo_s = hi_s = a_s;
+            lo_e = hi_e = a_e;
+        }
+        lo_s = warp_min(lo_s);
+        hi_s = warp_max(hi_s);
+        lo_e = warp_min(lo_e);
+        hi_e = warp_max(hi_e);
+        if ((tid & 31) == 0 && lo_s <= hi_s) {
+            atomicMin(&mmk[0], ord_key(lo_s));
+            atomicMax(&mmk[1], ord_key(hi_s));
+            atomicMin(&mmk[2], ord_key(lo_e));
+            atomicMax(&mmk[3], ord_key(hi_e));
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------- anchors of one head
+// Block sums -> block means (in place), stable mean (compensated sums), reciprocal anchor norms.
+// Called by all compute threads of the CTA that finished the head's last pass-A tile.
+template <typename T, int D>
+__device__ __forceinline__ void finalize_head(const FusedArgs& A, int u, float* pp) {
+    using G = Geo<T, D>;
+    constexpr int kParts = G::kThreads / D;
+    const int N = A.K.N, b = A.sp.block, nb = A.sp.nblocks;
+    const int tid = threadIdx.x;
+    const int part = tid / D, c = tid - part * D;
+    float* bs = A.block_sums + (int64_t)u * nb * D;
+    if (part < kParts) {
+        const int per = (nb + kParts - 1) / kParts;
+        const int t0 = part * per, t1 = min(nb, t0 + per);
+        float sum = 0.f, comp = 0.f;
+        for (int t = t0; t < t1; ++t) {
+            const float s = __ldcg(bs + (size_t)t * D + c);
+            const float y = s - comp;
+            const float z = sum + y;
+            comp = (z - sum) - y;
+            sum = z;
+            const int cnt = min(N, (t + 1) * b) - t * b;
+            bs[(size_t)t * D + c] = s / (float)cnt;
+        }
+        pp[(2 * part) * D + c] = sum;
+        pp[(2 * part + 1) * D + c] = comp;
+    }
+    bar_sync(kBarCompute, G::kThreads);
+    if (tid < D) {
+        float sum = 0.f, comp = 0.f;
+        for (int p = 0; p < kParts; ++p) {
+            // add the partial sum, then its pending correction, both compensated
+            const float v[2] = {pp[(2 * p) * D + tid], -pp[(2 * p + 1) * D + tid]};
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const float y = v[k] - comp;
+                const float z = sum + y;
+                comp = (z - sum) - y;
+                sum = z;
+            }
+        }
+        const float m = sum / (float)N;
+        A.mu_s[(int64_t)u * D + tid] = m;
+        pp[2 * kParts * D + tid] = m;
+    }
+    bar_sync(kBarCompute, G::kThreads);
+    // reciprocal norms: one warp per vector (vector -1 is the stable mean)
+    const int w = tid >> 5, lane = tid & 31;
+    for (int t = w - 1; t < nb; t += G::kThreads / 32) {
+        const float* v = (t < 0) ? pp + 2 * kParts * D : bs + (size_t)t * D;
+        float ss = 0.f;
+        for (int cc = lane; cc < D; cc += 32) ss = fmaf(v[cc], v[cc], ss);
+        ss = warp_sum(ss);
+        if (lane == 0) {
+            const float inv = 1.0f / fmaxf(sqrtf(ss), kEps);
+            if (t < 0) A.inv_s[u] = inv;
+            else A.inv_e[(int64_t)u * nb + t] = inv;
+        }
+    }
+    __threadfence();
+    bar_sync(kBarCompute, G::kThreads);
+    if (tid == 0) st_release(A.ctrl + kCtrlHeader + A.units + u, 1);
+}
