@@ -569,3 +569,74 @@ __device__ __forceinline__ void finalize_head(const FusedArgs& A, int u, float* 
     bar_sync(kBarCompute, G::kThreads);
     if (tid == 0) st_release(A.ctrl + kCtrlHeader + A.units + u, 1);
 }
+
+// ---------------------------------------------------------------------------- the persistent kernel
+// Small shared-memory state after the big arrays (byte offsets inside `small`):
+//   0  item[2]      descriptors of the items in the two tile buffers
+//   32 mmk[2][6]    per-item ordered min/max keys (double buffered like the tiles)
+//   80 fin[2]       head whose anchors this CTA owes after item k (or -1), written by the control warp
+//   88 abort_flag   a bounded wait ran out somewhere in this CTA
+//   92 book_seq     index of the last item whose bookkeeping is complete
+//   96 full[2]      mbarriers of the two tile buffers
+template <typename T, int D>
+struct Ctl {
+    using G = Geo<T, D>;
+    const FusedArgs& A;
+    unsigned char* tiles;
+    Item* item;
+    uint64_t* full;
+    int* abort_flag;
+    int tiles_per_unit;
+    long long per_step, total;
+    uint64_t pol_a, pol_b;
+
+    // take the next real ticket, publish its descriptor in `slot` and start its copy
+    __device__ __forceinline__ void fetch_and_issue(int slot) {
+        unsigned long long* ticket = reinterpret_cast<unsigned long long*>(A.ctrl);
+        Item it;
+        it.kind = 2;
+        it.unit = it.tile = it.pad = 0;
+        while (*reinterpret_cast<volatile int*>(abort_flag) == 0) {
+            const unsigned long long t = atomicAdd(ticket, 1ULL);
+            if ((long long)t >= total) break;
+            const long long step = (long long)(t / (unsigned long long)per_step);
+            const int j = (int)(t - (unsigned long long)step * (unsigned long long)per_step);
+            if (j < tiles_per_unit) {
+                if (step < A.units) {
+                    it.kind = 0;
+                    it.unit = (int)step;
+                    it.tile = j;
+                    break;
+                }
+            } else if (step >= A.lag) {
+                it.kind = 1;
+                it.unit = (int)(step - A.lag);
+                it.tile = j - tiles_per_unit;
+                break;
+            }
+        }
+        item[slot] = it;
+        if (it.kind == 2) return;
+        const int N = A.K.N;
+        const int g = it.unit / A.K.H, h = it.unit % A.K.H;
+        const unsigned char* base = reinterpret_cast<const unsigned char*>(A.K.ptr) +
+                                    ((int64_t)g * A.K.stride_g + (int64_t)h * A.K.stride_h) * (int64_t)sizeof(T);
+        const int i0 = it.tile * G::kTile;
+        unsigned char* dst = tiles + (size_t)slot * G::kTileBytes;
+        int r0, r1;
+        if (it.kind == 0) {   // pass A stages the 64 rows in front of the tile as well
+            r0 = max(0, i0 - kHalo);
+            r1 = min(N, i0 + G::kTile);
+            dst += (size_t)(r0 - (i0 - kHalo)) * G::kRowBytes;
+        } else {
+            r0 = i0;
+            r1 = min(N, i0 + G::kTile);
+        }
+        const uint32_t bytes = (uint32_t)(r1 - r0) * G::kRowBytes;
+        const unsigned char* src = base + (int64_t)r0 * G::kRowBytes;
+        fence_async_smem();
+        mbar_expect_tx(&full[slot], bytes);
+        for (uint32_t off = 0; off < bytes; off += 32768u)
+            bulk_load(dst + off, src + off, min(32768u, bytes - off), &full[slot], it.kind == 0 ? pol_a : pol_b);
+    }
+};
