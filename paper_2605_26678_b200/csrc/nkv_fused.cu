@@ -640,3 +640,149 @@ struct Ctl {
             bulk_load(dst + off, src + off, min(32768u, bytes - off), &full[slot], it.kind == 0 ? pol_a : pol_b);
     }
 };
+
+template <typename T, int D>
+__global__ void __launch_bounds__(Geo<T, D>::kThreads + 32, 1) fused_scan_kernel(FusedArgs A) {
+    using G = Geo<T, D>;
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* tiles = smem;
+    float* pp = reinterpret_cast<float*>(smem + 2 * G::kTileBytes);          // [kSegs][D]
+    float* invs = pp + G::kSegs * D;                                         // [kRows]
+    unsigned char* small = reinterpret_cast<unsigned char*>(invs + G::kRows);
+    Item* item = reinterpret_cast<Item*>(small);
+    uint32_t* mmk = reinterpret_cast<uint32_t*>(small + 32);
+    int* fin = reinterpret_cast<int*>(small + 80);
+    int* abort_flag = reinterpret_cast<int*>(small + 88);
+    int* book_seq = reinterpret_cast<int*>(small + 92);
+    uint64_t* full = reinterpret_cast<uint64_t*>(small + 96);
+
+    const int N = A.K.N;
+    const int tiles_per_unit = (N + G::kTile - 1) / G::kTile;
+    const int tid = threadIdx.x;
+    constexpr int kAll = G::kThreads + 32;
+
+    if (tid == 0) {
+        mbar_init(&full[0], 1);
+        mbar_init(&full[1], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        for (int i = 0; i < 12; ++i) mmk[i] = (i & 1) ? 0u : 0xffffffffu;
+        fin[0] = fin[1] = -1;
+        *abort_flag = 0;
+        *book_seq = -1;
+    }
+    __syncthreads();
+
+    if (tid >= G::kThreads) {
+        // ------------------------------------------------------------------ control warp
+        // All 32 lanes run the loop together (the per-item barrier is warp-aligned); lane 0 works.
+        const int lane = tid - G::kThreads;
+        Ctl<T, D> C{A, tiles, item, full, abort_flag, tiles_per_unit, 2LL * tiles_per_unit,
+                    ((long long)A.units + A.lag) * 2LL * tiles_per_unit,
+                    A.hints ? l2_policy_keep() : l2_policy_normal(), A.hints ? l2_policy_stream() : l2_policy_normal()};
+        if (lane == 0) {
+            C.fetch_and_issue(0);
+            C.fetch_and_issue(1);
+        }
+        __syncwarp();
+        bar_sync(kBarEnd, kAll);   // start: both descriptors are visible
+        bool prev_done = false;
+        for (int k = 0;; ++k) {
+            const Item cur = item[k & 1];
+            bar_sync(kBarEnd, kAll);   // the compute threads have finished item k
+            const bool done = cur.kind == 2;
+            if (done && prev_done) break;
+            prev_done = done;
+            if (lane == 0) {
+                // count the tile and find out whether this CTA completed the head; publish that first,
+                // because the compute threads may be waiting for it before they start a pass-B item
+                int fin_unit = -1;
+                if (cur.kind == 0) {
+                    __threadfence();
+                    const int prev = atomicAdd(A.ctrl + kCtrlHeader + cur.unit, 1);
+                    __threadfence();
+                    if (prev == tiles_per_unit - 1) fin_unit = cur.unit;
+                }
+                *reinterpret_cast<volatile int*>(&fin[k & 1]) = fin_unit;
+                __threadfence_block();
+                *reinterpret_cast<volatile int*>(book_seq) = k;
+                if (!done) {   // publish the tile's min/max and re-arm the slots
+                    uint32_t* m = mmk + (k & 1) * 6;
+                    const int q0 = cur.kind == 0 ? 4 : 0, q1 = cur.kind == 0 ? 6 : 4;
+                    for (int q = q0; q < q1; ++q) {
+                        const uint32_t v = m[q];
+                        if (q & 1) {
+                            if (v != 0u) atomicMax(&A.mm[(int64_t)cur.unit * 6 + q], v);
+                            m[q] = 0u;
+                        } else {
+                            if (v != 0xffffffffu) atomicMin(&A.mm[(int64_t)cur.unit * 6 + q], v);
+                            m[q] = 0xffffffffu;
+                        }
+                    }
+                }
+                C.fetch_and_issue(k & 1);   // item k + 2 goes into the buffer that item k has released
+            }
+            __syncwarp();
+        }
+        return;
+    }
+
+    // ---------------------------------------------------------------------- compute threads
+    bar_sync(kBarEnd, kAll);   // start
+    bool prev_done = false;
+    int prev_kind = 2;
+    for (int k = 0;; ++k) {
+        const Item cur = item[k & 1];
+        const int buf = k & 1;
+        const uint32_t parity = (uint32_t)((k >> 1) & 1);
+        unsigned char* tile = tiles + (size_t)buf * G::kTileBytes;
+        // A pass-B item may have to wait for anchors.  This CTA must not wait while it still owes
+        // some head its anchors, so first learn whether the previous pass-A item completed a head.
+        bool owed_paid = false;
+        if (cur.kind == 1 && prev_kind == 0) {
+            if (tid == 0) {
+                const unsigned long long t0 = now_ns();
+                for (uint32_t spin = 0; *reinterpret_cast<volatile int*>(book_seq) < k - 1; ++spin) {
+                    if ((spin & 63u) == 63u && now_ns() - t0 > kWaitLimitNs) {
+                        set_status(A.status, NKV_ERR_TIMEOUT, 504);
+                        *abort_flag = 1;
+                        break;
+                    }
+                }
+            }
+            bar_sync(kBarCompute, G::kThreads);
+            const int f = *reinterpret_cast<volatile int*>(&fin[(k - 1) & 1]);
+            if (f >= 0 && *reinterpret_cast<volatile int*>(book_seq) >= k - 1) {
+                finalize_head<T, D>(A, f, pp);
+                owed_paid = true;
+            }
+        }
+        prev_kind = cur.kind;
+        if (cur.kind == 0) pass_a<T, D>(A, cur.unit, cur.tile, tile, pp, invs, mmk + buf * 6, &full[buf], parity, abort_flag);
+        else if (cur.kind == 1) pass_b<T, D>(A, cur.unit, cur.tile, tile, pp, invs, mmk + buf * 6, &full[buf], parity, abort_flag);
+        bar_sync(kBarEnd, kAll);   // end of item k
+        const bool done = cur.kind == 2;
+        if (done && prev_done) break;
+        prev_done = done;
+        if (k >= 1 && !owed_paid) {
+            const int f = fin[(k - 1) & 1];
+            if (f >= 0) finalize_head<T, D>(A, f, pp);
+        }
+    }
+}
+
+__global__ void fused_init_kernel(int units, uint32_t* mm, int* ctrl) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < (long long)units * 6) mm[i] = (i & 1) ? 0u : 0xffffffffu;
+    if (i < (long long)kCtrlHeader + 2LL * units) ctrl[i] = 0;
+}
+
+template <typename T, int D>
+cudaError_t launch_one(const FusedArgs& A, int sm_count, cudaStream_t stream) {
+    using G = Geo<T, D>;
+    const long long tiles = (long long)A.units * ((A.K.N + G::kTile - 1) / G::kTile);
+    const unsigned grid = (unsigned)(2 * tiles < sm_count ? 2 * tiles : sm_count);
+    fused_scan_kernel<T, D><<<grid, G::kThreads + 32, G::kSmem, stream>>>(A);
+    return cudaGetLastError();
+}
+
+}  // namespace
