@@ -15,6 +15,8 @@ struct nkv_handle {
     int64_t launches;
     int timing;
     int timing_valid;
+    int scan_lag;     // heads between the two passes of the fused scan (0: use the separate passes)
+    int scan_hints;   // L2 eviction hints on the key loads of the fused scan
     cudaEvent_t ev[NKV_NUM_STAGES + 1];
     cudaStream_t copy_streams[2];
     cudaEvent_t slot_done[2];
@@ -48,7 +50,7 @@ int64_t keep_count(int64_t N, double r) { return (int64_t)floor((1.0 - r) * (dou
 
 // Workspace carving shared by every entry point.
 struct Layout {
-    size_t status, inv_norm, mu_s, mu_e, inv_s, inv_e, mm, a_raw, a_star, thr, total;
+    size_t status, inv_norm, mu_s, mu_e, inv_s, inv_e, mm, a_raw, a_star, thr, ctrl, total;
 };
 
 Layout make_layout(int64_t units, int64_t N, int64_t d, int64_t nb) {
@@ -69,6 +71,7 @@ Layout make_layout(int64_t units, int64_t N, int64_t d, int64_t nb) {
     L.a_raw = take((size_t)units * 3 * N * 4);
     L.a_star = take((size_t)units * N * 4);
     L.thr = take((size_t)units * 2 * 4);
+    L.ctrl = take(fused_ctrl_bytes(units));
     L.total = o;
     return L;
 }
@@ -212,7 +215,10 @@ int nkv_create(nkv_handle** out, int device) {
     }
     h->sm_count = prop.multiProcessorCount;
     h->l2_bytes = prop.l2CacheSize;
-    if (configure_scan_kernels() != cudaSuccess || configure_stream_kernels() != cudaSuccess) {
+    h->scan_lag = 3;
+    h->scan_hints = 1;
+    if (configure_scan_kernels() != cudaSuccess || configure_stream_kernels() != cudaSuccess ||
+        configure_fused_kernels() != cudaSuccess) {
         delete h;
         return NKV_ERR_CUDA;
     }
@@ -390,7 +396,14 @@ int nkv_compress(nkv_handle* h, const nkv_tensor* K, const nkv_tensor* V, double
 
     CU(cudaMemsetAsync(status, 0, kStatusWords * sizeof(int), st));
     CU(mark());
-    if (stream_path_supported(sp)) {
+    if (h->scan_lag > 0 && fused_scan_supported(sp, K->dtype, d)) {
+        // both key passes in one persistent kernel; the stage mark between them stays empty
+        CU(launch_fused_scan(kv, K->dtype, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.mu_s), at<float>(ws, L.inv_s),
+                             at<float>(ws, L.inv_e), at<float>(ws, L.inv_norm), at<float>(ws, L.a_raw),
+                             at<uint32_t>(ws, L.mm), at<int>(ws, L.ctrl), status, h->sm_count, h->scan_lag,
+                             h->scan_hints, st, &h->launches));
+        CU(mark());
+    } else if (stream_path_supported(sp)) {
         // pass A: norms, block sums and the current-memory anomaly; pass B: the two anchor anomalies
         CU(launch_stream_a(kv, K->dtype, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm),
                            at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));
@@ -554,5 +567,12 @@ int nkv_get_stage_ms(nkv_handle* h, float* ms_out) {
 }
 
 int64_t nkv_launch_count(const nkv_handle* h) { return h ? h->launches : -1; }
+
+int nkv_set_scan_options(nkv_handle* h, int lag, int l2_hints) {
+    if (!h || lag < 0 || lag > 64) return NKV_ERR_INVALID_ARG;
+    h->scan_lag = lag;
+    h->scan_hints = l2_hints ? 1 : 0;
+    return NKV_OK;
+}
 
 }  // extern "C"

@@ -114,6 +114,14 @@ cudaError_t launch_stream_b(const TensorView& K, int dtype, int G, const ScorePa
                             const float* mu_e, const float* inv_norm, const float* inv_s, const float* inv_e,
                             float* a_raw, uint32_t* mm, int* status, int sm_count, cudaStream_t stream,
                             int64_t* launches);
+// fused two-pass scan (one persistent kernel; the second pass reads the keys from L2)
+bool fused_scan_supported(const ScoreParams& sp, int dtype, int d);
+size_t fused_ctrl_bytes(int64_t units);
+cudaError_t configure_fused_kernels();
+cudaError_t launch_fused_scan(const TensorView& K, int dtype, int G, const ScoreParams& sp, float* block_sums,
+                              float* mu_s, float* inv_s, float* inv_e, float* inv_norm, float* a_raw, uint32_t* mm,
+                              int* ctrl, int* status, int sm_count, int lag, int hints, cudaStream_t stream,
+                              int64_t* launches);
 cudaError_t configure_scan_kernels();
 cudaError_t configure_stream_kernels();
 cudaError_t launch_scan_scores(const TensorView& K, int dtype, int G, const ScoreParams& sp, const float* mu_s,

@@ -786,3 +786,69 @@ cudaError_t launch_one(const FusedArgs& A, int sm_count, cudaStream_t stream) {
 }
 
 }  // namespace
+
+#define NKV_DISPATCH(dtype, d, CALL)                                         \
+    do {                                                                     \
+        if ((dtype) == NKV_BF16 && (d) == 64) { CALL(__nv_bfloat16, 64); }   \
+        else if ((dtype) == NKV_BF16 && (d) == 128) { CALL(__nv_bfloat16, 128); } \
+        else if ((dtype) == NKV_F32 && (d) == 64) { CALL(float, 64); }       \
+        else if ((dtype) == NKV_F32 && (d) == 128) { CALL(float, 128); }     \
+        else return cudaErrorInvalidValue;                                   \
+    } while (0)
+
+cudaError_t configure_fused_kernels() {
+    cudaError_t e = cudaSuccess;
+#define CALL(T, D)                                                                                          \
+    if (e == cudaSuccess)                                                                                   \
+    e = cudaFuncSetAttribute(fused_scan_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,          \
+                             (int)Geo<T, D>::kSmem)
+    CALL(__nv_bfloat16, 64);
+    CALL(__nv_bfloat16, 128);
+    CALL(float, 64);
+    CALL(float, 128);
+#undef CALL
+    return e;
+}
+
+// The fused scan needs episodic blocks that are whole 8-row segments and tiles that are whole blocks.
+bool fused_scan_supported(const ScoreParams& sp, int dtype, int d) {
+    const int row_bytes = d * (dtype == NKV_BF16 ? 2 : 4);
+    const int tile = 65536 / row_bytes;
+    return sp.block % kSeg == 0 && tile % sp.block == 0;
+}
+
+size_t fused_ctrl_bytes(int64_t units) { return (size_t)(kCtrlHeader + 2 * units) * sizeof(int); }
+
+cudaError_t launch_fused_scan(const TensorView& K, int dtype, int G, const ScoreParams& sp, float* block_sums,
+                              float* mu_s, float* inv_s, float* inv_e, float* inv_norm, float* a_raw, uint32_t* mm,
+                              int* ctrl, int* status, int sm_count, int lag, int hints, cudaStream_t stream,
+                              int64_t* launches) {
+    FusedArgs A;
+    A.K = K;
+    A.sp = sp;
+    A.units = G * K.H;
+    A.lag = lag < 1 ? 1 : lag;
+    A.hints = hints;
+    A.block_sums = block_sums;
+    A.mu_s = mu_s;
+    A.inv_s = inv_s;
+    A.inv_e = inv_e;
+    A.inv_norm = inv_norm;
+    A.a_raw = a_raw;
+    A.mm = mm;
+    A.ctrl = ctrl;
+    A.status = status;
+    const long long words = (long long)kCtrlHeader + 2LL * A.units;
+    const long long n_init = words > 6LL * A.units ? words : 6LL * A.units;
+    fused_init_kernel<<<(unsigned)((n_init + 255) / 256), 256, 0, stream>>>(A.units, mm, ctrl);
+    ++*launches;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+#define CALL(T, D) e = launch_one<T, D>(A, sm_count, stream)
+    NKV_DISPATCH(dtype, K.d, CALL);
+#undef CALL
+    ++*launches;
+    return e;
+}
+
+}  // namespace nkv
