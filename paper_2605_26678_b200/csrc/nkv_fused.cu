@@ -452,12 +452,14 @@ __device__ __forceinline__ void pass_b(const FusedArgs& A, int u, int tile_idx, 
     bar_sync(kBarCompute, G::kThreads);
 
     const int gi0 = i0 + grp * kSeg;
-    const bool active = grp < G::kTile / kSeg && gi0 < N;
+    // Whole warps take part (kTile threads = a multiple of 32): the shuffles below name every lane.
+    // Groups past the end of the sequence compute on stale rows and write nothing.
+    const bool active = grp < G::kTile / kSeg;
     float inv_mine = 0.f;
     F2 ms[NP], me[NP];
     float rs = 0.f, re = 0.f;
     if (active) {
-        const int q = min(gi0 / b, nb - 1) - blk0;
+        const int q = min(max(min(gi0 / b, nb - 1) - blk0, 0), nblk - 1);
         G::load_vec(pp, l, ms);
         G::load_vec(pp + (1 + q) * D, l, me);
         rs = invs[0];
