@@ -266,10 +266,42 @@ __device__ __forceinline__ void range_sum(const float* pp, int l, int s0, int s1
     }
 }
 
+// Anchors of the next pass-B item, fetched into registers by the first D threads while the current
+// item is still being computed (the two dependent global round trips would otherwise sit at the start
+// of every pass-B item).  Thread c holds column c of mu_s and of up to four block means; thread 0 also
+// holds 1/||mu_s||, threads 1..nblk hold 1/||mu_e|| of block (thread - 1).
+struct Prefetched {
+    int unit, tile, have;
+    float mu, me[4], aux;
+};
+
+template <typename T, int D>
+__device__ __forceinline__ void prefetch_anchors(const FusedArgs& A, const volatile Item* next, int next_seq,
+                                                 Prefetched& pre) {
+    using G = Geo<T, D>;
+    pre.have = 0;
+    const int tid = threadIdx.x;
+    if (tid >= D || next->pad != next_seq || next->kind != 1) return;
+    const int u = next->unit, tl = next->tile;
+    const int b = A.sp.block, nb = A.sp.nblocks;
+    const int blk0 = (tl * G::kTile) / b;
+    const int nblk = min(nb - blk0, G::kTile / b);
+    if (nblk > 4 || ld_acquire(A.ctrl + kCtrlHeader + A.units + u) == 0) return;
+    pre.mu = __ldcg(A.mu_s + (int64_t)u * D + tid);
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+        pre.me[q] = q < nblk ? __ldcg(A.block_sums + ((int64_t)u * nb + blk0 + q) * D + tid) : 0.f;
+    pre.aux = tid == 0 ? __ldcg(A.inv_s + u) : (tid <= nblk ? __ldcg(A.inv_e + (int64_t)u * nb + blk0 + tid - 1) : 0.f);
+    pre.unit = u;
+    pre.tile = tl;
+    pre.have = 1;
+}
+
 // ---------------------------------------------------------------------------- pass A on one tile
 template <typename T, int D>
 __device__ __forceinline__ void pass_a(const FusedArgs& A, int u, int tile_idx, unsigned char* tile, float* pp,
-                                       float* invs, uint32_t* mmk, uint64_t* full, uint32_t parity, int* abort_flag) {
+                                       float* invs, uint32_t* mmk, uint64_t* full, uint32_t parity, int* abort_flag,
+                                       const volatile Item* next, int next_seq, Prefetched& pre) {
     using G = Geo<T, D>;
     constexpr int NP = G::kNP;
     const int N = A.K.N, W = A.sp.window;
@@ -328,6 +360,7 @@ __device__ __forceinline__ void pass_a(const FusedArgs& A, int u, int tile_idx, 
         G::store_vec(pp + (size_t)grp * D, l, acc);
     }
     bar_sync(kBarCompute, G::kThreads);
+    prefetch_anchors<T, D>(A, next, next_seq, pre);
     // ---- S1b: inclusive prefix of the segment sums inside every 64-row chunk (one column per task)
     for (int task = tid; task < (G::kRows / 64) * D; task += G::kThreads) {
         const int c64 = task / D, col = task - c64 * D;
@@ -416,7 +449,8 @@ __device__ __forceinline__ void pass_a(const FusedArgs& A, int u, int tile_idx, 
 // the tile's blocks [nblk][D]; `invs` = 1/||mu_s|| at [0], 1/||mu_e|| of the tile's blocks at [1 ..].
 template <typename T, int D>
 __device__ __forceinline__ void pass_b(const FusedArgs& A, int u, int tile_idx, const unsigned char* tile, float* pp,
-                                       float* invs, uint32_t* mmk, uint64_t* full, uint32_t parity, int* abort_flag) {
+                                       float* invs, uint32_t* mmk, uint64_t* full, uint32_t parity, int* abort_flag,
+                                       const volatile Item* next, int next_seq, Prefetched& pre) {
     using G = Geo<T, D>;
     constexpr int NP = G::kNP;
     const int N = A.K.N, b = A.sp.block, nb = A.sp.nblocks;
@@ -426,30 +460,41 @@ __device__ __forceinline__ void pass_b(const FusedArgs& A, int u, int tile_idx, 
     const int nblk = min(nb - blk0, G::kTile / b);
 
     if (tid < D) {
-        // wait (bounded) until the head's anchors have been published
-        const int* ready = A.ctrl + kCtrlHeader + A.units + u;
-        bool ok = ld_acquire(ready) != 0;
-        if (!ok && *reinterpret_cast<volatile int*>(abort_flag) == 0) {
-            const unsigned long long t0 = now_ns();
-            for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
-                if (ld_acquire(ready) != 0) {
-                    ok = true;
-                    break;
+        if (pre.have && pre.unit == u && pre.tile == tile_idx) {
+            // the anchors were fetched while the previous item was being computed
+            pp[tid] = pre.mu;
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (q < nblk) pp[(1 + q) * D + tid] = pre.me[q];
+            if (tid <= nblk) invs[tid] = pre.aux;
+        } else {
+            // wait (bounded) until the head's anchors have been published
+            const int* ready = A.ctrl + kCtrlHeader + A.units + u;
+            bool ok = ld_acquire(ready) != 0;
+            if (!ok && *reinterpret_cast<volatile int*>(abort_flag) == 0) {
+                const unsigned long long t0 = now_ns();
+                for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+                    if (ld_acquire(ready) != 0) {
+                        ok = true;
+                        break;
+                    }
+                    __nanosleep(64);
+                    if ((spin & 63u) == 63u && now_ns() - t0 > kWaitLimitNs) break;
                 }
-                __nanosleep(64);
-                if ((spin & 63u) == 63u && now_ns() - t0 > kWaitLimitNs) break;
             }
+            if (!ok) {
+                set_status(A.status, NKV_ERR_TIMEOUT, 502);
+                *abort_flag = 1;
+            }
+            pp[tid] = __ldcg(A.mu_s + (int64_t)u * D + tid);
+            for (int q = 0; q < nblk; ++q) pp[(1 + q) * D + tid] = __ldcg(A.block_sums + ((int64_t)u * nb + blk0 + q) * D + tid);
+            if (tid == 0) invs[0] = __ldcg(A.inv_s + u);
+            if (tid >= 1 && tid <= nblk) invs[tid] = __ldcg(A.inv_e + (int64_t)u * nb + blk0 + tid - 1);
+    
         }
-        if (!ok) {
-            set_status(A.status, NKV_ERR_TIMEOUT, 502);
-            *abort_flag = 1;
-        }
-        pp[tid] = __ldcg(A.mu_s + (int64_t)u * D + tid);
-        for (int q = 0; q < nblk; ++q) pp[(1 + q) * D + tid] = __ldcg(A.block_sums + ((int64_t)u * nb + blk0 + q) * D + tid);
-        if (tid == 0) invs[0] = __ldcg(A.inv_s + u);
-        if (tid >= 1 && tid <= nblk) invs[tid] = __ldcg(A.inv_e + (int64_t)u * nb + blk0 + tid - 1);
     }
     bar_sync(kBarCompute, G::kThreads);
+    prefetch_anchors<T, D>(A, next, next_seq, pre);
 
     const int gi0 = i0 + grp * kSeg;
     // Whole warps take part (kTile threads = a multiple of 32): the shuffles below name every lane.
@@ -512,28 +557,45 @@ __device__ __forceinline__ void pass_b(const FusedArgs& A, int u, int tile_idx, 
 // Block sums -> block means (in place), stable mean (compensated sums), reciprocal anchor norms.
 // Called by all compute threads of the CTA that finished the head's last pass-A tile.
 template <typename T, int D>
-__device__ __forceinline__ void finalize_head(const FusedArgs& A, int u, float* pp) {
+__device__ __forceinline__ void finalize_head(const FusedArgs& A, int u, float* pp, float* invs) {
     using G = Geo<T, D>;
-    constexpr int kParts = G::kThreads / D;
+    constexpr int Q = D / 4;                      // column quads
+    constexpr int kParts = G::kThreads / Q;       // every thread owns one quad of one slice of the blocks
+    static_assert(2 * kParts <= G::kSegs && D <= G::kRows, "finalize scratch does not fit");
     const int N = A.K.N, b = A.sp.block, nb = A.sp.nblocks;
     const int tid = threadIdx.x;
-    const int part = tid / D, c = tid - part * D;
+    const int part = tid / Q, q4 = (tid - part * Q) * 4;
     float* bs = A.block_sums + (int64_t)u * nb * D;
-    if (part < kParts) {
+    {
         const int per = (nb + kParts - 1) / kParts;
         const int t0 = part * per, t1 = min(nb, t0 + per);
-        float sum = 0.f, comp = 0.f;
-        for (int t = t0; t < t1; ++t) {
-            const float s = __ldcg(bs + (size_t)t * D + c);
-            const float y = s - comp;
-            const float z = sum + y;
-            comp = (z - sum) - y;
-            sum = z;
-            const int cnt = min(N, (t + 1) * b) - t * b;
-            bs[(size_t)t * D + c] = s / (float)cnt;
+        float sum[4] = {0.f, 0.f, 0.f, 0.f}, comp[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int t = t0; t < t1; t += 4) {
+            float4 v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)   // four independent loads in flight
+                v[j] = (t + j < t1) ? __ldcg(reinterpret_cast<const float4*>(bs + (size_t)(t + j) * D + q4))
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (t + j < t1) {
+                    const float s[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+                    const float cnt = (float)(min(N, (t + j + 1) * b) - (t + j) * b);
+                    float m[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float y = s[e] - comp[e];
+                        const float z = sum[e] + y;
+                        comp[e] = (z - sum[e]) - y;
+                        sum[e] = z;
+                        m[e] = s[e] / cnt;
+                    }
+                    *reinterpret_cast<float4*>(bs + (size_t)(t + j) * D + q4) = make_float4(m[0], m[1], m[2], m[3]);
+                }
+            }
         }
-        pp[(2 * part) * D + c] = sum;
-        pp[(2 * part + 1) * D + c] = comp;
+        *reinterpret_cast<float4*>(pp + (size_t)(2 * part) * D + q4) = make_float4(sum[0], sum[1], sum[2], sum[3]);
+        *reinterpret_cast<float4*>(pp + (size_t)(2 * part + 1) * D + q4) = make_float4(comp[0], comp[1], comp[2], comp[3]);
     }
     bar_sync(kBarCompute, G::kThreads);
     if (tid < D) {
@@ -551,13 +613,13 @@ __device__ __forceinline__ void finalize_head(const FusedArgs& A, int u, float* 
         }
         const float m = sum / (float)N;
         A.mu_s[(int64_t)u * D + tid] = m;
-        pp[2 * kParts * D + tid] = m;
+        invs[tid] = m;
     }
     bar_sync(kBarCompute, G::kThreads);
     // reciprocal norms: one warp per vector (vector -1 is the stable mean)
     const int w = tid >> 5, lane = tid & 31;
     for (int t = w - 1; t < nb; t += G::kThreads / 32) {
-        const float* v = (t < 0) ? pp + 2 * kParts * D : bs + (size_t)t * D;
+        const float* v = (t < 0) ? invs : bs + (size_t)t * D;
         float ss = 0.f;
         for (int cc = lane; cc < D; cc += 32) ss = fmaf(v[cc], v[cc], ss);
         ss = warp_sum(ss);
@@ -592,8 +654,8 @@ struct Ctl {
     long long per_step, total;
     uint64_t pol_a, pol_b;
 
-    // take the next real ticket, publish its descriptor in `slot` and start its copy
-    __device__ __forceinline__ void fetch_and_issue(int slot) {
+    // take the next real ticket (tickets of steps that have no pass-A or no pass-B head are skipped)
+    __device__ __forceinline__ Item fetch() {
         unsigned long long* ticket = reinterpret_cast<unsigned long long*>(A.ctrl);
         Item it;
         it.kind = 2;
@@ -617,7 +679,18 @@ struct Ctl {
                 break;
             }
         }
-        item[slot] = it;
+        return it;
+    }
+    // publish `it` as item number `seq` in `slot` and start its copy
+    __device__ __forceinline__ void issue(int slot, Item it, int seq) {
+        volatile Item* d = item + slot;
+        d->pad = -1;
+        __threadfence_block();
+        d->kind = it.kind;
+        d->unit = it.unit;
+        d->tile = it.tile;
+        __threadfence_block();
+        d->pad = seq;   // readers that find `seq` here may trust the other fields
         if (it.kind == 2) return;
         const int N = A.K.N;
         const int g = it.unit / A.K.H, h = it.unit % A.K.H;
@@ -681,9 +754,13 @@ __global__ void __launch_bounds__(Geo<T, D>::kThreads + 32, 1) fused_scan_kernel
         Ctl<T, D> C{A, tiles, item, full, abort_flag, tiles_per_unit, 2LL * tiles_per_unit,
                     ((long long)A.units + A.lag) * 2LL * tiles_per_unit,
                     A.hints ? l2_policy_keep() : l2_policy_normal(), A.hints ? l2_policy_stream() : l2_policy_normal()};
+        Item nxt;   // the ticket after the two in flight, fetched ahead of time (lane 0)
+        nxt.kind = 2;
+        nxt.unit = nxt.tile = nxt.pad = 0;
         if (lane == 0) {
-            C.fetch_and_issue(0);
-            C.fetch_and_issue(1);
+            C.issue(0, C.fetch(), 0);
+            C.issue(1, C.fetch(), 1);
+            nxt = C.fetch();
         }
         __syncwarp();
         bar_sync(kBarEnd, kAll);   // start: both descriptors are visible
@@ -695,8 +772,8 @@ __global__ void __launch_bounds__(Geo<T, D>::kThreads + 32, 1) fused_scan_kernel
             if (done && prev_done) break;
             prev_done = done;
             if (lane == 0) {
-                // count the tile and find out whether this CTA completed the head; publish that first,
-                // because the compute threads may be waiting for it before they start a pass-B item
+                C.issue(k & 1, nxt, k + 2);   // item k + 2 goes into the buffer that item k has released
+                // count the tile and find out whether this CTA completed the head
                 int fin_unit = -1;
                 if (cur.kind == 0) {
                     __threadfence();
@@ -721,7 +798,7 @@ __global__ void __launch_bounds__(Geo<T, D>::kThreads + 32, 1) fused_scan_kernel
                         }
                     }
                 }
-                C.fetch_and_issue(k & 1);   // item k + 2 goes into the buffer that item k has released
+                if (nxt.kind != 2) nxt = C.fetch();
             }
             __syncwarp();
         }
@@ -732,9 +809,12 @@ __global__ void __launch_bounds__(Geo<T, D>::kThreads + 32, 1) fused_scan_kernel
     bar_sync(kBarEnd, kAll);   // start
     bool prev_done = false;
     int prev_kind = 2;
+    Prefetched pre;
+    pre.have = 0;
     for (int k = 0;; ++k) {
         const Item cur = item[k & 1];
         const int buf = k & 1;
+        const volatile Item* next = item + ((k + 1) & 1);
         const uint32_t parity = (uint32_t)((k >> 1) & 1);
         unsigned char* tile = tiles + (size_t)buf * G::kTileBytes;
         // A pass-B item may have to wait for anchors.  This CTA must not wait while it still owes
@@ -754,20 +834,22 @@ __global__ void __launch_bounds__(Geo<T, D>::kThreads + 32, 1) fused_scan_kernel
             bar_sync(kBarCompute, G::kThreads);
             const int f = *reinterpret_cast<volatile int*>(&fin[(k - 1) & 1]);
             if (f >= 0 && *reinterpret_cast<volatile int*>(book_seq) >= k - 1) {
-                finalize_head<T, D>(A, f, pp);
+                finalize_head<T, D>(A, f, pp, invs);
                 owed_paid = true;
             }
         }
         prev_kind = cur.kind;
-        if (cur.kind == 0) pass_a<T, D>(A, cur.unit, cur.tile, tile, pp, invs, mmk + buf * 6, &full[buf], parity, abort_flag);
-        else if (cur.kind == 1) pass_b<T, D>(A, cur.unit, cur.tile, tile, pp, invs, mmk + buf * 6, &full[buf], parity, abort_flag);
+        if (cur.kind == 0) pass_a<T, D>(A, cur.unit, cur.tile, tile, pp, invs, mmk + buf * 6, &full[buf], parity, abort_flag,
+                                       next, k + 1, pre);
+        else if (cur.kind == 1) pass_b<T, D>(A, cur.unit, cur.tile, tile, pp, invs, mmk + buf * 6, &full[buf], parity, abort_flag,
+                                            next, k + 1, pre);
         bar_sync(kBarEnd, kAll);   // end of item k
         const bool done = cur.kind == 2;
         if (done && prev_done) break;
         prev_done = done;
         if (k >= 1 && !owed_paid) {
             const int f = fin[(k - 1) & 1];
-            if (f >= 0) finalize_head<T, D>(A, f, pp);
+            if (f >= 0) finalize_head<T, D>(A, f, pp, invs);
         }
     }
 }
