@@ -51,6 +51,8 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--scan-lag", type=int, default=None, help="heads between the two key passes (library default if unset)")
+    ap.add_argument("--scan-hints", type=int, default=1, help="L2 eviction hints on the key loads (0/1)")
     return ap.parse_args()
 
 
@@ -242,6 +244,8 @@ def run_nkv(args, cfg, r):
     ws = nkv.alloc_workspace(K, params)
     out = nkv.alloc_outputs(K, V, r)
     h = nkv.handle(local)
+    if args.scan_lag is not None:
+        nkv.nkv_set_scan_options(args.scan_lag, bool(args.scan_hints), h)
 
     def step():
         nkv.nkv_compress(K, V, r, params, out=out, ws=ws, h=h)
