@@ -553,6 +553,178 @@ __device__ __forceinline__ void pass_b(const FusedArgs& A, int u, int tile_idx, 
     }
 }
 
+// ---------------------------------------------------------------------------- pass B on tensor cores
+// For bf16 keys the two dots of every key against the fixed vectors mu_s and mu_e are a skinny matrix
+// product [16 keys x d] x [d x 8]: the fp32 anchors are split three ways into bf16 (hi + mid + lo
+// carries all 24 mantissa bits), products of bf16 numbers are exact in fp32 and the accumulation is
+// fp32, so the result is an fp32 dot product up to summation order.  Columns of the right-hand side:
+// 0..2 = mu_s hi/mid/lo, 3..5 = mu_e hi/mid/lo, 6..7 = 0.  The contraction index may be visited in any
+// order, so lane (g, t) of a warp takes the 16-byte chunks t, t+4, t+8, ... of rows g and g+8 straight
+// from the staged tile (no transposition, no conversion) and the right-hand side uses the same order.
+__device__ __forceinline__ void mma_bf16_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ void split3_bf16(float x, __nv_bfloat16* out, int stride) {
+    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+    const float r1 = x - __bfloat162float(hi);
+    const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+    const float r2 = r1 - __bfloat162float(mid);
+    out[0] = hi;
+    out[stride] = mid;
+    out[2 * stride] = __float2bfloat16_rn(r2);
+}
+
+// Requires block % 16 == 0 and at most four episodic blocks per tile.  `pp`/`invs` staging as in pass_b;
+// behind the staged floats `pp` also holds the split right-hand sides [nblk][8][D] in bf16.
+template <int D>
+__device__ __forceinline__ void pass_b_mma(const FusedArgs& A, int u, int tile_idx, const unsigned char* tile, float* pp,
+                                           float* invs, uint32_t* mmk, uint64_t* full, uint32_t parity,
+                                           int* abort_flag, const volatile Item* next, int next_seq,
+                                           Prefetched& pre) {
+    using G = Geo<__nv_bfloat16, D>;
+    constexpr int kSteps = D / 16;        // k-steps of the MMA
+    constexpr int kCh = D / 32;           // 16-byte chunks per lane and row
+    const int N = A.K.N, b = A.sp.block, nb = A.sp.nblocks;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    const int i0 = tile_idx * G::kTile;
+    const int blk0 = i0 / b;
+    const int nblk = min(nb - blk0, G::kTile / b);
+    __nv_bfloat16* rhs = reinterpret_cast<__nv_bfloat16*>(pp + 5 * D);   // [nblk][8][D]
+
+    if (tid < D) {
+        float mu, me[4], aux = 0.f;
+        if (pre.have && pre.unit == u && pre.tile == tile_idx) {
+            mu = pre.mu;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) me[q] = pre.me[q];
+            aux = pre.aux;
+        } else {
+            const int* ready = A.ctrl + kCtrlHeader + A.units + u;
+            bool ok = ld_acquire(ready) != 0;
+            if (!ok && *reinterpret_cast<volatile int*>(abort_flag) == 0) {
+                const unsigned long long t0 = now_ns();
+                for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+                    if (ld_acquire(ready) != 0) {
+                        ok = true;
+                        break;
+                    }
+                    __nanosleep(64);
+                    if ((spin & 63u) == 63u && now_ns() - t0 > kWaitLimitNs) break;
+                }
+            }
+            if (!ok) {
+                set_status(A.status, NKV_ERR_TIMEOUT, 505);
+                *abort_flag = 1;
+            }
+            mu = __ldcg(A.mu_s + (int64_t)u * D + tid);
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                me[q] = q < nblk ? __ldcg(A.block_sums + ((int64_t)u * nb + blk0 + q) * D + tid) : 0.f;
+            if (tid == 0) aux = __ldcg(A.inv_s + u);
+            else if (tid <= nblk) aux = __ldcg(A.inv_e + (int64_t)u * nb + blk0 + tid - 1);
+        }
+        if (tid <= nblk) invs[tid] = aux;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            if (q < nblk) {
+                __nv_bfloat16* r = rhs + (size_t)q * 8 * D + tid;
+                split3_bf16(mu, r, D);
+                split3_bf16(me[q], r + 3 * D, D);
+                r[6 * D] = __float2bfloat16_rn(0.f);
+                r[7 * D] = __float2bfloat16_rn(0.f);
+            }
+        }
+    }
+    bar_sync(kBarCompute, G::kThreads);
+    prefetch_anchors<__nv_bfloat16, D>(A, next, next_seq, pre);
+
+    const int rows = min(N, i0 + G::kTile) - i0;
+    const float rs = invs[0];
+    // each lane finishes one of the four results of its quad: t=0: a_s(row g), t=1: a_e(row g),
+    // t=2: a_s(row g+8), t=3: a_e(row g+8); its key's reciprocal norm is fetched before the copy is awaited
+    constexpr int kWarps = G::kThreads / 32;
+    constexpr int kIters = (G::kTile / 16 + kWarps - 1) / kWarps;
+    const int row_in_block = g + ((t & 2) ? 8 : 0);
+    float inv_pre[kIters];
+#pragma unroll
+    for (int it = 0; it < kIters; ++it) {
+        const int gi = i0 + (warp + it * kWarps) * 16 + row_in_block;
+        inv_pre[it] = (warp + it * kWarps) * 16 < rows && gi < N ? __ldcg(A.inv_norm + (int64_t)u * N + gi) : 0.f;
+    }
+    if (!mbar_wait(full, parity, abort_flag)) {
+        set_status(A.status, NKV_ERR_TIMEOUT, 503);
+        *abort_flag = 1;
+    }
+    float lo_s = INFINITY, hi_s = -INFINITY, lo_e = INFINITY, hi_e = -INFINITY;
+#pragma unroll
+    for (int it = 0; it < kIters; ++it) {
+        const int rb = warp + it * kWarps;
+        if (rb * 16 >= rows) break;
+        const int r0 = rb * 16;
+        const int q = min((i0 + r0) / b, nb - 1) - blk0;
+        const float re = invs[1 + q];
+        const int my_row = r0 + row_in_block;
+        const float inv_mine = inv_pre[it];
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+        const unsigned char* row_lo = tile + (size_t)(r0 + g) * G::kRowBytes;
+        const unsigned char* row_hi = row_lo + 8 * G::kRowBytes;
+        const __nv_bfloat16* rq = rhs + ((size_t)q * 8 + g) * D;
+#pragma unroll
+        for (int j = 0; j < kCh; ++j) {
+            const uint4 x = *reinterpret_cast<const uint4*>(row_lo + (t + 4 * j) * 16);
+            const uint4 y = *reinterpret_cast<const uint4*>(row_hi + (t + 4 * j) * 16);
+            const uint4 w = *reinterpret_cast<const uint4*>(rq + (t + 4 * j) * 8);
+            const uint32_t a_first[4] = {x.x, y.x, x.y, y.y};
+            const uint32_t a_second[4] = {x.z, y.z, x.w, y.w};
+            mma_bf16_16816(c, a_first, w.x, w.y);
+            mma_bf16_16816(c, a_second, w.z, w.w);
+        }
+        static_assert(kSteps == 2 * kCh, "two k-steps per chunk");
+        // columns: 0,1 (t=0) and 2 (t=1, c[0]) belong to mu_s; 3 (t=1, c[1]) and 4,5 (t=2) to mu_e
+        float xs_lo = t == 0 ? c[0] + c[1] : (t == 1 ? c[0] : 0.f);
+        float xe_lo = t == 1 ? c[1] : (t == 2 ? c[0] + c[1] : 0.f);
+        float xs_hi = t == 0 ? c[2] + c[3] : (t == 1 ? c[2] : 0.f);
+        float xe_hi = t == 1 ? c[3] : (t == 2 ? c[2] + c[3] : 0.f);
+#pragma unroll
+        for (int o = 1; o <= 2; o <<= 1) {
+            xs_lo += __shfl_xor_sync(0xffffffffu, xs_lo, o);
+            xe_lo += __shfl_xor_sync(0xffffffffu, xe_lo, o);
+            xs_hi += __shfl_xor_sync(0xffffffffu, xs_hi, o);
+            xe_hi += __shfl_xor_sync(0xffffffffu, xe_hi, o);
+        }
+        const float dot = t == 0 ? xs_lo : (t == 1 ? xe_lo : (t == 2 ? xs_hi : xe_hi));
+        const float a = -(dot * inv_mine) * ((t & 1) ? re : rs) + 0.f;
+        if (i0 + my_row < N) {
+            A.a_raw[((int64_t)u * 3 + (t & 1)) * N + i0 + my_row] = a;
+            if (t & 1) {
+                lo_e = fminf(lo_e, a);
+                hi_e = fmaxf(hi_e, a);
+            } else {
+                lo_s = fminf(lo_s, a);
+                hi_s = fmaxf(hi_s, a);
+            }
+        }
+    }
+    lo_s = warp_min(lo_s);
+    hi_s = warp_max(hi_s);
+    lo_e = warp_min(lo_e);
+    hi_e = warp_max(hi_e);
+    if (lane == 0) {
+        if (lo_s <= hi_s) {
+            atomicMin(&mmk[0], ord_key(lo_s));
+            atomicMax(&mmk[1], ord_key(hi_s));
+        }
+        if (lo_e <= hi_e) {
+            atomicMin(&mmk[2], ord_key(lo_e));
+            atomicMax(&mmk[3], ord_key(hi_e));
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------- anchors of one head
 // Block sums -> block means (in place), stable mean (compensated sums), reciprocal anchor norms.
 // Called by all compute threads of the CTA that finished the head's last pass-A tile.
@@ -841,8 +1013,19 @@ __global__ void __launch_bounds__(Geo<T, D>::kThreads + 32, 1) fused_scan_kernel
         prev_kind = cur.kind;
         if (cur.kind == 0) pass_a<T, D>(A, cur.unit, cur.tile, tile, pp, invs, mmk + buf * 6, &full[buf], parity, abort_flag,
                                        next, k + 1, pre);
-        else if (cur.kind == 1) pass_b<T, D>(A, cur.unit, cur.tile, tile, pp, invs, mmk + buf * 6, &full[buf], parity, abort_flag,
-                                            next, k + 1, pre);
+        else if (cur.kind == 1) {
+            bool on_tensor_cores = false;
+            if constexpr (sizeof(T) == 2) {
+                if (A.sp.block % 16 == 0 && G::kTile / A.sp.block <= 4) {
+                    on_tensor_cores = true;
+                    pass_b_mma<D>(A, cur.unit, cur.tile, tile, pp, invs, mmk + buf * 6, &full[buf], parity, abort_flag,
+                                  next, k + 1, pre);
+                }
+            }
+            if (!on_tensor_cores)
+                pass_b<T, D>(A, cur.unit, cur.tile, tile, pp, invs, mmk + buf * 6, &full[buf], parity, abort_flag,
+                             next, k + 1, pre);
+        }
         bar_sync(kBarEnd, kAll);   // end of item k
         const bool done = cur.kind == 2;
         if (done && prev_done) break;
