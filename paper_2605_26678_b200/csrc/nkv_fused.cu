@@ -29,7 +29,6 @@ namespace {
 constexpr int kHalo = kMaxWindow;
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr unsigned long long kWaitLimitNs = 2000000000ULL;   // every device-side wait gives up after 2 s
-constexpr int kLanes = 8;
 
 // control words (ints) in the workspace: [0..1] 64-bit ticket counter, [8 + u] tiles of head u
 // finished by pass A, [8 + units + u] anchors of head u published
@@ -150,27 +149,29 @@ template <> struct Pairs<float> {
     }
 };
 
-// Geometry for element type T and head dimension D with 8 lanes per row.
+// Geometry for element type T and head dimension D.  A row is split over kL lanes (16 when the row
+// has at least 256 bytes, else 8); lane l owns the 16-byte chunks l, l + kL, ...
 template <typename T, int D>
 struct Geo {
     static constexpr int kRowBytes = D * (int)sizeof(T);
-    static constexpr int kChunks = kRowBytes / 128;            // 16-byte chunks per lane
+    static constexpr int kL = kRowBytes >= 256 ? 16 : 8;       // lanes per row
+    static constexpr int kChunks = kRowBytes / (16 * kL);      // 16-byte chunks per lane
     static constexpr int kPerChunk = 16 / (int)sizeof(T);      // elements per chunk
-    static constexpr int kCols = D / kLanes;                   // columns per lane
+    static constexpr int kCols = D / kL;                       // columns per lane
     static constexpr int kNP = kCols / 2;                      // packed pairs per lane
     static constexpr int kTile = 65536 / kRowBytes;            // rows per tile (64 KB of keys)
     static constexpr int kRows = kTile + kHalo;
     static constexpr int kSegs = kRows / kSeg;
-    static constexpr int kThreads = kSegs * kLanes;            // compute threads (== kRows)
+    static constexpr int kThreads = kSegs * kL;                // compute threads: one lane group per staged segment
     static constexpr size_t kTileBytes = (size_t)kRows * kRowBytes;
     static constexpr size_t kSmem = 2 * kTileBytes + (size_t)kSegs * D * 4 + (size_t)kRows * 4 + 128;
     static_assert(kChunks >= 1 && kThreads % 32 == 0 && kThreads + 32 <= 1024, "bad geometry");
 
-    __device__ __forceinline__ static int col0(int l, int j) { return (l + kLanes * j) * kPerChunk; }
+    __device__ __forceinline__ static int col0(int l, int j) { return (l + kL * j) * kPerChunk; }
     __device__ __forceinline__ static void load_row(const unsigned char* row, int l, F2* p) {
 #pragma unroll
         for (int j = 0; j < kChunks; ++j) {
-            const uint4 q = *reinterpret_cast<const uint4*>(row + (l + kLanes * j) * 16);
+            const uint4 q = *reinterpret_cast<const uint4*>(row + (l + kL * j) * 16);
             Pairs<T>::unpack(q, p + j * Pairs<T>::kPairs);
         }
     }
@@ -198,14 +199,14 @@ struct Geo {
     }
 };
 
-// Transposed reduction of V per-lane partial values over the 8 lanes of a group (V a power of two).
-// Afterwards, with V >= 8, lane l holds the complete sums of values l*(V/8) .. l*(V/8)+V/8-1 in
-// v[0 .. V/8); with V == 4, v[0] of lane l is the complete sum of value l/2.
-template <int V>
-__device__ __forceinline__ void treduce8(float* v, int l) {
+// Transposed reduction of V per-lane partial values over the L lanes of a group (L, V powers of two).
+// Afterwards v[0 .. max(1, V/L)) hold complete sums: with V >= L lane l owns values l*(V/L)+j,
+// with V < L lane l owns value l / (L/V) (shared by L/V lanes).
+template <int V, int L>
+__device__ __forceinline__ void treduce(float* v, int l) {
     int n = V;
 #pragma unroll
-    for (int o = kLanes / 2; o >= 1; o >>= 1) {
+    for (int o = L / 2; o >= 1; o >>= 1) {
         if (n > 1) {
             const int half = n / 2;
             const bool up = (l & o) != 0;
@@ -304,8 +305,9 @@ __device__ __forceinline__ void pass_a(const FusedArgs& A, int u, int tile_idx, 
                                        const volatile Item* next, int next_seq, Prefetched& pre) {
     using G = Geo<T, D>;
     constexpr int NP = G::kNP;
+    constexpr int L = G::kL;
     const int N = A.K.N, W = A.sp.window;
-    const int tid = threadIdx.x, grp = tid >> 3, l = tid & 7;
+    const int tid = threadIdx.x, grp = tid / L, l = tid % L;
     const int i0 = tile_idx * G::kTile;
 
     // rows outside [0, N) are not copied: zero them (disjoint from the bytes in flight)
@@ -341,17 +343,17 @@ __device__ __forceinline__ void pass_a(const FusedArgs& A, int u, int tile_idx, 
                 for (int p = 0; p < NP; ++p) s = fma2(x[r][p], x[r][p], s);
                 n2[r] = hsum2(s);
             }
-            treduce8<4>(n2, l);   // lane l: squared norm of row l/2 of this half
+            treduce<4, L>(n2, l);   // lane l: squared norm of row l / (L/4) of this half
             const float inv = 1.0f / fmaxf(sqrtf(n2[0]), kEps);
-            if ((l & 1) == 0) {
-                const int sr = grp * kSeg + half * 4 + (l >> 1);
+            if ((l & (L / 4 - 1)) == 0) {
+                const int sr = grp * kSeg + half * 4 + l / (L / 4);
                 invs[sr] = inv;
                 const int gi = i0 - kHalo + sr;
                 if (sr >= kHalo && gi < N) A.inv_norm[(int64_t)u * N + gi] = inv;
             }
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
-                const float ir = __shfl_sync(0xffffffffu, inv, 2 * r, kLanes);
+                const float ir = __shfl_sync(0xffffffffu, inv, r * (L / 4), L);
                 const F2 ir2 = pack2(ir, ir);
 #pragma unroll
                 for (int p = 0; p < NP; ++p) acc[p] = fma2(x[r][p], ir2, acc[p]);
@@ -409,11 +411,27 @@ __device__ __forceinline__ void pass_a(const FusedArgs& A, int u, int tile_idx, 
             part[2 * o] = hsum2(dc);
             part[2 * o + 1] = hsum2(nc);
         }
-        treduce8<16>(part, l);   // lane l: (dc, nc) of token l
-        const int j = (s - kHaloSegs) * kSeg + l;
-        const float a_c = -(part[0] * invs[s * kSeg + l]) / fmaxf(sqrtf(part[1]), kEps) + 0.f;
+        treduce<16, L>(part, l);
+        // L == 8: lane l owns (dc, nc) of token l.  L == 16: lane l owns value l = (token l/2, quantity l%2).
+        float dcv, ncv;
+        int o;
+        bool writer;
+        if (L == 16) {
+            const float other = __shfl_xor_sync(0xffffffffu, part[0], 1);
+            dcv = (l & 1) ? other : part[0];
+            ncv = (l & 1) ? part[0] : other;
+            o = l >> 1;
+            writer = (l & 1) == 0;
+        } else {
+            dcv = part[0];
+            ncv = part[1];
+            o = l;
+            writer = true;
+        }
+        const int j = (s - kHaloSegs) * kSeg + o;
+        const float a_c = -(dcv * invs[s * kSeg + o]) / fmaxf(sqrtf(ncv), kEps) + 0.f;
         float lo = INFINITY, hi = -INFINITY;
-        if (i0 + j < N) {
+        if (writer && i0 + j < N) {
             A.a_raw[((int64_t)u * 3 + 2) * N + i0 + j] = a_c;
             lo = hi = a_c;
         }
@@ -453,8 +471,9 @@ __device__ __forceinline__ void pass_b(const FusedArgs& A, int u, int tile_idx, 
                                        const volatile Item* next, int next_seq, Prefetched& pre) {
     using G = Geo<T, D>;
     constexpr int NP = G::kNP;
+    constexpr int L = G::kL;
     const int N = A.K.N, b = A.sp.block, nb = A.sp.nblocks;
-    const int tid = threadIdx.x, grp = tid >> 3, l = tid & 7;
+    const int tid = threadIdx.x, grp = tid / L, l = tid % L;
     const int i0 = tile_idx * G::kTile;
     const int blk0 = i0 / b;
     const int nblk = min(nb - blk0, G::kTile / b);
@@ -509,7 +528,8 @@ __device__ __forceinline__ void pass_b(const FusedArgs& A, int u, int tile_idx, 
         G::load_vec(pp + (1 + q) * D, l, me);
         rs = invs[0];
         re = invs[1 + q];
-        if (gi0 + l < N) inv_mine = __ldcg(A.inv_norm + (int64_t)u * N + gi0 + l);
+        const int o_mine = L == 16 ? (l >> 1) : l;   // the token this lane finishes
+        if (gi0 + o_mine < N) inv_mine = __ldcg(A.inv_norm + (int64_t)u * N + gi0 + o_mine);
     }
     if (!mbar_wait(full, parity, abort_flag)) {
         set_status(A.status, NKV_ERR_TIMEOUT, 503);
@@ -530,25 +550,40 @@ __device__ __forceinline__ void pass_b(const FusedArgs& A, int u, int tile_idx, 
             part[2 * o] = hsum2(ds);
             part[2 * o + 1] = hsum2(de);
         }
-        treduce8<16>(part, l);   // lane l: (k_l . mu_s, k_l . mu_e)
-        const float a_s = -(part[0] * inv_mine) * rs + 0.f;
-        const float a_e = -(part[1] * inv_mine) * re + 0.f;
+        treduce<16, L>(part, l);
         float lo_s = INFINITY, hi_s = -INFINITY, lo_e = INFINITY, hi_e = -INFINITY;
-        if (gi0 + l < N) {
-            A.a_raw[((int64_t)u * 3 + 0) * N + gi0 + l] = a_s;
-            A.a_raw[((int64_t)u * 3 + 1) * N + gi0 + l] = a_e;
-            lo_s = hi_s = a_s;
-            lo_e = hi_e = a_e;
+        if (L == 16) {
+            // lane l owns value l: token l/2, quantity l%2 (0: stable, 1: episodic)
+            const int o = l >> 1;
+            const float a = -(part[0] * inv_mine) * ((l & 1) ? re : rs) + 0.f;
+            if (gi0 + o < N) {
+                A.a_raw[((int64_t)u * 3 + (l & 1)) * N + gi0 + o] = a;
+                if (l & 1) lo_e = hi_e = a;
+                else lo_s = hi_s = a;
+            }
+        } else {
+            const float a_s = -(part[0] * inv_mine) * rs + 0.f;
+            const float a_e = -(part[1] * inv_mine) * re + 0.f;
+            if (gi0 + l < N) {
+                A.a_raw[((int64_t)u * 3 + 0) * N + gi0 + l] = a_s;
+                A.a_raw[((int64_t)u * 3 + 1) * N + gi0 + l] = a_e;
+                lo_s = hi_s = a_s;
+                lo_e = hi_e = a_e;
+            }
         }
         lo_s = warp_min(lo_s);
         hi_s = warp_max(hi_s);
         lo_e = warp_min(lo_e);
         hi_e = warp_max(hi_e);
-        if ((tid & 31) == 0 && lo_s <= hi_s) {
-            atomicMin(&mmk[0], ord_key(lo_s));
-            atomicMax(&mmk[1], ord_key(hi_s));
-            atomicMin(&mmk[2], ord_key(lo_e));
-            atomicMax(&mmk[3], ord_key(hi_e));
+        if ((tid & 31) == 0) {
+            if (lo_s <= hi_s) {
+                atomicMin(&mmk[0], ord_key(lo_s));
+                atomicMax(&mmk[1], ord_key(hi_s));
+            }
+            if (lo_e <= hi_e) {
+                atomicMin(&mmk[2], ord_key(lo_e));
+                atomicMax(&mmk[3], ord_key(hi_e));
+            }
         }
     }
 }
@@ -732,13 +767,13 @@ template <typename T, int D>
 __device__ __forceinline__ void finalize_head(const FusedArgs& A, int u, float* pp, float* invs) {
     using G = Geo<T, D>;
     constexpr int Q = D / 4;                      // column quads
-    constexpr int kParts = G::kThreads / Q;       // every thread owns one quad of one slice of the blocks
+    constexpr int kParts = (G::kThreads / Q) < (G::kSegs / 2) ? (G::kThreads / Q) : (G::kSegs / 2);   // slices of the blocks
     static_assert(2 * kParts <= G::kSegs && D <= G::kRows, "finalize scratch does not fit");
     const int N = A.K.N, b = A.sp.block, nb = A.sp.nblocks;
     const int tid = threadIdx.x;
     const int part = tid / Q, q4 = (tid - part * Q) * 4;
     float* bs = A.block_sums + (int64_t)u * nb * D;
-    {
+    if (part < kParts) {
         const int per = (nb + kParts - 1) / kParts;
         const int t0 = part * per, t1 = min(nb, t0 + per);
         float sum[4] = {0.f, 0.f, 0.f, 0.f}, comp[4] = {0.f, 0.f, 0.f, 0.f};
