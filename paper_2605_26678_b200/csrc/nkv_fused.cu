@@ -272,29 +272,45 @@ __device__ __forceinline__ void range_sum(const float* pp, int l, int s0, int s1
 // of every pass-B item).  Thread c holds column c of mu_s and of up to four block means; thread 0 also
 // holds 1/||mu_s||, threads 1..nblk hold 1/||mu_e|| of block (thread - 1).
 struct Prefetched {
-    int unit, tile, have;
+    int unit, tile, have, flag, blk0, nblk;
     float mu, me[4], aux;
 };
 
+__device__ __forceinline__ int ld_relaxed(const int* p) {
+    int v;
+    asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Step 1, at the start of an item: look at the next item; if it is a pass-B item, start reading its
+// head's "anchors published" flag.  Nothing here waits: the value is first used in step 2.
 template <typename T, int D>
-__device__ __forceinline__ void prefetch_anchors(const FusedArgs& A, const volatile Item* next, int next_seq,
-                                                 Prefetched& pre) {
+__device__ __forceinline__ void prefetch_flag(const FusedArgs& A, const volatile Item* next, int next_seq,
+                                              Prefetched& pre) {
     using G = Geo<T, D>;
     pre.have = 0;
-    const int tid = threadIdx.x;
-    if (tid >= D || next->pad != next_seq || next->kind != 1) return;
-    const int u = next->unit, tl = next->tile;
+    pre.flag = 0;
+    if (threadIdx.x >= D || next->pad != next_seq || next->kind != 1) return;
+    pre.unit = next->unit;
+    pre.tile = next->tile;
     const int b = A.sp.block, nb = A.sp.nblocks;
-    const int blk0 = (tl * G::kTile) / b;
-    const int nblk = min(nb - blk0, G::kTile / b);
-    if (nblk > 4 || ld_acquire(A.ctrl + kCtrlHeader + A.units + u) == 0) return;
+    pre.blk0 = (pre.tile * G::kTile) / b;
+    pre.nblk = min(nb - pre.blk0, G::kTile / b);
+    if (pre.nblk > 4) return;
+    pre.flag = ld_relaxed(A.ctrl + kCtrlHeader + A.units + pre.unit);
+}
+// Step 2, a barrier later: if the flag was up, fetch the anchors (L2 loads that are issued only after
+// the flag's value has arrived, so they cannot return anything older than what the flag announces).
+template <typename T, int D>
+__device__ __forceinline__ void prefetch_data(const FusedArgs& A, Prefetched& pre) {
+    if (pre.flag == 0) return;
+    const int tid = threadIdx.x, u = pre.unit, nb = A.sp.nblocks;
     pre.mu = __ldcg(A.mu_s + (int64_t)u * D + tid);
 #pragma unroll
     for (int q = 0; q < 4; ++q)
-        pre.me[q] = q < nblk ? __ldcg(A.block_sums + ((int64_t)u * nb + blk0 + q) * D + tid) : 0.f;
-    pre.aux = tid == 0 ? __ldcg(A.inv_s + u) : (tid <= nblk ? __ldcg(A.inv_e + (int64_t)u * nb + blk0 + tid - 1) : 0.f);
-    pre.unit = u;
-    pre.tile = tl;
+        pre.me[q] = q < pre.nblk ? __ldcg(A.block_sums + ((int64_t)u * nb + pre.blk0 + q) * D + tid) : 0.f;
+    pre.aux = tid == 0 ? __ldcg(A.inv_s + u)
+                       : (tid <= pre.nblk ? __ldcg(A.inv_e + (int64_t)u * nb + pre.blk0 + tid - 1) : 0.f);
     pre.have = 1;
 }
 
@@ -309,6 +325,7 @@ __device__ __forceinline__ void pass_a(const FusedArgs& A, int u, int tile_idx, 
     const int N = A.K.N, W = A.sp.window;
     const int tid = threadIdx.x, grp = tid / L, l = tid % L;
     const int i0 = tile_idx * G::kTile;
+    prefetch_flag<T, D>(A, next, next_seq, pre);
 
     // rows outside [0, N) are not copied: zero them (disjoint from the bytes in flight)
     const int r0 = max(0, i0 - kHalo), r1 = min(N, i0 + G::kTile);
@@ -362,7 +379,7 @@ __device__ __forceinline__ void pass_a(const FusedArgs& A, int u, int tile_idx, 
         G::store_vec(pp + (size_t)grp * D, l, acc);
     }
     bar_sync(kBarCompute, G::kThreads);
-    prefetch_anchors<T, D>(A, next, next_seq, pre);
+    prefetch_data<T, D>(A, pre);
     // ---- S1b: inclusive prefix of the segment sums inside every 64-row chunk (one column per task)
     for (int task = tid; task < (G::kRows / 64) * D; task += G::kThreads) {
         const int c64 = task / D, col = task - c64 * D;
@@ -513,7 +530,7 @@ __device__ __forceinline__ void pass_b(const FusedArgs& A, int u, int tile_idx, 
         }
     }
     bar_sync(kBarCompute, G::kThreads);
-    prefetch_anchors<T, D>(A, next, next_seq, pre);
+    prefetch_flag<T, D>(A, next, next_seq, pre);
 
     const int gi0 = i0 + grp * kSeg;
     // Whole warps take part (kTile threads = a multiple of 32): the shuffles below name every lane.
@@ -586,6 +603,7 @@ __device__ __forceinline__ void pass_b(const FusedArgs& A, int u, int tile_idx, 
             }
         }
     }
+    prefetch_data<T, D>(A, pre);
 }
 
 // ---------------------------------------------------------------------------- pass B on tensor cores
@@ -675,7 +693,7 @@ __device__ __forceinline__ void pass_b_mma(const FusedArgs& A, int u, int tile_i
         }
     }
     bar_sync(kBarCompute, G::kThreads);
-    prefetch_anchors<__nv_bfloat16, D>(A, next, next_seq, pre);
+    prefetch_flag<__nv_bfloat16, D>(A, next, next_seq, pre);
 
     const int rows = min(N, i0 + G::kTile) - i0;
     const float rs = invs[0];
@@ -744,6 +762,7 @@ __device__ __forceinline__ void pass_b_mma(const FusedArgs& A, int u, int tile_i
             }
         }
     }
+    prefetch_data<__nv_bfloat16, D>(A, pre);
     lo_s = warp_min(lo_s);
     hi_s = warp_max(hi_s);
     lo_e = warp_min(lo_e);
@@ -861,33 +880,42 @@ struct Ctl {
     long long per_step, total;
     uint64_t pol_a, pol_b;
 
-    // take the next real ticket (tickets of steps that have no pass-A or no pass-B head are skipped)
-    __device__ __forceinline__ Item fetch() {
-        unsigned long long* ticket = reinterpret_cast<unsigned long long*>(A.ctrl);
+    // ticket number -> item; kind 2 with pad 1 means "this ticket names no item, take another"
+    __device__ __forceinline__ Item decode(unsigned long long t) const {
         Item it;
         it.kind = 2;
         it.unit = it.tile = it.pad = 0;
-        while (*reinterpret_cast<volatile int*>(abort_flag) == 0) {
-            const unsigned long long t = atomicAdd(ticket, 1ULL);
-            if ((long long)t >= total) break;
-            const long long step = (long long)(t / (unsigned long long)per_step);
-            const int j = (int)(t - (unsigned long long)step * (unsigned long long)per_step);
-            if (j < tiles_per_unit) {
-                if (step < A.units) {
-                    it.kind = 0;
-                    it.unit = (int)step;
-                    it.tile = j;
-                    break;
-                }
-            } else if (step >= A.lag) {
-                it.kind = 1;
-                it.unit = (int)(step - A.lag);
-                it.tile = j - tiles_per_unit;
-                break;
+        if ((long long)t >= total) return it;
+        const long long step = (long long)(t / (unsigned long long)per_step);
+        const int j = (int)(t - (unsigned long long)step * (unsigned long long)per_step);
+        if (j < tiles_per_unit) {
+            if (step < A.units) {
+                it.kind = 0;
+                it.unit = (int)step;
+                it.tile = j;
+                return it;
             }
+        } else if (step >= A.lag) {
+            it.kind = 1;
+            it.unit = (int)(step - A.lag);
+            it.tile = j - tiles_per_unit;
+            return it;
         }
+        it.pad = 1;
         return it;
     }
+    __device__ __forceinline__ unsigned long long take_ticket() {
+        return atomicAdd(reinterpret_cast<unsigned long long*>(A.ctrl), 1ULL);
+    }
+    // the item of ticket t, or of the next ticket that names one (steps at both ends of the order
+    // have no pass-A or no pass-B head)
+    __device__ __forceinline__ Item item_from(unsigned long long t) {
+        Item it = decode(t);
+        while (it.kind == 2 && it.pad == 1 && *reinterpret_cast<volatile int*>(abort_flag) == 0) it = decode(take_ticket());
+        it.pad = 0;
+        return it;
+    }
+    __device__ __forceinline__ Item fetch() { return item_from(take_ticket()); }
     // publish `it` as item number `seq` in `slot` and start its copy
     __device__ __forceinline__ void issue(int slot, Item it, int seq) {
         volatile Item* d = item + slot;
@@ -980,12 +1008,15 @@ __global__ void __launch_bounds__(Geo<T, D>::kThreads + 32, 1) fused_scan_kernel
             prev_done = done;
             if (lane == 0) {
                 C.issue(k & 1, nxt, k + 2);   // item k + 2 goes into the buffer that item k has released
-                // count the tile and find out whether this CTA completed the head
+                // Two global atomics per item, both in flight at once: the next ticket (needed at the
+                // next item barrier) and the tile counter of the head (needed now).  No fence here: the
+                // compute threads fence their block sums before the item barrier.
+                const bool more = nxt.kind != 2 && *reinterpret_cast<volatile int*>(abort_flag) == 0;
+                unsigned long long t_raw = ~0ULL;
+                if (more) t_raw = C.take_ticket();
                 int fin_unit = -1;
                 if (cur.kind == 0) {
-                    __threadfence();
                     const int prev = atomicAdd(A.ctrl + kCtrlHeader + cur.unit, 1);
-                    __threadfence();
                     if (prev == tiles_per_unit - 1) fin_unit = cur.unit;
                 }
                 *reinterpret_cast<volatile int*>(&fin[k & 1]) = fin_unit;
@@ -1005,7 +1036,8 @@ __global__ void __launch_bounds__(Geo<T, D>::kThreads + 32, 1) fused_scan_kernel
                         }
                     }
                 }
-                if (nxt.kind != 2) nxt = C.fetch();
+                if (more) nxt = C.item_from(t_raw);
+                else nxt.kind = 2;
             }
             __syncwarp();
         }
