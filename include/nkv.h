@@ -247,12 +247,13 @@ NKV_API int nkv_get_stage_ms(nkv_handle* h, float* ms_out);
 /* Number of kernels this handle has launched since creation. */
 NKV_API int64_t nkv_launch_count(const nkv_handle* h);
 
-/* Tuning of the key scan inside nkv_compress (Sections 2.1-2.3 need two passes over the keys of a
- * head; one kernel interleaves them head by head so that the second pass reads the keys from L2).
- * `lag` = how many heads the second pass trails the first (1..64, default 3: larger hides the
- * anchor reduction better, smaller keeps fewer keys live in L2; 0 = run the two passes as separate
- * kernels over the whole cache).  `l2_hints` non-zero = first-pass loads ask L2 to keep the lines,
- * second-pass loads mark them disposable (default on).  Results do not depend on either. */
+/* Choice of the key scan inside nkv_compress.  Sections 2.1-2.3 need two passes over the keys of a
+ * head.  lag = 0 (default) runs them as two kernels over the whole cache.  lag in 1..64 runs one
+ * kernel that interleaves the passes head by head, the second pass trailing the first by `lag`
+ * heads so that it reads the keys from L2 (larger hides the anchor reduction better, smaller keeps
+ * fewer keys live in L2).  `l2_hints` non-zero = first-pass loads ask L2 to keep the lines and
+ * second-pass loads mark them disposable (interleaved kernel only).  Results do not depend on
+ * either setting. */
 NKV_API int nkv_set_scan_options(nkv_handle* h, int lag, int l2_hints);
 
 /*

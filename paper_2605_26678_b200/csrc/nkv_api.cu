@@ -215,7 +215,7 @@ int nkv_create(nkv_handle** out, int device) {
     }
     h->sm_count = prop.multiProcessorCount;
     h->l2_bytes = prop.l2CacheSize;
-    h->scan_lag = 3;
+    h->scan_lag = 0;   // the separate passes are faster today; see nkv_set_scan_options
     h->scan_hints = 1;
     if (configure_scan_kernels() != cudaSuccess || configure_stream_kernels() != cudaSuccess ||
         configure_fused_kernels() != cudaSuccess) {

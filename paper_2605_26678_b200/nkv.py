@@ -419,7 +419,7 @@ def nkv_launch_count(h: Optional[Handle] = None) -> int:
     return int(h.lib.nkv_launch_count(h.h))
 
 
-def nkv_set_scan_options(lag: int = 3, l2_hints: bool = True, h: Optional[Handle] = None) -> None:
+def nkv_set_scan_options(lag: int = 0, l2_hints: bool = True, h: Optional[Handle] = None) -> None:
     """lag = heads between the two key passes of the fused scan (0: separate kernels); see nkv.h."""
     h = h or handle()
     _check(h.lib.nkv_set_scan_options(h.h, int(lag), 1 if l2_hints else 0), "nkv_set_scan_options")
