@@ -50,7 +50,7 @@ int64_t keep_count(int64_t N, double r) { return (int64_t)floor((1.0 - r) * (dou
 
 // Workspace carving shared by every entry point.
 struct Layout {
-    size_t status, inv_norm, mu_s, mu_e, inv_s, inv_e, mm, a_raw, a_star, thr, ctrl, total;
+    size_t status, inv_norm, mu_s, mu_e, inv_s, inv_e, mm, a_raw, a_star, thr, ctrl, hstat, total;
 };
 
 Layout make_layout(int64_t units, int64_t N, int64_t d, int64_t nb) {
@@ -72,6 +72,7 @@ Layout make_layout(int64_t units, int64_t N, int64_t d, int64_t nb) {
     L.a_star = take((size_t)units * N * 4);
     L.thr = take((size_t)units * 2 * 4);
     L.ctrl = take(fused_ctrl_bytes(units));
+    L.hstat = take(head_stat_bytes(units));
     L.total = o;
     return L;
 }
@@ -295,7 +296,7 @@ int nkv_score(nkv_handle* h, const nkv_tensor* K, const float* mu_s, const float
     CU(launch_scan_scores(kv, K->dtype, (int)K->G, sp, mu_s, mu_e, inv_norm, at<float>(ws, L.inv_s),
                           at<float>(ws, L.inv_e), a_raw, at<uint32_t>(ws, L.mm), st, &h->launches));
     CU(launch_head_scores(units, (int)K->N, sp, a_raw, at<uint32_t>(ws, L.mm), a_star, head_stats_opt,
-                          at<int>(ws, L.status), st, &h->launches));
+                          at<float>(ws, L.hstat), at<int>(ws, L.status), st, &h->launches));
     return NKV_OK;
 }
 
@@ -426,8 +427,8 @@ int nkv_compress(nkv_handle* h, const nkv_tensor* K, const nkv_tensor* V, double
                               at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), st, &h->launches));
     }
     CU(mark());
-    CU(launch_head_scores(units, N, sp, at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), a_star, nullptr, status, st,
-                          &h->launches));
+    CU(launch_head_scores(units, N, sp, at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), a_star, nullptr,
+                          at<float>(ws, L.hstat), status, st, &h->launches));
     CU(mark());
     CU(launch_budget(G, H, N, (int)keep, (int)n_safe, a_star, budgets, at<uint32_t>(ws, L.thr), status, st,
                      &h->launches));

@@ -128,9 +128,10 @@ cudaError_t launch_scan_scores(const TensorView& K, int dtype, int G, const Scor
                                const float* mu_e, const float* inv_norm, const float* inv_mu_s_norm,
                                const float* inv_mu_e_norm, float* a_raw, uint32_t* minmax_keys,
                                cudaStream_t stream, int64_t* launches);
+size_t head_stat_bytes(int64_t units);   // scratch of launch_head_scores (`hstat`)
 cudaError_t launch_head_scores(int units, int N, const ScoreParams& sp, const float* a_raw,
-                               const uint32_t* minmax_keys, float* a_star, float* head_stats_opt, int* status,
-                               cudaStream_t stream, int64_t* launches);
+                               const uint32_t* minmax_keys, float* a_star, float* head_stats_opt, float* hstat,
+                               int* status, cudaStream_t stream, int64_t* launches);
 cudaError_t launch_budget(int G, int H, int N, int keep, int n_safe, const float* a_star, int32_t* budgets,
                           uint32_t* sel_thresholds, int* status, cudaStream_t stream, int64_t* launches);
 cudaError_t launch_select(int G, int H, int N, int64_t idx_capacity, const float* a_star, const int32_t* budgets,

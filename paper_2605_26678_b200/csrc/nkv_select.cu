@@ -283,13 +283,17 @@ __device__ __forceinline__ float block_reduce_f(SelectShared& S, float v, int op
     return r;
 }
 
-__global__ void __launch_bounds__(kThreads) head_scores_kernel(int N, ScoreParams sp, const float* __restrict__ a_raw,
-                                                               const uint32_t* __restrict__ mm,
-                                                               float* __restrict__ a_star, float* __restrict__ stats_out,
-                                                               int* status) {
+// Layout of the per-head statistics scratch written by scale_stats_kernel (floats per head).
+constexpr int kHeadStat = 8;   // Delta_s, Delta_e, Delta_c, min s, max s, sum s, unused, unused
+constexpr int kStatThreads = 512;
+
+// scale_stats: one CTA per (head, task).  Tasks 0..2: the reliability gap of one scale (exact sums of
+// the m largest and m smallest values); task 3: min, max and sum of the surprise over the head.
+__global__ void __launch_bounds__(kStatThreads) scale_stats_kernel(int N, ScoreParams sp, const float* __restrict__ a_raw,
+                                                                   const uint32_t* __restrict__ mm,
+                                                                   float* __restrict__ hstat, int* status) {
     __shared__ SelectShared S;
-    __shared__ float sh_delta[3], sh_w[3], sh_s[3];
-    const int u = blockIdx.x;
+    const int u = blockIdx.x >> 2, task = blockIdx.x & 3;
     const float* a[3] = {a_raw + ((int64_t)u * 3 + 0) * N, a_raw + ((int64_t)u * 3 + 1) * N,
                          a_raw + ((int64_t)u * 3 + 2) * N};
     float lo[3], range[3];
@@ -300,96 +304,126 @@ __global__ void __launch_bounds__(kThreads) head_scores_kernel(int N, ScoreParam
     }
     if (threadIdx.x == 0) S.ncorr = 0;
     __syncthreads();
+    float* out = hstat + (int64_t)u * kHeadStat;
 
-    // reliability gaps: (sum of the m largest - sum of the m smallest) / (m * range)
-    const int m = sp.top_m;
-    for (int k = 0; k < 3; ++k) {
+    if (task < 3) {
+        // reliability gap: (sum of the m largest - sum of the m smallest) / (m * range)
+        const int k = task, m = sp.top_m;
+        const float lok = k == 0 ? lo[0] : (k == 1 ? lo[1] : lo[2]);
+        const float rk = k == 0 ? range[0] : (k == 1 ? range[1] : range[2]);
+        const float* ak = k == 0 ? a[0] : (k == 1 ? a[1] : a[2]);
         float gap = 0.f;
-        if (range[k] > 0.f) {
+        if (rk > 0.f) {
             float side_sum[2];
             for (int side = 0; side < 2; ++side) {
-                ScaleSrc src{a[k], side == 0 ? 1.f : -1.f};
-                const float lo0 = side == 0 ? lo[k] : -(lo[k] + range[k]);
-                block_select_desc(S, src, N, m, lo0, (float)kBins / range[k], status);
+                ScaleSrc src{ak, side == 0 ? 1.f : -1.f};
+                const float lo0 = side == 0 ? lok : -(lok + rk);
+                block_select_desc(S, src, N, m, lo0, (float)kBins / rk, status);
                 const uint32_t theta = S.theta;
                 const int gt = S.gt;
                 __syncthreads();
                 float part = 0.f;
                 for (int j = threadIdx.x; j < N; j += blockDim.x) {
-                    const float v = src.sign * a[k][j];
+                    const float v = src.sign * ak[j];
                     if (ord_key(v) > theta) part += v;
                 }
                 const float above = block_reduce_f(S, part, 0);
                 side_sum[side] = above + (float)(m - gt) * ord_float(theta);
             }
             // side 1 summed the negated values: top_sum - bot_sum = side_sum[0] + side_sum[1]
-            gap = (side_sum[0] + side_sum[1]) / ((float)m * range[k]);
+            gap = (side_sum[0] + side_sum[1]) / ((float)m * rk);
         }
-        if (threadIdx.x == 0) sh_delta[k] = gap;
+        if (threadIdx.x == 0) out[k] = gap;
+    } else {
+        float smin = INFINITY, smax = -INFINITY, ssum = 0.f;
+        for (int j = threadIdx.x; j < N; j += blockDim.x) {
+            const float s = surprise3(norm01(a[0][j], lo[0], range[0]), norm01(a[1][j], lo[1], range[1]),
+                                      norm01(a[2][j], lo[2], range[2]));
+            smin = fminf(smin, s);
+            smax = fmaxf(smax, s);
+            ssum += s;
+        }
+        smin = block_reduce_f(S, smin, 1);
+        smax = block_reduce_f(S, smax, 2);
+        ssum = block_reduce_f(S, ssum, 0);
+        if (threadIdx.x == 0) {
+            out[3] = smin;
+            out[4] = smax;
+            out[5] = ssum;
+        }
     }
+}
 
-    // surprise statistics over the head
-    float smin = INFINITY, smax = -INFINITY, ssum = 0.f;
-    for (int j = threadIdx.x; j < N; j += blockDim.x) {
-        const float s = surprise3(norm01(a[0][j], lo[0], range[0]), norm01(a[1][j], lo[1], range[1]),
-                                  norm01(a[2][j], lo[2], range[2]));
-        smin = fminf(smin, s);
-        smax = fmaxf(smax, s);
-        ssum += s;
+// mix: elementwise.  Every CTA recomputes its head's three weights and surprise constants (a handful of
+// flops) and routes a chunk of tokens: a* = (1 - alpha) * blend + alpha * max, sinks pinned to +inf.
+constexpr int kMixThreads = 256;
+constexpr int kMixPerThread = 8;
+__global__ void __launch_bounds__(kMixThreads) mix_kernel(int N, ScoreParams sp, const float* __restrict__ a_raw,
+                                                          const uint32_t* __restrict__ mm,
+                                                          const float* __restrict__ hstat, float* __restrict__ a_star,
+                                                          float* __restrict__ stats_out) {
+    const int u = blockIdx.y;
+    const float* a0 = a_raw + ((int64_t)u * 3 + 0) * N;
+    const float* a1 = a0 + N;
+    const float* a2 = a1 + N;
+    float lo[3], range[3];
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+        lo[k] = ord_float(mm[(int64_t)u * 6 + 2 * k]);
+        range[k] = ord_float(mm[(int64_t)u * 6 + 2 * k + 1]) - lo[k];
     }
-    smin = block_reduce_f(S, smin, 1);
-    smax = block_reduce_f(S, smax, 2);
-    ssum = block_reduce_f(S, ssum, 0);
-    if (threadIdx.x == 0) {
-        float z[3], zmax = -INFINITY, wsum = 0.f;
-        for (int k = 0; k < 3; ++k) {
-            z[k] = sp.log_prior[k] + sp.beta * sh_delta[k];
-            zmax = fmaxf(zmax, z[k]);
-        }
-        for (int k = 0; k < 3; ++k) {
-            z[k] = expf(z[k] - zmax);
-            wsum += z[k];
-        }
-        for (int k = 0; k < 3; ++k) sh_w[k] = z[k] / wsum;
-        const float srange = smax - smin;
-        sh_s[0] = smin;
-        sh_s[1] = srange;
-        sh_s[2] = srange > 0.f ? (ssum / (float)N - smin) / srange : 0.f;
+    const float* hs = hstat + (int64_t)u * kHeadStat;
+    float z[3], zmax = -INFINITY, wsum = 0.f, w[3];
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+        z[k] = sp.log_prior[k] + sp.beta * hs[k];
+        zmax = fmaxf(zmax, z[k]);
     }
-    __syncthreads();
-    const float w0 = sh_w[0], w1 = sh_w[1], w2 = sh_w[2];
-    const float s_lo = sh_s[0], s_range = sh_s[1], s_mean = sh_s[2];
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+        z[k] = expf(z[k] - zmax);
+        wsum += z[k];
+    }
+#pragma unroll
+    for (int k = 0; k < 3; ++k) w[k] = z[k] / wsum;
+    const float s_lo = hs[3], s_range = hs[4] - hs[3];
+    const float s_mean = s_range > 0.f ? (hs[5] / (float)N - s_lo) / s_range : 0.f;
 
-    for (int j = threadIdx.x; j < N; j += blockDim.x) {
-        const float x0 = norm01(a[0][j], lo[0], range[0]);
-        const float x1 = norm01(a[1][j], lo[1], range[1]);
-        const float x2 = norm01(a[2][j], lo[2], range[2]);
-        const float blend = w0 * x0 + w1 * x1 + w2 * x2;
-        const float win = fmaxf(x0, fmaxf(x1, x2));
-        float alpha;
-        if (sp.gate_mode == NKV_GATE_AVERAGE) alpha = 0.f;
-        else if (sp.gate_mode == NKV_GATE_MAX) alpha = 1.f;
-        else {
-            const float sn = norm01(surprise3(x0, x1, x2), s_lo, s_range);
-            const float sprime = fmaxf(0.f, sn - s_mean);
-            alpha = 1.0f / (1.0f + expf(-sp.kappa * (sprime - sp.tau)));
+    const int base = blockIdx.x * (kMixThreads * kMixPerThread);
+#pragma unroll
+    for (int e = 0; e < kMixPerThread; ++e) {
+        const int j = base + e * kMixThreads + threadIdx.x;
+        if (j < N) {
+            const float x0 = norm01(a0[j], lo[0], range[0]);
+            const float x1 = norm01(a1[j], lo[1], range[1]);
+            const float x2 = norm01(a2[j], lo[2], range[2]);
+            const float blend = w[0] * x0 + w[1] * x1 + w[2] * x2;
+            const float win = fmaxf(x0, fmaxf(x1, x2));
+            float alpha;
+            if (sp.gate_mode == NKV_GATE_AVERAGE) alpha = 0.f;
+            else if (sp.gate_mode == NKV_GATE_MAX) alpha = 1.f;
+            else {
+                const float sn = norm01(surprise3(x0, x1, x2), s_lo, s_range);
+                const float sprime = fmaxf(0.f, sn - s_mean);
+                alpha = 1.0f / (1.0f + expf(-sp.kappa * (sprime - sp.tau)));
+            }
+            float v = (1.0f - alpha) * blend + alpha * win + 0.f;
+            if (j < sp.n_sink) v = INFINITY;
+            a_star[(int64_t)u * N + j] = v;
         }
-        float v = (1.0f - alpha) * blend + alpha * win + 0.f;
-        if (j < sp.n_sink) v = INFINITY;
-        a_star[(int64_t)u * N + j] = v;
     }
-    if (stats_out && threadIdx.x == 0) {
+    if (stats_out && blockIdx.x == 0 && threadIdx.x == 0) {
         float* o = stats_out + (int64_t)u * NKV_HEAD_STATS;
         for (int k = 0; k < 3; ++k) {
             o[k] = lo[k];
             o[3 + k] = lo[k] + range[k];
-            o[6 + k] = sh_delta[k];
-            o[9 + k] = sh_w[k];
+            o[6 + k] = hs[k];
+            o[9 + k] = w[k];
         }
         o[12] = s_lo;
         o[13] = s_lo + s_range;
         o[14] = s_mean;
-        o[15] = (float)m;
+        o[15] = (float)sp.top_m;
     }
 }
 
@@ -413,35 +447,44 @@ struct PoolSrc {       // all (head, token) pairs of a group whose key does not 
     }
 };
 
+// safeguard: one CTA per head.  The n_safe best tokens of each head are kept unconditionally:
+// thr[2u] = ordered key of the n_safe-th best score, thr[2u+1] = how many tokens tied at that key
+// belong to the safeguard.  (The group kernel below overwrites both words with the final threshold.)
+__global__ void __launch_bounds__(kStatThreads) safeguard_kernel(int N, int n_safe, const float* __restrict__ a_star,
+                                                                 uint32_t* __restrict__ thr, int* status) {
+    __shared__ SelectShared S;
+    const int u = blockIdx.x;
+    if (threadIdx.x == 0) S.ncorr = 0;
+    __syncthreads();
+    if (n_safe > 0) {
+        HeadSrc src{a_star + (int64_t)u * N};
+        block_select_desc(S, src, N, n_safe, 0.f, (float)kBins, status);
+        if (threadIdx.x == 0) {
+            thr[(int64_t)u * 2] = S.theta;
+            thr[(int64_t)u * 2 + 1] = (uint32_t)(n_safe - S.gt);
+        }
+    } else if (threadIdx.x == 0) {
+        thr[(int64_t)u * 2] = 0xffffffffu;
+        thr[(int64_t)u * 2 + 1] = 0u;
+    }
+}
+
+// budget: one CTA per layer group, after safeguard_kernel.
 __global__ void __launch_bounds__(kThreads) budget_kernel(int H, int N, int keep, int n_safe,
                                                           const float* __restrict__ a_star,
                                                           int32_t* __restrict__ budgets, uint32_t* __restrict__ thr,
                                                           int* status) {
     __shared__ SelectShared S;
     __shared__ uint32_t T[kMaxCorr];
-    __shared__ int c_gt[kMaxCorr], corr[kMaxCorr], cnt_mid[kMaxCorr], cnt_eq[kMaxCorr];
+    __shared__ int corr[kMaxCorr], cnt_mid[kMaxCorr], cnt_eq[kMaxCorr];
     const int g = blockIdx.x;
     const float* v = a_star + (int64_t)g * H * N;
     if (threadIdx.x == 0) S.ncorr = 0;
-    __syncthreads();
-
-    // per-head safeguard: the n_safe best tokens of each head are kept unconditionally
-    for (int h = 0; h < H; ++h) {
-        if (n_safe > 0) {
-            HeadSrc src{v + (int64_t)h * N};
-            block_select_desc(S, src, N, n_safe, 0.f, (float)kBins, status);
-            if (threadIdx.x == 0) {
-                T[h] = S.theta;
-                c_gt[h] = S.gt;
-                corr[h] = n_safe - S.gt;   // ties at the threshold that belong to the safeguard
-            }
-        } else if (threadIdx.x == 0) {
-            T[h] = 0xffffffffu;
-            c_gt[h] = 0;
-            corr[h] = 0;
-        }
-        __syncthreads();
+    if (threadIdx.x < H) {
+        T[threadIdx.x] = thr[((int64_t)g * H + threadIdx.x) * 2];
+        corr[threadIdx.x] = (int)thr[((int64_t)g * H + threadIdx.x) * 2 + 1];
     }
+    __syncthreads();
 
     // cross-head competition for the remaining slots
     const int rest = H * keep - H * n_safe;
@@ -628,16 +671,27 @@ __global__ void __launch_bounds__(256) ranks_kernel(int N, const float* __restri
 }  // namespace
 
 cudaError_t launch_head_scores(int units, int N, const ScoreParams& sp, const float* a_raw,
-                               const uint32_t* minmax_keys, float* a_star, float* head_stats_opt, int* status,
-                               cudaStream_t stream, int64_t* launches) {
-    head_scores_kernel<<<units, kThreads, 0, stream>>>(N, sp, a_raw, minmax_keys, a_star, head_stats_opt, status);
+                               const uint32_t* minmax_keys, float* a_star, float* head_stats_opt, float* hstat,
+                               int* status, cudaStream_t stream, int64_t* launches) {
+    scale_stats_kernel<<<units * 4, kStatThreads, 0, stream>>>(N, sp, a_raw, minmax_keys, hstat, status);
+    ++*launches;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    dim3 grid((N + kMixThreads * kMixPerThread - 1) / (kMixThreads * kMixPerThread), units);
+    mix_kernel<<<grid, kMixThreads, 0, stream>>>(N, sp, a_raw, minmax_keys, hstat, a_star, head_stats_opt);
     ++*launches;
     return cudaGetLastError();
 }
 
+size_t head_stat_bytes(int64_t units) { return (size_t)units * kHeadStat * sizeof(float); }
+
 cudaError_t launch_budget(int G, int H, int N, int keep, int n_safe, const float* a_star, int32_t* budgets,
                           uint32_t* sel_thresholds, int* status, cudaStream_t stream, int64_t* launches) {
     if (H > kMaxCorr) return cudaErrorInvalidValue;
+    safeguard_kernel<<<G * H, kStatThreads, 0, stream>>>(N, n_safe, a_star, sel_thresholds, status);
+    ++*launches;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
     budget_kernel<<<G, kThreads, 0, stream>>>(H, N, keep, n_safe, a_star, budgets, sel_thresholds, status);
     ++*launches;
     return cudaGetLastError();
