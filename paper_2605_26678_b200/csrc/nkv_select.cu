@@ -283,6 +283,186 @@ __device__ __forceinline__ float block_reduce_f(SelectShared& S, float v, int op
     return r;
 }
 
+// ------------------------------------------------------------------------------------------
+// Bracketed selection.  block_select_desc touches a shared-memory histogram once per element and
+// pass, which serialises on the crowded bins.  Here a strided sample of the source first brackets
+// the wanted order statistic between two pivots P_lo <= theta <= P_hi (a few standard deviations of
+// the sample's rank error on either side); one pass then counts (and optionally sums) the elements
+// above P_hi in registers and appends only the elements inside the bracket, a few percent of the
+// source, to a shared list; block_select_desc finishes exactly on that list.  Whenever the bracket
+// turns out wrong (rank outside the list, list overflow) the full-histogram path runs instead, so the
+// result is always exact.
+// ------------------------------------------------------------------------------------------
+constexpr int kSample = 1024;
+constexpr int kCandCap = 6144;
+
+struct BracketShared {
+    float samp[kSample];
+    float cand[kCandCap];
+    int samp_n, cand_n, cnt_gt, ok;
+    float sum_gt;
+    float p_lo, p_hi;
+    float save_v[kMaxCorr];
+    int save_m[kMaxCorr], save_n;
+};
+
+struct SmemSrc {
+    const float* p;
+    __device__ __forceinline__ bool get(int j, float& v) const {
+        v = p[j];
+        return true;
+    }
+};
+
+// Same contract as block_select_desc (results in S.theta / S.gt / S.eq, S.corr honoured).  `n_eff` is the
+// number of elements the source really yields (n minus those its get() rejects).  If `sum_above` is not
+// null it receives the sum of the elements strictly greater than theta.
+template <class Src>
+__device__ void block_select_bracket(SelectShared& S, BracketShared& X, const Src& src, int n, long long n_eff,
+                                     int rank, float lo0, float sc0, int* status, float* sum_above) {
+    const int tid = threadIdx.x, nt = blockDim.x;
+    bool use_bracket = n > kCandCap && n_eff > 0;
+    if (use_bracket) {
+        // 1. strided sample (rejected elements are skipped)
+        if (tid == 0) X.samp_n = 0;
+        __syncthreads();
+        for (int i = tid; i < kSample; i += nt) {
+            float v;
+            if (src.get((int)(((long long)i * n) / kSample), v)) X.samp[atomicAdd(&X.samp_n, 1)] = v;
+        }
+        __syncthreads();
+        const int sn = X.samp_n;
+        // 2. pivots: sample ranks around rank * sn / n_eff, four standard deviations of the rank error apart
+        const float q = (float)rank * (float)sn / (float)n_eff;
+        const float sd = sqrtf(fmaxf(q * (1.0f - q / fmaxf((float)sn, 1.0f)), 1.0f));
+        const int r_hi = (int)floorf(q - 4.0f * sd - 4.0f), r_lo = (int)ceilf(q + 4.0f * sd + 4.0f);
+        // save the correction multiset: the sample selections below must not see it
+        if (tid == 0) {
+            X.save_n = S.ncorr;
+            for (int c = 0; c < S.ncorr; ++c) {
+                X.save_v[c] = S.corr_v[c];
+                X.save_m[c] = S.corr_m[c];
+            }
+            S.ncorr = 0;
+            X.p_hi = INFINITY;
+            X.p_lo = -INFINITY;
+        }
+        __syncthreads();
+        SmemSrc ssrc{X.samp};
+        if (sn >= 64 && r_hi >= 1) {
+            block_select_desc(S, ssrc, sn, r_hi, lo0, sc0, status);
+            if (tid == 0) X.p_hi = ord_float(S.theta);
+            __syncthreads();
+        }
+        if (sn >= 64 && r_lo <= sn) {
+            block_select_desc(S, ssrc, sn, r_lo, lo0, sc0, status);
+            if (tid == 0) X.p_lo = ord_float(S.theta);
+            __syncthreads();
+        }
+        const float p_hi = X.p_hi, p_lo = X.p_lo;
+        // 3. one pass: count / sum above the bracket, collect the bracket
+        if (tid == 0) {
+            X.cand_n = 0;
+            X.cnt_gt = 0;
+            X.sum_gt = 0.f;
+        }
+        __syncthreads();
+        int cnt = 0;
+        float sum = 0.f;
+        const int lane = tid & 31;
+        for (int j0 = 0; j0 < n; j0 += nt) {
+            const int j = j0 + tid;
+            float v = 0.f;
+            const bool in = j < n && src.get(j, v);
+            const bool above = in && v > p_hi;
+            const bool inside = in && !above && v >= p_lo;
+            cnt += above;
+            if (above) sum += v;
+            const unsigned ballot = __ballot_sync(0xffffffffu, inside);
+            if (ballot) {
+                int base = 0;
+                if (lane == 0) base = atomicAdd(&X.cand_n, __popc(ballot));
+                base = __shfl_sync(0xffffffffu, base, 0);
+                const int pos = base + __popc(ballot & ((1u << lane) - 1u));
+                if (inside && pos < kCandCap) X.cand[pos] = v;
+            }
+        }
+        cnt = block_sum_int(S, cnt);
+        __syncthreads();
+        const float total_sum = sum_above ? block_reduce_f(S, sum, 0) : 0.f;
+        // 4. move the correction multiset inside / above the bracket
+        if (tid == 0) {
+            int above_corr = 0, ncorr = 0;
+            for (int c = 0; c < X.save_n; ++c) {
+                if (X.save_m[c] <= 0) continue;
+                if (X.save_v[c] > p_hi) above_corr += X.save_m[c];
+                else if (X.save_v[c] >= p_lo) {
+                    S.corr_v[ncorr] = X.save_v[c];
+                    S.corr_m[ncorr] = X.save_m[c];
+                    ++ncorr;
+                }
+            }
+            S.ncorr = ncorr;
+            X.cnt_gt = cnt - above_corr;
+            X.sum_gt = total_sum;
+            int inner = X.cand_n;
+            for (int c = 0; c < ncorr; ++c) inner -= S.corr_m[c];
+            const int r2 = rank - X.cnt_gt;
+            X.ok = (X.cand_n <= kCandCap && r2 >= 1 && r2 <= inner) ? 1 : 0;
+        }
+        __syncthreads();
+        if (X.ok) {
+            const int cn = X.cand_n, r2 = rank - X.cnt_gt;
+            const float width = p_hi - p_lo;
+            const bool own_bins = width > 0.f && isfinite(width) && isfinite(p_lo);
+            SmemSrc csrc{X.cand};
+            block_select_desc(S, csrc, cn, r2, own_bins ? p_lo : lo0, own_bins ? (float)kBins / width : sc0, status);
+            if (sum_above) {
+                const uint32_t theta = S.theta;
+                float part = 0.f;
+                for (int j = tid; j < cn; j += nt)
+                    if (ord_key(X.cand[j]) > theta) part += X.cand[j];
+                const float inner_sum = block_reduce_f(S, part, 0);
+                if (tid == 0) *sum_above = X.sum_gt + inner_sum;
+            }
+            __syncthreads();
+            if (tid == 0) {
+                S.gt += X.cnt_gt;
+                // restore the caller's correction multiset
+                S.ncorr = X.save_n;
+                for (int c = 0; c < X.save_n; ++c) {
+                    S.corr_v[c] = X.save_v[c];
+                    S.corr_m[c] = X.save_m[c];
+                }
+            }
+            __syncthreads();
+            return;
+        }
+        if (tid == 0) {
+            S.ncorr = X.save_n;
+            for (int c = 0; c < X.save_n; ++c) {
+                S.corr_v[c] = X.save_v[c];
+                S.corr_m[c] = X.save_m[c];
+            }
+        }
+        __syncthreads();
+    }
+    // full-histogram path
+    block_select_desc(S, src, n, rank, lo0, sc0, status);
+    if (sum_above) {
+        const uint32_t theta = S.theta;
+        __syncthreads();
+        float part = 0.f;
+        for (int j = tid; j < n; j += nt) {
+            float v;
+            if (src.get(j, v) && ord_key(v) > theta) part += v;
+        }
+        const float above = block_reduce_f(S, part, 0);
+        if (tid == 0) *sum_above = above;
+        __syncthreads();
+    }
+}
+
 // Layout of the per-head statistics scratch written by scale_stats_kernel (floats per head).
 constexpr int kHeadStat = 8;   // Delta_s, Delta_e, Delta_c, min s, max s, sum s, unused, unused
 constexpr int kStatThreads = 512;
@@ -293,6 +473,8 @@ __global__ void __launch_bounds__(kStatThreads) scale_stats_kernel(int N, ScoreP
                                                                    const uint32_t* __restrict__ mm,
                                                                    float* __restrict__ hstat, int* status) {
     __shared__ SelectShared S;
+    __shared__ BracketShared X;
+    __shared__ float sh_above;
     const int u = blockIdx.x >> 2, task = blockIdx.x & 3;
     const float* a[3] = {a_raw + ((int64_t)u * 3 + 0) * N, a_raw + ((int64_t)u * 3 + 1) * N,
                          a_raw + ((int64_t)u * 3 + 2) * N};
@@ -318,17 +500,10 @@ __global__ void __launch_bounds__(kStatThreads) scale_stats_kernel(int N, ScoreP
             for (int side = 0; side < 2; ++side) {
                 ScaleSrc src{ak, side == 0 ? 1.f : -1.f};
                 const float lo0 = side == 0 ? lok : -(lok + rk);
-                block_select_desc(S, src, N, m, lo0, (float)kBins / rk, status);
-                const uint32_t theta = S.theta;
-                const int gt = S.gt;
+                block_select_bracket(S, X, src, N, (long long)N, m, lo0, (float)kBins / rk, status, &sh_above);
                 __syncthreads();
-                float part = 0.f;
-                for (int j = threadIdx.x; j < N; j += blockDim.x) {
-                    const float v = src.sign * ak[j];
-                    if (ord_key(v) > theta) part += v;
-                }
-                const float above = block_reduce_f(S, part, 0);
-                side_sum[side] = above + (float)(m - gt) * ord_float(theta);
+                side_sum[side] = sh_above + (float)(m - S.gt) * ord_float(S.theta);
+                __syncthreads();
             }
             // side 1 summed the negated values: top_sum - bot_sum = side_sum[0] + side_sum[1]
             gap = (side_sum[0] + side_sum[1]) / ((float)m * rk);
@@ -453,12 +628,13 @@ struct PoolSrc {       // all (head, token) pairs of a group whose key does not 
 __global__ void __launch_bounds__(kStatThreads) safeguard_kernel(int N, int n_safe, const float* __restrict__ a_star,
                                                                  uint32_t* __restrict__ thr, int* status) {
     __shared__ SelectShared S;
+    __shared__ BracketShared X;
     const int u = blockIdx.x;
     if (threadIdx.x == 0) S.ncorr = 0;
     __syncthreads();
     if (n_safe > 0) {
         HeadSrc src{a_star + (int64_t)u * N};
-        block_select_desc(S, src, N, n_safe, 0.f, (float)kBins, status);
+        block_select_bracket(S, X, src, N, (long long)N, n_safe, 0.f, (float)kBins, status, nullptr);
         if (threadIdx.x == 0) {
             thr[(int64_t)u * 2] = S.theta;
             thr[(int64_t)u * 2 + 1] = (uint32_t)(n_safe - S.gt);
@@ -475,6 +651,7 @@ __global__ void __launch_bounds__(kThreads) budget_kernel(int H, int N, int keep
                                                           int32_t* __restrict__ budgets, uint32_t* __restrict__ thr,
                                                           int* status) {
     __shared__ SelectShared S;
+    __shared__ BracketShared X;
     __shared__ uint32_t T[kMaxCorr];
     __shared__ int corr[kMaxCorr], cnt_mid[kMaxCorr], cnt_eq[kMaxCorr];
     const int g = blockIdx.x;
@@ -497,7 +674,8 @@ __global__ void __launch_bounds__(kThreads) budget_kernel(int H, int N, int keep
         if (threadIdx.x == 0) S.ncorr = H;
         __syncthreads();
         PoolSrc src{v, T, N};
-        block_select_desc(S, src, H * N, rest, 0.f, (float)kBins, status);
+        block_select_bracket(S, X, src, H * N, (long long)H * N - (long long)H * n_safe, rest, 0.f, (float)kBins, status,
+                             nullptr);
         tau = S.theta;
         __syncthreads();
     }
