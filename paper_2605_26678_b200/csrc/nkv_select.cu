@@ -108,7 +108,7 @@ __device__ __forceinline__ int block_sum_int(SelectShared& S, int v) {
 // minus the S.corr multiset.  Results in S.theta (ordered key), S.gt (#elements > theta),
 // S.eq (#elements == theta).  lo/scale give the level-0 binning.  Must be called by all threads.
 template <class Src>
-__device__ void block_select_desc(SelectShared& S, const Src& src, int n, int rank, float lo0, float sc0, int* status) {
+__device__ __noinline__ void block_select_desc(SelectShared& S, const Src& src, int n, int rank, float lo0, float sc0, int* status) {
     Levels L;
     L.n = 0;
     float lo = lo0, sc = sc0;
@@ -348,16 +348,24 @@ __device__ void block_select_bracket(SelectShared& S, BracketShared& X, const Sr
             X.p_lo = -INFINITY;
         }
         __syncthreads();
-        SmemSrc ssrc{X.samp};
-        if (sn >= 64 && r_hi >= 1) {
-            block_select_desc(S, ssrc, sn, r_hi, lo0, sc0, status);
-            if (tid == 0) X.p_hi = ord_float(S.theta);
+        // pivots = edges of the value-linear bins that hold the r_hi-th and r_lo-th largest sample elements
+        if (sn >= 64) {
+            for (int b = tid; b < kBins; b += nt) S.hist[b] = 0;
             __syncthreads();
-        }
-        if (sn >= 64 && r_lo <= sn) {
-            block_select_desc(S, ssrc, sn, r_lo, lo0, sc0, status);
-            if (tid == 0) X.p_lo = ord_float(S.theta);
+            for (int i = tid; i < sn; i += nt) atomicAdd(&S.hist[bin_of(X.samp[i], lo0, sc0)], 1);
             __syncthreads();
+            if (r_hi >= 1) {
+                find_bin_desc(S, r_hi);
+                __syncthreads();
+                if (tid == 0) X.p_hi = lo0 + (float)(S.bin + 1) / sc0;
+                __syncthreads();
+            }
+            if (r_lo <= sn) {
+                find_bin_desc(S, r_lo);
+                __syncthreads();
+                if (tid == 0) X.p_lo = lo0 + (float)S.bin / sc0;
+                __syncthreads();
+            }
         }
         const float p_hi = X.p_hi, p_lo = X.p_lo;
         // 3. one pass: count / sum above the bracket, collect the bracket
@@ -465,11 +473,11 @@ __device__ void block_select_bracket(SelectShared& S, BracketShared& X, const Sr
 
 // Layout of the per-head statistics scratch written by scale_stats_kernel (floats per head).
 constexpr int kHeadStat = 8;   // Delta_s, Delta_e, Delta_c, min s, max s, sum s, unused, unused
-constexpr int kStatThreads = 512;
+constexpr int kStatThreads = 256;
 
 // scale_stats: one CTA per (head, task).  Tasks 0..2: the reliability gap of one scale (exact sums of
 // the m largest and m smallest values); task 3: min, max and sum of the surprise over the head.
-__global__ void __launch_bounds__(kStatThreads) scale_stats_kernel(int N, ScoreParams sp, const float* __restrict__ a_raw,
+__global__ void __launch_bounds__(kStatThreads, 4) scale_stats_kernel(int N, ScoreParams sp, const float* __restrict__ a_raw,
                                                                    const uint32_t* __restrict__ mm,
                                                                    float* __restrict__ hstat, int* status) {
     __shared__ SelectShared S;
@@ -625,7 +633,7 @@ struct PoolSrc {       // all (head, token) pairs of a group whose key does not 
 // safeguard: one CTA per head.  The n_safe best tokens of each head are kept unconditionally:
 // thr[2u] = ordered key of the n_safe-th best score, thr[2u+1] = how many tokens tied at that key
 // belong to the safeguard.  (The group kernel below overwrites both words with the final threshold.)
-__global__ void __launch_bounds__(kStatThreads) safeguard_kernel(int N, int n_safe, const float* __restrict__ a_star,
+__global__ void __launch_bounds__(kStatThreads, 4) safeguard_kernel(int N, int n_safe, const float* __restrict__ a_star,
                                                                  uint32_t* __restrict__ thr, int* status) {
     __shared__ SelectShared S;
     __shared__ BracketShared X;
