@@ -219,7 +219,7 @@ int nkv_create(nkv_handle** out, int device) {
     h->scan_lag = 0;   // the separate passes are faster today; see nkv_set_scan_options
     h->scan_hints = 1;
     if (configure_scan_kernels() != cudaSuccess || configure_stream_kernels() != cudaSuccess ||
-        configure_fused_kernels() != cudaSuccess) {
+        configure_fused_kernels() != cudaSuccess || configure_select_kernels() != cudaSuccess) {
         delete h;
         return NKV_ERR_CUDA;
     }

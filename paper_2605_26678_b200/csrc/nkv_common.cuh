@@ -122,6 +122,7 @@ cudaError_t launch_fused_scan(const TensorView& K, int dtype, int G, const Score
                               float* mu_s, float* inv_s, float* inv_e, float* inv_norm, float* a_raw, uint32_t* mm,
                               int* ctrl, int* status, int sm_count, int lag, int hints, cudaStream_t stream,
                               int64_t* launches);
+cudaError_t configure_select_kernels();
 cudaError_t configure_scan_kernels();
 cudaError_t configure_stream_kernels();
 cudaError_t launch_scan_scores(const TensorView& K, int dtype, int G, const ScoreParams& sp, const float* mu_s,

@@ -293,13 +293,14 @@ __device__ __forceinline__ float block_reduce_f(SelectShared& S, float v, int op
 // turns out wrong (rank outside the list, list overflow) the full-histogram path runs instead, so the
 // result is always exact.
 // ------------------------------------------------------------------------------------------
-constexpr int kSample = 1024;
-constexpr int kCandCap = 6144;
+constexpr int kSampleMin = 1024, kSampleMax = 32768;   // sample positions: n / 8, clamped
+constexpr int kCandSmall = 3072;                       // bracket capacity of the per-head kernels
+constexpr int kCandLarge = 12288;                      // ... of the per-group kernel (dynamic shared memory)
 
+template <int CAP>
 struct BracketShared {
-    float samp[kSample];
-    float cand[kCandCap];
-    int samp_n, cand_n, cnt_gt, ok;
+    float cand[CAP];
+    int cand_n, cnt_gt, ok;
     float sum_gt;
     float p_lo, p_hi;
     float save_v[kMaxCorr];
@@ -317,21 +318,26 @@ struct SmemSrc {
 // Same contract as block_select_desc (results in S.theta / S.gt / S.eq, S.corr honoured).  `n_eff` is the
 // number of elements the source really yields (n minus those its get() rejects).  If `sum_above` is not
 // null it receives the sum of the elements strictly greater than theta.
-template <class Src>
-__device__ void block_select_bracket(SelectShared& S, BracketShared& X, const Src& src, int n, long long n_eff,
+template <int CAP, class Src>
+__device__ void block_select_bracket(SelectShared& S, BracketShared<CAP>& X, const Src& src, int n, long long n_eff,
                                      int rank, float lo0, float sc0, int* status, float* sum_above) {
+    constexpr int kCandCap = CAP;
     const int tid = threadIdx.x, nt = blockDim.x;
     bool use_bracket = n > kCandCap && n_eff > 0;
     if (use_bracket) {
-        // 1. strided sample (rejected elements are skipped)
-        if (tid == 0) X.samp_n = 0;
+        // 1. histogram of a strided sample (rejected elements are skipped)
+        const int positions = min(max(n / 8, kSampleMin), kSampleMax);
+        for (int b = tid; b < kBins; b += nt) S.hist[b] = 0;
         __syncthreads();
-        for (int i = tid; i < kSample; i += nt) {
+        int mine = 0;
+        for (int i = tid; i < positions; i += nt) {
             float v;
-            if (src.get((int)(((long long)i * n) / kSample), v)) X.samp[atomicAdd(&X.samp_n, 1)] = v;
+            if (src.get((int)(((long long)i * n) / positions), v)) {
+                atomicAdd(&S.hist[bin_of(v, lo0, sc0)], 1);
+                ++mine;
+            }
         }
-        __syncthreads();
-        const int sn = X.samp_n;
+        const int sn = block_sum_int(S, mine);
         // 2. pivots: sample ranks around rank * sn / n_eff, four standard deviations of the rank error apart
         const float q = (float)rank * (float)sn / (float)n_eff;
         const float sd = sqrtf(fmaxf(q * (1.0f - q / fmaxf((float)sn, 1.0f)), 1.0f));
@@ -350,10 +356,6 @@ __device__ void block_select_bracket(SelectShared& S, BracketShared& X, const Sr
         __syncthreads();
         // pivots = edges of the value-linear bins that hold the r_hi-th and r_lo-th largest sample elements
         if (sn >= 64) {
-            for (int b = tid; b < kBins; b += nt) S.hist[b] = 0;
-            __syncthreads();
-            for (int i = tid; i < sn; i += nt) atomicAdd(&S.hist[bin_of(X.samp[i], lo0, sc0)], 1);
-            __syncthreads();
             if (r_hi >= 1) {
                 find_bin_desc(S, r_hi);
                 __syncthreads();
@@ -481,7 +483,7 @@ __global__ void __launch_bounds__(kStatThreads, 4) scale_stats_kernel(int N, Sco
                                                                    const uint32_t* __restrict__ mm,
                                                                    float* __restrict__ hstat, int* status) {
     __shared__ SelectShared S;
-    __shared__ BracketShared X;
+    __shared__ BracketShared<kCandSmall> X;
     __shared__ float sh_above;
     const int u = blockIdx.x >> 2, task = blockIdx.x & 3;
     const float* a[3] = {a_raw + ((int64_t)u * 3 + 0) * N, a_raw + ((int64_t)u * 3 + 1) * N,
@@ -636,7 +638,7 @@ struct PoolSrc {       // all (head, token) pairs of a group whose key does not 
 __global__ void __launch_bounds__(kStatThreads, 4) safeguard_kernel(int N, int n_safe, const float* __restrict__ a_star,
                                                                  uint32_t* __restrict__ thr, int* status) {
     __shared__ SelectShared S;
-    __shared__ BracketShared X;
+    __shared__ BracketShared<kCandSmall> X;
     const int u = blockIdx.x;
     if (threadIdx.x == 0) S.ncorr = 0;
     __syncthreads();
@@ -659,7 +661,8 @@ __global__ void __launch_bounds__(kThreads) budget_kernel(int H, int N, int keep
                                                           int32_t* __restrict__ budgets, uint32_t* __restrict__ thr,
                                                           int* status) {
     __shared__ SelectShared S;
-    __shared__ BracketShared X;
+    extern __shared__ __align__(16) unsigned char budget_dyn[];
+    BracketShared<kCandLarge>& X = *reinterpret_cast<BracketShared<kCandLarge>*>(budget_dyn);
     __shared__ uint32_t T[kMaxCorr];
     __shared__ int corr[kMaxCorr], cnt_mid[kMaxCorr], cnt_eq[kMaxCorr];
     const int g = blockIdx.x;
@@ -871,14 +874,31 @@ cudaError_t launch_head_scores(int units, int N, const ScoreParams& sp, const fl
 
 size_t head_stat_bytes(int64_t units) { return (size_t)units * kHeadStat * sizeof(float); }
 
+// Raises the dynamic shared-memory limit of the group kernel on the current device (once per device;
+// callers without a handle reach the kernel through launch_budget, which calls this too).
+cudaError_t configure_select_kernels() {
+    static bool done[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(budget_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)sizeof(BracketShared<kCandLarge>));
+    if (e == cudaSuccess && dev >= 0 && dev < 64) done[dev] = true;
+    return e;
+}
+
 cudaError_t launch_budget(int G, int H, int N, int keep, int n_safe, const float* a_star, int32_t* budgets,
                           uint32_t* sel_thresholds, int* status, cudaStream_t stream, int64_t* launches) {
     if (H > kMaxCorr) return cudaErrorInvalidValue;
+    cudaError_t cfg = configure_select_kernels();
+    if (cfg != cudaSuccess) return cfg;
     safeguard_kernel<<<G * H, kStatThreads, 0, stream>>>(N, n_safe, a_star, sel_thresholds, status);
     ++*launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    budget_kernel<<<G, kThreads, 0, stream>>>(H, N, keep, n_safe, a_star, budgets, sel_thresholds, status);
+    budget_kernel<<<G, kThreads, sizeof(BracketShared<kCandLarge>), stream>>>(H, N, keep, n_safe, a_star, budgets,
+                                                                                 sel_thresholds, status);
     ++*launches;
     return cudaGetLastError();
 }
