@@ -228,7 +228,7 @@ __device__ __forceinline__ void treduce(float* v, int l) {
 struct FusedArgs {
     TensorView K;
     ScoreParams sp;
-    int units, lag, hints;
+    int units, lag, hints, strip;   // strip: consecutive tiles of one pass handed out per ticket
     float* block_sums;   // [units, nb, d]: block sums, turned into block means (mu_e) by finalize
     float* mu_s;         // [units, d]
     float* inv_s;        // [units]
@@ -888,17 +888,18 @@ struct Ctl {
         if ((long long)t >= total) return it;
         const long long step = (long long)(t / (unsigned long long)per_step);
         const int j = (int)(t - (unsigned long long)step * (unsigned long long)per_step);
-        if (j < tiles_per_unit) {
+        const int strips = (int)(per_step / 2);
+        if (j < strips) {
             if (step < A.units) {
                 it.kind = 0;
                 it.unit = (int)step;
-                it.tile = j;
+                it.tile = j * A.strip;   // first tile of the strip
                 return it;
             }
         } else if (step >= A.lag) {
             it.kind = 1;
             it.unit = (int)(step - A.lag);
-            it.tile = j - tiles_per_unit;
+            it.tile = (j - strips) * A.strip;
             return it;
         }
         it.pad = 1;
@@ -916,6 +917,10 @@ struct Ctl {
         return it;
     }
     __device__ __forceinline__ Item fetch() { return item_from(take_ticket()); }
+    // tiles that follow `it` in its strip
+    __device__ __forceinline__ int rest_of_strip(const Item& it) const {
+        return it.kind == 2 ? 0 : min(A.strip, tiles_per_unit - it.tile) - 1;
+    }
     // publish `it` as item number `seq` in `slot` and start its copy
     __device__ __forceinline__ void issue(int slot, Item it, int seq) {
         volatile Item* d = item + slot;
@@ -986,16 +991,29 @@ __global__ void __launch_bounds__(Geo<T, D>::kThreads + 32, 1) fused_scan_kernel
         // ------------------------------------------------------------------ control warp
         // All 32 lanes run the loop together (the per-item barrier is warp-aligned); lane 0 works.
         const int lane = tid - G::kThreads;
-        Ctl<T, D> C{A, tiles, item, full, abort_flag, tiles_per_unit, 2LL * tiles_per_unit,
-                    ((long long)A.units + A.lag) * 2LL * tiles_per_unit,
+        const long long strips = (tiles_per_unit + A.strip - 1) / A.strip;
+        Ctl<T, D> C{A, tiles, item, full, abort_flag, tiles_per_unit, 2LL * strips,
+                    ((long long)A.units + A.lag) * 2LL * strips,
                     A.hints ? l2_policy_keep() : l2_policy_normal(), A.hints ? l2_policy_stream() : l2_policy_normal()};
         Item nxt;   // the ticket after the two in flight, fetched ahead of time (lane 0)
         nxt.kind = 2;
         nxt.unit = nxt.tile = nxt.pad = 0;
+        int left = 0;   // tiles that follow `nxt` in its strip
+        auto advance = [&]() {   // nxt <- the item after nxt (blocking ticket fetch when the strip is used up)
+            if (left > 0) {
+                ++nxt.tile;
+                --left;
+            } else {
+                nxt = C.fetch();
+                left = C.rest_of_strip(nxt);
+            }
+        };
         if (lane == 0) {
-            C.issue(0, C.fetch(), 0);
-            C.issue(1, C.fetch(), 1);
-            nxt = C.fetch();
+            advance();
+            C.issue(0, nxt, 0);
+            advance();
+            C.issue(1, nxt, 1);
+            advance();
         }
         __syncwarp();
         bar_sync(kBarEnd, kAll);   // start: both descriptors are visible
@@ -1011,7 +1029,8 @@ __global__ void __launch_bounds__(Geo<T, D>::kThreads + 32, 1) fused_scan_kernel
                 // Two global atomics per item, both in flight at once: the next ticket (needed at the
                 // next item barrier) and the tile counter of the head (needed now).  No fence here: the
                 // compute threads fence their block sums before the item barrier.
-                const bool more = nxt.kind != 2 && *reinterpret_cast<volatile int*>(abort_flag) == 0;
+                const bool in_strip = left > 0;
+                const bool more = !in_strip && nxt.kind != 2 && *reinterpret_cast<volatile int*>(abort_flag) == 0;
                 unsigned long long t_raw = ~0ULL;
                 if (more) t_raw = C.take_ticket();
                 int fin_unit = -1;
@@ -1036,8 +1055,15 @@ __global__ void __launch_bounds__(Geo<T, D>::kThreads + 32, 1) fused_scan_kernel
                         }
                     }
                 }
-                if (more) nxt = C.item_from(t_raw);
-                else nxt.kind = 2;
+                if (in_strip) {
+                    ++nxt.tile;
+                    --left;
+                } else if (more) {
+                    nxt = C.item_from(t_raw);
+                    left = C.rest_of_strip(nxt);
+                } else {
+                    nxt.kind = 2;
+                }
             }
             __syncwarp();
         }
@@ -1163,6 +1189,7 @@ cudaError_t launch_fused_scan(const TensorView& K, int dtype, int G, const Score
     A.units = G * K.H;
     A.lag = lag < 1 ? 1 : lag;
     A.hints = hints;
+    A.strip = 4;
     A.block_sums = block_sums;
     A.mu_s = mu_s;
     A.inv_s = inv_s;
