@@ -9,7 +9,9 @@ namespace nkv {
 
 namespace {
 
-constexpr int kRowsPerBatch = 32;
+constexpr int kRowsPerBatch = 32;   // in-place kernel
+constexpr int kGatherRows = 64;     // out-of-place kernel: rows per batch
+constexpr int kGatherInFlight = 8;  // 16-byte loads each thread issues before its first store
 
 struct GatherArgs {
     const unsigned char* src[2];
@@ -23,12 +25,14 @@ struct GatherArgs {
 
 __global__ void __launch_bounds__(256) gather_kernel(GatherArgs A, const int32_t* __restrict__ idx,
                                                      const int32_t* __restrict__ head_offsets) {
-    __shared__ int64_t src_off[2][kRowsPerBatch];
-    const int64_t nbatch = (A.total_rows + kRowsPerBatch - 1) / kRowsPerBatch;
+    __shared__ int64_t src_off[2][kGatherRows];
+    const int64_t nbatch = (A.total_rows + kGatherRows - 1) / kGatherRows;
+    const int cpr0 = A.row_bytes[0] >> 4, cpr1 = A.dst[1] ? (A.row_bytes[1] >> 4) : 0;   // 16-byte chunks per row
+    const int total0 = A.dst[0] ? kGatherRows * cpr0 : 0, total = total0 + kGatherRows * cpr1;
     for (int64_t batch = blockIdx.x; batch < nbatch; batch += gridDim.x) {
-        const int64_t row0 = batch * kRowsPerBatch;
+        const int64_t row0 = batch * kGatherRows;
         __syncthreads();
-        if (threadIdx.x < kRowsPerBatch) {
+        if (threadIdx.x < kGatherRows) {
             const int64_t J = row0 + threadIdx.x;
             int64_t o0 = -1, o1 = -1;
             if (J < A.total_rows) {
@@ -49,36 +53,30 @@ __global__ void __launch_bounds__(256) gather_kernel(GatherArgs A, const int32_t
             src_off[1][threadIdx.x] = o1;
         }
         __syncthreads();
+        // the chunks of the batch's K rows, then of its V rows, form one list; every thread keeps
+        // kGatherInFlight loads in flight before it stores
+        for (int c0 = threadIdx.x; c0 < total; c0 += 256 * kGatherInFlight) {
+            uint4 q[kGatherInFlight];
+            uint4* dst[kGatherInFlight];
 #pragma unroll
-        for (int t = 0; t < 2; ++t) {
-            if (A.dst[t] == nullptr) continue;
-            const int cpr = A.row_bytes[t] >> 4;  // 16-byte chunks per row
-            const int total = kRowsPerBatch * cpr;
-            for (int c0 = threadIdx.x; c0 < total; c0 += 256 * 4) {
-                uint4 q[4];
-                bool ok[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int c = c0 + e * 256;
-                    ok[e] = false;
-                    if (c < total) {
-                        const int r = c / cpr;
-                        const int64_t so = src_off[t][r];
-                        if (so >= 0) {
-                            ok[e] = true;
-                            q[e] = __ldcs(reinterpret_cast<const uint4*>(A.src[t] + so) + (c - r * cpr));
-                        }
-                    }
-                }
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int c = c0 + e * 256;
-                    if (ok[e]) {
-                        const int r = c / cpr;
-                        __stcs(reinterpret_cast<uint4*>(A.dst[t] + (row0 + r) * A.row_bytes[t]) + (c - r * cpr), q[e]);
+            for (int e = 0; e < kGatherInFlight; ++e) {
+                const int c = c0 + e * 256;
+                dst[e] = nullptr;
+                if (c < total) {
+                    const int t = c >= total0 ? 1 : 0;
+                    const int cc = t ? c - total0 : c;
+                    const int cpr = t ? cpr1 : cpr0;
+                    const int r = cc / cpr, k = cc - r * cpr;
+                    const int64_t so = src_off[t][r];
+                    if (so >= 0) {
+                        q[e] = __ldcs(reinterpret_cast<const uint4*>(A.src[t] + so) + k);
+                        dst[e] = reinterpret_cast<uint4*>(A.dst[t] + (row0 + r) * A.row_bytes[t]) + k;
                     }
                 }
             }
+#pragma unroll
+            for (int e = 0; e < kGatherInFlight; ++e)
+                if (dst[e]) __stcs(dst[e], q[e]);
         }
     }
 }
@@ -156,7 +154,7 @@ cudaError_t launch_gather(const TensorView& K, int k_elem_bytes, const TensorVie
                           const int32_t* idx, const int32_t* head_offsets, int64_t idx_capacity, void* K_out,
                           void* V_out, int sm_count, cudaStream_t stream, int64_t* launches) {
     GatherArgs A = make_args(K, k_elem_bytes, V, v_elem_bytes, G, idx_capacity, K_out, V_out);
-    const int64_t nbatch = (A.total_rows + kRowsPerBatch - 1) / kRowsPerBatch;
+    const int64_t nbatch = (A.total_rows + kGatherRows - 1) / kGatherRows;
     if (nbatch == 0) return cudaSuccess;
     int64_t grid = (int64_t)sm_count * 8;
     if (grid > nbatch) grid = nbatch;

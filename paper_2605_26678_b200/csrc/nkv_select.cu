@@ -542,7 +542,7 @@ __global__ void __launch_bounds__(kStatThreads, 4) scale_stats_kernel(int N, Sco
 // mix: elementwise.  Every CTA recomputes its head's three weights and surprise constants (a handful of
 // flops) and routes a chunk of tokens: a* = (1 - alpha) * blend + alpha * max, sinks pinned to +inf.
 constexpr int kMixThreads = 256;
-constexpr int kMixPerThread = 32;
+constexpr int kMixPerThread = 8;
 __global__ void __launch_bounds__(kMixThreads) mix_kernel(int N, ScoreParams sp, const float* __restrict__ a_raw,
                                                           const uint32_t* __restrict__ mm,
                                                           const float* __restrict__ hstat, float* __restrict__ a_star,
