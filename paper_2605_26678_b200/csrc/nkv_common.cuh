@@ -91,6 +91,25 @@ __device__ __forceinline__ float warp_min(float v) {
     return v;
 }
 
+// One m16n8k16 bf16 tensor-core product with fp32 accumulation: c += a * b.
+__device__ __forceinline__ void mma_bf16_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// x = hi + mid + lo with all three in bf16: together they carry the 24 mantissa bits of an fp32 number.
+__device__ __forceinline__ void split3_bf16(float x, __nv_bfloat16* out, int stride) {
+    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+    const float r1 = x - __bfloat162float(hi);
+    const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+    const float r2 = r1 - __bfloat162float(mid);
+    out[0] = hi;
+    out[stride] = mid;
+    out[2 * stride] = __float2bfloat16_rn(r2);
+}
+
 __device__ __forceinline__ void set_status(int* status, int code, int detail) {
     if (atomicCAS(&status[kStatusCode], 0, code) == 0) status[kStatusDetail] = detail;
 }

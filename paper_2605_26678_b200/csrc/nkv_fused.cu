@@ -614,23 +614,6 @@ __device__ __forceinline__ void pass_b(const FusedArgs& A, int u, int tile_idx, 
 // 0..2 = mu_s hi/mid/lo, 3..5 = mu_e hi/mid/lo, 6..7 = 0.  The contraction index may be visited in any
 // order, so lane (g, t) of a warp takes the 16-byte chunks t, t+4, t+8, ... of rows g and g+8 straight
 // from the staged tile (no transposition, no conversion) and the right-hand side uses the same order.
-__device__ __forceinline__ void mma_bf16_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-__device__ __forceinline__ void split3_bf16(float x, __nv_bfloat16* out, int stride) {
-    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
-    const float r1 = x - __bfloat162float(hi);
-    const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
-    const float r2 = r1 - __bfloat162float(mid);
-    out[0] = hi;
-    out[stride] = mid;
-    out[2 * stride] = __float2bfloat16_rn(r2);
-}
-
 // Requires block % 16 == 0 and at most four episodic blocks per tile.  `pp`/`invs` staging as in pass_b;
 // behind the staged floats `pp` also holds the split right-hand sides [nblk][8][D] in bf16.
 template <int D>
