@@ -630,8 +630,26 @@ stream_b_mma_kernel(TensorView K, ScoreParams sp, int units, const float* __rest
             bulk_load(dst + off, src + off, min(16384u, bytes - off), &full[buf]);
     };
 
+    // anchors of a tile, one column per thread (threads < D), fetched one iteration ahead
+    struct Anchors {
+        float ms, me[4], sc;
+    };
+    auto load_anchors = [&](long long t2, Anchors& an) {
+        const int u2 = (int)(t2 / tiles_per_unit);
+        const int blk2 = ((int)(t2 - (long long)u2 * tiles_per_unit) * TILE) / b;
+        const int n2 = min(nb - blk2, TILE / b);
+        an.ms = mu_s[(int64_t)u2 * D + tid];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) an.me[q] = q < n2 ? mu_e[((int64_t)u2 * nb + blk2 + q) * D + tid] : 0.f;
+        an.sc = tid == 0 ? inv_s[u2] : (tid <= n2 ? inv_e[(int64_t)u2 * nb + blk2 + tid - 1] : 0.f);
+    };
+    uint32_t* keys = reinterpret_cast<uint32_t*>(red);   // [2][4] ordered min/max keys of the tile in flight
+    if (tid < 8) keys[tid] = (tid & 1) ? 0u : 0xffffffffu;
+
     long long tt = blockIdx.x;
     if (tt < total && tid == 0) issue(tt, 0);
+    Anchors cur_an;
+    if (tt < total && tid < D) load_anchors(tt, cur_an);
     int it = 0;
     for (; tt < total; tt += gridDim.x, ++it) {
         const int buf = it & 1;
@@ -644,18 +662,20 @@ stream_b_mma_kernel(TensorView K, ScoreParams sp, int units, const float* __rest
         const int nblk = min(nb - blk0, TILE / b);
         const int rows = min(N, i0 + TILE) - i0;
 
-        // split right-hand sides of this tile's blocks (one column of the anchors per thread)
+        // split right-hand sides of this tile's blocks from the prefetched anchors, then start the next fetch
         if (tid < D) {
-            const float ms = mu_s[(int64_t)u * D + tid];
-            for (int q = 0; q < nblk; ++q) {
-                __nv_bfloat16* r = rhs + (size_t)q * 8 * D + tid;
-                split3_bf16(ms, r, D);
-                split3_bf16(mu_e[((int64_t)u * nb + blk0 + q) * D + tid], r + 3 * D, D);
-                r[6 * D] = __float2bfloat16_rn(0.f);
-                r[7 * D] = __float2bfloat16_rn(0.f);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (q < nblk) {
+                    __nv_bfloat16* r = rhs + (size_t)q * 8 * D + tid;
+                    split3_bf16(cur_an.ms, r, D);
+                    split3_bf16(cur_an.me[q], r + 3 * D, D);
+                    r[6 * D] = __float2bfloat16_rn(0.f);
+                    r[7 * D] = __float2bfloat16_rn(0.f);
+                }
             }
-            if (tid == 0) scal[0] = inv_s[u];
-            else if (tid <= nblk) scal[tid] = inv_e[(int64_t)u * nb + blk0 + tid - 1];
+            if (tid <= nblk) scal[tid] = cur_an.sc;
+            if (tn < total) load_anchors(tn, cur_an);
         }
         // each lane finishes one of the four results of its quad: t=0: a_s(row g), t=1: a_e(row g),
         // t=2: a_s(row g+8), t=3: a_e(row g+8); its key's reciprocal norm is fetched before the copy is awaited
@@ -717,10 +737,32 @@ stream_b_mma_kernel(TensorView K, ScoreParams sp, int units, const float* __rest
                 }
             }
         }
-        cta_minmax_to_global(lo_s, hi_s, red, C::kWarps, &mm[(int64_t)u * 6 + 0], &mm[(int64_t)u * 6 + 1]);
-        __syncthreads();
-        cta_minmax_to_global(lo_e, hi_e, red, C::kWarps, &mm[(int64_t)u * 6 + 2], &mm[(int64_t)u * 6 + 3]);
-        __syncthreads();   // the tile, rhs and scal may be overwritten from here on
+        lo_s = warp_min(lo_s);
+        hi_s = warp_max(hi_s);
+        lo_e = warp_min(lo_e);
+        hi_e = warp_max(hi_e);
+        uint32_t* kk = keys + (it & 1) * 4;
+        if (lane == 0) {
+            if (lo_s <= hi_s) {
+                atomicMin(&kk[0], ord_key(lo_s));
+                atomicMax(&kk[1], ord_key(hi_s));
+            }
+            if (lo_e <= hi_e) {
+                atomicMin(&kk[2], ord_key(lo_e));
+                atomicMax(&kk[3], ord_key(hi_e));
+            }
+        }
+        __syncthreads();   // the tile, rhs and scal may be overwritten from here on; the tile's keys are final
+        if (tid < 4) {
+            const uint32_t v = kk[tid];
+            if (tid & 1) {
+                if (v != 0u) atomicMax(&mm[(int64_t)u * 6 + tid], v);
+                kk[tid] = 0u;
+            } else {
+                if (v != 0xffffffffu) atomicMin(&mm[(int64_t)u * 6 + tid], v);
+                kk[tid] = 0xffffffffu;
+            }
+        }
     }
 }
 
