@@ -586,7 +586,8 @@ struct BMmaCfg {
     static constexpr int kIters = (TILE / 16 + kWarps - 1) / kWarps;
     static constexpr size_t kTileBytes = (size_t)TILE * kRowBytes;
     static constexpr size_t kRhsBytes = (size_t)4 * 8 * D * 2;           // [4 blocks][8 columns][D] bf16
-    static constexpr size_t kSmem = 2 * kTileBytes + kRhsBytes + 8 * 4 + 64 * 4 + 64;
+    static constexpr int kBufs = 3;   // two tiles in flight while one is consumed: the pass is a pure stream
+    static constexpr size_t kSmem = kBufs * kTileBytes + kRhsBytes + 8 * 4 + 64 * 4 + 64;
 };
 
 template <int D, int TILE>
@@ -599,8 +600,8 @@ stream_b_mma_kernel(TensorView K, ScoreParams sp, int units, const float* __rest
     constexpr int kCh = D / 32;   // 16-byte chunks per lane and row
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* tiles = smem;
-    __nv_bfloat16* rhs = reinterpret_cast<__nv_bfloat16*>(smem + 2 * C::kTileBytes);
-    float* scal = reinterpret_cast<float*>(smem + 2 * C::kTileBytes + C::kRhsBytes);   // [0] 1/|mu_s|, [1..4] 1/|mu_e|
+    __nv_bfloat16* rhs = reinterpret_cast<__nv_bfloat16*>(smem + C::kBufs * C::kTileBytes);
+    float* scal = reinterpret_cast<float*>(smem + C::kBufs * C::kTileBytes + C::kRhsBytes);   // [0] 1/|mu_s|, [1..4] 1/|mu_e|
     float* red = scal + 8;
     uint64_t* full = reinterpret_cast<uint64_t*>(red + 64);
 
@@ -610,8 +611,7 @@ stream_b_mma_kernel(TensorView K, ScoreParams sp, int units, const float* __rest
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
 
     if (tid == 0) {
-        mbar_init(&full[0], 1);
-        mbar_init(&full[1], 1);
+        for (int i = 0; i < C::kBufs; ++i) mbar_init(&full[i], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -647,14 +647,18 @@ stream_b_mma_kernel(TensorView K, ScoreParams sp, int units, const float* __rest
     if (tid < 8) keys[tid] = (tid & 1) ? 0u : 0xffffffffu;
 
     long long tt = blockIdx.x;
-    if (tt < total && tid == 0) issue(tt, 0);
+    if (tid == 0) {
+        if (tt < total) issue(tt, 0);
+        if (tt + gridDim.x < total) issue(tt + gridDim.x, 1);
+    }
     Anchors cur_an;
     if (tt < total && tid < D) load_anchors(tt, cur_an);
     int it = 0;
     for (; tt < total; tt += gridDim.x, ++it) {
-        const int buf = it & 1;
+        const int buf = it % C::kBufs;
         const long long tn = tt + gridDim.x;
-        if (tn < total && tid == 0) issue(tn, buf ^ 1);
+        // the buffer of the tile before this one was released by the barrier that ended it
+        if (tt + 2LL * gridDim.x < total && tid == 0) issue(tt + 2LL * gridDim.x, (it + 2) % C::kBufs);
         const int u = (int)(tt / tiles_per_unit);
         const int i0 = (int)(tt - (long long)u * tiles_per_unit) * TILE;
         const unsigned char* tile = tiles + (size_t)buf * C::kTileBytes;
@@ -688,7 +692,7 @@ stream_b_mma_kernel(TensorView K, ScoreParams sp, int units, const float* __rest
         }
         __syncthreads();
         const float rs = scal[0];
-        if (!mbar_wait(&full[buf], (uint32_t)((it >> 1) & 1), status, 403)) return;
+        if (!mbar_wait(&full[buf], (uint32_t)((it / C::kBufs) & 1), status, 403)) return;
 
         float lo_s = INFINITY, hi_s = -INFINITY, lo_e = INFINITY, hi_e = -INFINITY;
 #pragma unroll
