@@ -267,65 +267,16 @@ __device__ __forceinline__ void range_sum(const float* pp, int l, int s0, int s1
     }
 }
 
-// Anchors of the next pass-B item, fetched into registers by the first D threads while the current
-// item is still being computed (the two dependent global round trips would otherwise sit at the start
-// of every pass-B item).  Thread c holds column c of mu_s and of up to four block means; thread 0 also
-// holds 1/||mu_s||, threads 1..nblk hold 1/||mu_e|| of block (thread - 1).
-struct Prefetched {
-    int unit, tile, have, flag, blk0, nblk;
-    float mu, me[4], aux;
-};
-
-__device__ __forceinline__ int ld_relaxed(const int* p) {
-    int v;
-    asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-
-// Step 1, at the start of an item: look at the next item; if it is a pass-B item, start reading its
-// head's "anchors published" flag.  Nothing here waits: the value is first used in step 2.
-template <typename T, int D>
-__device__ __forceinline__ void prefetch_flag(const FusedArgs& A, const volatile Item* next, int next_seq,
-                                              Prefetched& pre) {
-    using G = Geo<T, D>;
-    pre.have = 0;
-    pre.flag = 0;
-    if (threadIdx.x >= D || next->pad != next_seq || next->kind != 1) return;
-    pre.unit = next->unit;
-    pre.tile = next->tile;
-    const int b = A.sp.block, nb = A.sp.nblocks;
-    pre.blk0 = (pre.tile * G::kTile) / b;
-    pre.nblk = min(nb - pre.blk0, G::kTile / b);
-    if (pre.nblk > 4) return;
-    pre.flag = ld_relaxed(A.ctrl + kCtrlHeader + A.units + pre.unit);
-}
-// Step 2, a barrier later: if the flag was up, fetch the anchors (L2 loads that are issued only after
-// the flag's value has arrived, so they cannot return anything older than what the flag announces).
-template <typename T, int D>
-__device__ __forceinline__ void prefetch_data(const FusedArgs& A, Prefetched& pre) {
-    if (pre.flag == 0) return;
-    const int tid = threadIdx.x, u = pre.unit, nb = A.sp.nblocks;
-    pre.mu = __ldcg(A.mu_s + (int64_t)u * D + tid);
-#pragma unroll
-    for (int q = 0; q < 4; ++q)
-        pre.me[q] = q < pre.nblk ? __ldcg(A.block_sums + ((int64_t)u * nb + pre.blk0 + q) * D + tid) : 0.f;
-    pre.aux = tid == 0 ? __ldcg(A.inv_s + u)
-                       : (tid <= pre.nblk ? __ldcg(A.inv_e + (int64_t)u * nb + pre.blk0 + tid - 1) : 0.f);
-    pre.have = 1;
-}
-
 // ---------------------------------------------------------------------------- pass A on one tile
 template <typename T, int D>
 __device__ __forceinline__ void pass_a(const FusedArgs& A, int u, int tile_idx, unsigned char* tile, float* pp,
-                                       float* invs, uint32_t* mmk, uint64_t* full, uint32_t parity, int* abort_flag,
-                                       const volatile Item* next, int next_seq, Prefetched& pre) {
+                                       float* invs, uint32_t* mmk, uint64_t* full, uint32_t parity, int* abort_flag) {
     using G = Geo<T, D>;
     constexpr int NP = G::kNP;
     constexpr int L = G::kL;
     const int N = A.K.N, W = A.sp.window;
     const int tid = threadIdx.x, grp = tid / L, l = tid % L;
     const int i0 = tile_idx * G::kTile;
-    prefetch_flag<T, D>(A, next, next_seq, pre);
 
     // rows outside [0, N) are not copied: zero them (disjoint from the bytes in flight)
     const int r0 = max(0, i0 - kHalo), r1 = min(N, i0 + G::kTile);
@@ -379,7 +330,6 @@ __device__ __forceinline__ void pass_a(const FusedArgs& A, int u, int tile_idx, 
         G::store_vec(pp + (size_t)grp * D, l, acc);
     }
     bar_sync(kBarCompute, G::kThreads);
-    prefetch_data<T, D>(A, pre);
     // ---- S1b: inclusive prefix of the segment sums inside every 64-row chunk (one column per task)
     for (int task = tid; task < (G::kRows / 64) * D; task += G::kThreads) {
         const int c64 = task / D, col = task - c64 * D;
@@ -479,285 +429,247 @@ __device__ __forceinline__ void pass_a(const FusedArgs& A, int u, int tile_idx, 
     }
 }
 
-// ---------------------------------------------------------------------------- pass B on one tile
-// The first D threads stage the anchors in shared memory: `pp` = mu_s [D], then the block means of
-// the tile's blocks [nblk][D]; `invs` = 1/||mu_s|| at [0], 1/||mu_e|| of the tile's blocks at [1 ..].
-template <typename T, int D>
-__device__ __forceinline__ void pass_b(const FusedArgs& A, int u, int tile_idx, const unsigned char* tile, float* pp,
-                                       float* invs, uint32_t* mmk, uint64_t* full, uint32_t parity, int* abort_flag,
-                                       const volatile Item* next, int next_seq, Prefetched& pre) {
-    using G = Geo<T, D>;
-    constexpr int NP = G::kNP;
-    constexpr int L = G::kL;
-    const int N = A.K.N, b = A.sp.block, nb = A.sp.nblocks;
-    const int tid = threadIdx.x, grp = tid / L, l = tid % L;
-    const int i0 = tile_idx * G::kTile;
-    const int blk0 = i0 / b;
-    const int nblk = min(nb - blk0, G::kTile / b);
+// ---------------------------------------------------------------------------- pass B (own warp group)
+// Four warps beside the pass-A threads take pass-B tiles from their own ticket counter, wait (bounded)
+// until the tile's head has published its anchors, and stream the tile through a private buffer in
+// sub-tiles.  Pass A never waits for pass B, so the two cannot deadlock; pass B simply trails pass A as
+// closely as the anchors allow, which is what keeps its reads in L2.
+//
+// bf16 keys with blocks of 16k rows: the two dots of a key against mu_s and mu_e are a skinny matrix
+// product [16 keys x d] x [d x 8] on the tensor cores.  The fp32 anchors are split three ways into bf16
+// (hi + mid + lo carries all 24 mantissa bits), products of bf16 numbers are exact in fp32 and the
+// accumulation is fp32.  Columns: 0..2 = mu_s hi/mid/lo, 3..5 = mu_e hi/mid/lo, 6..7 = 0.  The
+// contraction index may be visited in any order, so lane (g, t) takes the 16-byte chunks t, t+4, ... of
+// rows g and g+8 straight from the staged rows and the right-hand side uses the same order.
+// Other cases (fp32 keys, odd block sizes) use packed FMAs with the anchors read from L2.
+constexpr int kBThreads = 128;
+constexpr int kBarB = 3;
 
-    if (tid < D) {
-        if (pre.have && pre.unit == u && pre.tile == tile_idx) {
-            // the anchors were fetched while the previous item was being computed
-            pp[tid] = pre.mu;
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-                if (q < nblk) pp[(1 + q) * D + tid] = pre.me[q];
-            if (tid <= nblk) invs[tid] = pre.aux;
-        } else {
-            // wait (bounded) until the head's anchors have been published
-            const int* ready = A.ctrl + kCtrlHeader + A.units + u;
-            bool ok = ld_acquire(ready) != 0;
-            if (!ok && *reinterpret_cast<volatile int*>(abort_flag) == 0) {
-                const unsigned long long t0 = now_ns();
-                for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
-                    if (ld_acquire(ready) != 0) {
-                        ok = true;
-                        break;
+template <typename T, int D>
+struct BGeo {
+    using G = Geo<T, D>;
+    static constexpr int kBytes = G::kRowBytes >= 512 ? 16384 : 32768;   // private buffer of the group
+    static constexpr int kRows = kBytes / G::kRowBytes;                  // rows per sub-tile
+    static constexpr int kAnchorBytes = 4 * 8 * D * 2;                   // split right-hand sides [4][8][D] bf16
+};
+
+template <typename T, int D>
+__device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* tileB, __nv_bfloat16* rhs, float* bsc,
+                                             int* bslot, uint64_t* mbarB, int* abort_flag) {
+    using G = Geo<T, D>;
+    using B = BGeo<T, D>;
+    constexpr int NP = G::kNP, L = G::kL;
+    const int N = A.K.N, b = A.sp.block, nb = A.sp.nblocks;
+    const int bt = threadIdx.x - (G::kThreads + 32), warp = bt >> 5, lane = bt & 31;
+    const int tiles_per_unit = (N + G::kTile - 1) / G::kTile;
+    const long long total = (long long)A.units * tiles_per_unit;
+    unsigned long long* ticket = reinterpret_cast<unsigned long long*>(A.ctrl + 2);
+    const uint64_t policy = A.hints ? l2_policy_stream() : l2_policy_normal();
+    const bool mma_path = sizeof(T) == 2 && b % 16 == 0 && B::kRows <= 4 * b;
+    uint32_t copies = 0;   // copies awaited so far (mbarrier parity)
+
+    for (;;) {
+        if (bt == 0) {
+            int u = -1, tile = 0;
+            if (*reinterpret_cast<volatile int*>(abort_flag) == 0) {
+                const unsigned long long t = atomicAdd(ticket, 1ULL);
+                if ((long long)t < total) {
+                    u = (int)(t / (unsigned long long)tiles_per_unit);
+                    tile = (int)(t - (unsigned long long)u * tiles_per_unit);
+                    // wait (bounded) until the head's anchors have been published
+                    const int* ready = A.ctrl + kCtrlHeader + A.units + u;
+                    bool ok = ld_acquire(ready) != 0;
+                    if (!ok) {
+                        const unsigned long long t0 = now_ns();
+                        for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+                            if (ld_acquire(ready) != 0) {
+                                ok = true;
+                                break;
+                            }
+                            __nanosleep(256);
+                            if ((spin & 15u) == 15u && (*reinterpret_cast<volatile int*>(abort_flag) != 0 ||
+                                                        now_ns() - t0 > kWaitLimitNs))
+                                break;
+                        }
                     }
-                    __nanosleep(64);
-                    if ((spin & 63u) == 63u && now_ns() - t0 > kWaitLimitNs) break;
+                    if (!ok) {
+                        set_status(A.status, NKV_ERR_TIMEOUT, 502);
+                        *abort_flag = 1;
+                        u = -1;
+                    }
                 }
             }
-            if (!ok) {
-                set_status(A.status, NKV_ERR_TIMEOUT, 502);
+            bslot[0] = u;
+            bslot[1] = tile;
+        }
+        bar_sync(kBarB, kBThreads);
+        const int u = bslot[0], tile_idx = bslot[1];
+        if (u < 0) break;
+        const int g = u / A.K.H, h = u % A.K.H;
+        const unsigned char* base = reinterpret_cast<const unsigned char*>(A.K.ptr) +
+                                    ((int64_t)g * A.K.stride_g + (int64_t)h * A.K.stride_h) * (int64_t)sizeof(T);
+        float lo_s = INFINITY, hi_s = -INFINITY, lo_e = INFINITY, hi_e = -INFINITY;
+        const float rs = __ldcg(A.inv_s + u);
+
+        for (int r0 = tile_idx * G::kTile; r0 < min(N, (tile_idx + 1) * G::kTile); r0 += B::kRows) {
+            const int rows = min(N, r0 + B::kRows) - r0;
+            if (bt == 0) {
+                const uint32_t bytes = (uint32_t)rows * G::kRowBytes;
+                fence_async_smem();
+                mbar_expect_tx(mbarB, bytes);
+                bulk_load(tileB, base + (int64_t)r0 * G::kRowBytes, bytes, mbarB, policy);
+            }
+            const int blk0 = r0 / b;
+            if (mma_path) {
+                if constexpr (sizeof(T) == 2) {
+                    // split right-hand sides of the sub-tile's blocks, one anchor column per thread
+                    const int nblk = min(nb - blk0, max(1, B::kRows / b));
+                    if (bt < D) {
+                        const float mu = __ldcg(A.mu_s + (int64_t)u * D + bt);
+                        for (int q = 0; q < nblk; ++q) {
+                            __nv_bfloat16* r = rhs + (size_t)q * 8 * D + bt;
+                            split3_bf16(mu, r, D);
+                            split3_bf16(__ldcg(A.block_sums + ((int64_t)u * nb + blk0 + q) * D + bt), r + 3 * D, D);
+                            r[6 * D] = __float2bfloat16_rn(0.f);
+                            r[7 * D] = __float2bfloat16_rn(0.f);
+                        }
+                        if (bt < nblk) bsc[bt] = __ldcg(A.inv_e + (int64_t)u * nb + blk0 + bt);
+                    }
+                }
+            }
+            bar_sync(kBarB, kBThreads);   // right-hand sides visible
+            if (!mbar_wait(mbarB, copies & 1u, abort_flag)) {
+                set_status(A.status, NKV_ERR_TIMEOUT, 503);
                 *abort_flag = 1;
             }
-            pp[tid] = __ldcg(A.mu_s + (int64_t)u * D + tid);
-            for (int q = 0; q < nblk; ++q) pp[(1 + q) * D + tid] = __ldcg(A.block_sums + ((int64_t)u * nb + blk0 + q) * D + tid);
-            if (tid == 0) invs[0] = __ldcg(A.inv_s + u);
-            if (tid >= 1 && tid <= nblk) invs[tid] = __ldcg(A.inv_e + (int64_t)u * nb + blk0 + tid - 1);
-    
-        }
-    }
-    bar_sync(kBarCompute, G::kThreads);
-    prefetch_flag<T, D>(A, next, next_seq, pre);
-
-    const int gi0 = i0 + grp * kSeg;
-    // Whole warps take part (kTile threads = a multiple of 32): the shuffles below name every lane.
-    // Groups past the end of the sequence compute on stale rows and write nothing.
-    const bool active = grp < G::kTile / kSeg;
-    float inv_mine = 0.f;
-    F2 ms[NP], me[NP];
-    float rs = 0.f, re = 0.f;
-    if (active) {
-        const int q = min(max(min(gi0 / b, nb - 1) - blk0, 0), nblk - 1);
-        G::load_vec(pp, l, ms);
-        G::load_vec(pp + (1 + q) * D, l, me);
-        rs = invs[0];
-        re = invs[1 + q];
-        const int o_mine = L == 16 ? (l >> 1) : l;   // the token this lane finishes
-        if (gi0 + o_mine < N) inv_mine = __ldcg(A.inv_norm + (int64_t)u * N + gi0 + o_mine);
-    }
-    if (!mbar_wait(full, parity, abort_flag)) {
-        set_status(A.status, NKV_ERR_TIMEOUT, 503);
-        *abort_flag = 1;
-    }
-    if (active) {
-        float part[16];
+            ++copies;
+            if (mma_path) {
+                if constexpr (sizeof(T) == 2) {
+                    constexpr int kCh = D / 32;
+                    const int gq = lane >> 2, t = lane & 3;
+                    const int row_in_block = gq + ((t & 2) ? 8 : 0);
+                    for (int rb = warp; rb * 16 < rows; rb += kBThreads / 32) {
+                        const int rr = rb * 16;
+                        const int q = min((r0 + rr) / b, nb - 1) - blk0;
+                        const float re = bsc[q];
+                        const int gi = r0 + rr + row_in_block;
+                        const float inv_mine = gi < N ? __ldcg(A.inv_norm + (int64_t)u * N + gi) : 0.f;
+                        float c[4] = {0.f, 0.f, 0.f, 0.f};
+                        const unsigned char* row_lo = tileB + (size_t)(rr + gq) * G::kRowBytes;
+                        const unsigned char* row_hi = row_lo + 8 * G::kRowBytes;
+                        const __nv_bfloat16* rq = rhs + ((size_t)q * 8 + gq) * D;
 #pragma unroll
-        for (int o = 0; o < kSeg; ++o) {
-            F2 kn[NP];
-            G::load_row(tile + (size_t)(grp * kSeg + o) * G::kRowBytes, l, kn);
-            F2 ds = pack2(0.f, 0.f), de = pack2(0.f, 0.f);
+                        for (int j = 0; j < kCh; ++j) {
+                            const uint4 x = *reinterpret_cast<const uint4*>(row_lo + (t + 4 * j) * 16);
+                            const uint4 y = *reinterpret_cast<const uint4*>(row_hi + (t + 4 * j) * 16);
+                            const uint4 w = *reinterpret_cast<const uint4*>(rq + (t + 4 * j) * 8);
+                            const uint32_t a_first[4] = {x.x, y.x, x.y, y.y};
+                            const uint32_t a_second[4] = {x.z, y.z, x.w, y.w};
+                            mma_bf16_16816(c, a_first, w.x, w.y);
+                            mma_bf16_16816(c, a_second, w.z, w.w);
+                        }
+                        // columns 0,1 (t=0) and 2 (t=1, c[0]) belong to mu_s; 3 (t=1, c[1]) and 4,5 (t=2) to mu_e
+                        float xs_lo = t == 0 ? c[0] + c[1] : (t == 1 ? c[0] : 0.f);
+                        float xe_lo = t == 1 ? c[1] : (t == 2 ? c[0] + c[1] : 0.f);
+                        float xs_hi = t == 0 ? c[2] + c[3] : (t == 1 ? c[2] : 0.f);
+                        float xe_hi = t == 1 ? c[3] : (t == 2 ? c[2] + c[3] : 0.f);
 #pragma unroll
-            for (int p = 0; p < NP; ++p) {
-                ds = fma2(kn[p], ms[p], ds);
-                de = fma2(kn[p], me[p], de);
+                        for (int o = 1; o <= 2; o <<= 1) {
+                            xs_lo += __shfl_xor_sync(0xffffffffu, xs_lo, o);
+                            xe_lo += __shfl_xor_sync(0xffffffffu, xe_lo, o);
+                            xs_hi += __shfl_xor_sync(0xffffffffu, xs_hi, o);
+                            xe_hi += __shfl_xor_sync(0xffffffffu, xe_hi, o);
+                        }
+                        // each lane finishes one of its quad's four results: t=0: a_s(row g), t=1: a_e(row g),
+                        // t=2: a_s(row g+8), t=3: a_e(row g+8)
+                        const float dot = t == 0 ? xs_lo : (t == 1 ? xe_lo : (t == 2 ? xs_hi : xe_hi));
+                        const float a = -(dot * inv_mine) * ((t & 1) ? re : rs) + 0.f;
+                        if (gi < N) {
+                            A.a_raw[((int64_t)u * 3 + (t & 1)) * N + gi] = a;
+                            if (t & 1) {
+                                lo_e = fminf(lo_e, a);
+                                hi_e = fmaxf(hi_e, a);
+                            } else {
+                                lo_s = fminf(lo_s, a);
+                                hi_s = fmaxf(hi_s, a);
+                            }
+                        }
+                    }
+                }
+            } else {
+                // packed FMAs: an L-lane group walks 8 rows; whole warps run every iteration (groups past
+                // the end compute on stale rows and write nothing)
+                const int grp = bt / L, l = bt % L;
+                F2 ms[NP];
+                G::load_vec(A.mu_s + (int64_t)u * D, l, ms);
+                for (int seg0 = 0; seg0 * kSeg < rows; seg0 += kBThreads / L) {
+                    const int seg = seg0 + grp;
+                    const int gi0 = r0 + seg * kSeg;
+                    const int blk = min(gi0 / b, nb - 1);
+                    F2 me[NP];
+                    G::load_vec(A.block_sums + ((int64_t)u * nb + blk) * D, l, me);
+                    const float re = __ldcg(A.inv_e + (int64_t)u * nb + blk);
+                    const int o_mine = L == 16 ? (l >> 1) : l;
+                    const float inv_mine = gi0 + o_mine < N ? __ldcg(A.inv_norm + (int64_t)u * N + gi0 + o_mine) : 0.f;
+                    float part[16];
+                    const int seg_c = min(seg, B::kRows / kSeg - 1);   // stay inside the buffer
+#pragma unroll
+                    for (int o = 0; o < kSeg; ++o) {
+                        F2 kn[NP];
+                        G::load_row(tileB + (size_t)(seg_c * kSeg + o) * G::kRowBytes, l, kn);
+                        F2 ds = pack2(0.f, 0.f), de = pack2(0.f, 0.f);
+#pragma unroll
+                        for (int p = 0; p < NP; ++p) {
+                            ds = fma2(kn[p], ms[p], ds);
+                            de = fma2(kn[p], me[p], de);
+                        }
+                        part[2 * o] = hsum2(ds);
+                        part[2 * o + 1] = hsum2(de);
+                    }
+                    treduce<16, L>(part, l);
+                    const bool live = seg * kSeg < rows;
+                    if (L == 16) {
+                        const int o = l >> 1;
+                        const float a = -(part[0] * inv_mine) * ((l & 1) ? re : rs) + 0.f;
+                        if (live && gi0 + o < N) {
+                            A.a_raw[((int64_t)u * 3 + (l & 1)) * N + gi0 + o] = a;
+                            if (l & 1) {
+                                lo_e = fminf(lo_e, a);
+                                hi_e = fmaxf(hi_e, a);
+                            } else {
+                                lo_s = fminf(lo_s, a);
+                                hi_s = fmaxf(hi_s, a);
+                            }
+                        }
+                    } else {
+                        const float a_s = -(part[0] * inv_mine) * rs + 0.f;
+                        const float a_e = -(part[1] * inv_mine) * re + 0.f;
+                        if (live && gi0 + l < N) {
+                            A.a_raw[((int64_t)u * 3 + 0) * N + gi0 + l] = a_s;
+                            A.a_raw[((int64_t)u * 3 + 1) * N + gi0 + l] = a_e;
+                            lo_s = fminf(lo_s, a_s);
+                            hi_s = fmaxf(hi_s, a_s);
+                            lo_e = fminf(lo_e, a_e);
+                            hi_e = fmaxf(hi_e, a_e);
+                        }
+                    }
+                }
             }
-            part[2 * o] = hsum2(ds);
-            part[2 * o + 1] = hsum2(de);
-        }
-        treduce<16, L>(part, l);
-        float lo_s = INFINITY, hi_s = -INFINITY, lo_e = INFINITY, hi_e = -INFINITY;
-        if (L == 16) {
-            // lane l owns value l: token l/2, quantity l%2 (0: stable, 1: episodic)
-            const int o = l >> 1;
-            const float a = -(part[0] * inv_mine) * ((l & 1) ? re : rs) + 0.f;
-            if (gi0 + o < N) {
-                A.a_raw[((int64_t)u * 3 + (l & 1)) * N + gi0 + o] = a;
-                if (l & 1) lo_e = hi_e = a;
-                else lo_s = hi_s = a;
-            }
-        } else {
-            const float a_s = -(part[0] * inv_mine) * rs + 0.f;
-            const float a_e = -(part[1] * inv_mine) * re + 0.f;
-            if (gi0 + l < N) {
-                A.a_raw[((int64_t)u * 3 + 0) * N + gi0 + l] = a_s;
-                A.a_raw[((int64_t)u * 3 + 1) * N + gi0 + l] = a_e;
-                lo_s = hi_s = a_s;
-                lo_e = hi_e = a_e;
-            }
+            bar_sync(kBarB, kBThreads);   // the buffer and the right-hand sides may be overwritten
         }
         lo_s = warp_min(lo_s);
         hi_s = warp_max(hi_s);
         lo_e = warp_min(lo_e);
         hi_e = warp_max(hi_e);
-        if ((tid & 31) == 0) {
+        if (lane == 0) {
             if (lo_s <= hi_s) {
-                atomicMin(&mmk[0], ord_key(lo_s));
-                atomicMax(&mmk[1], ord_key(hi_s));
+                atomicMin(&A.mm[(int64_t)u * 6 + 0], ord_key(lo_s));
+                atomicMax(&A.mm[(int64_t)u * 6 + 1], ord_key(hi_s));
             }
             if (lo_e <= hi_e) {
-                atomicMin(&mmk[2], ord_key(lo_e));
-                atomicMax(&mmk[3], ord_key(hi_e));
+                atomicMin(&A.mm[(int64_t)u * 6 + 2], ord_key(lo_e));
+                atomicMax(&A.mm[(int64_t)u * 6 + 3], ord_key(hi_e));
             }
-        }
-    }
-    prefetch_data<T, D>(A, pre);
-}
-
-// ---------------------------------------------------------------------------- pass B on tensor cores
-// For bf16 keys the two dots of every key against the fixed vectors mu_s and mu_e are a skinny matrix
-// product [16 keys x d] x [d x 8]: the fp32 anchors are split three ways into bf16 (hi + mid + lo
-// carries all 24 mantissa bits), products of bf16 numbers are exact in fp32 and the accumulation is
-// fp32, so the result is an fp32 dot product up to summation order.  Columns of the right-hand side:
-// 0..2 = mu_s hi/mid/lo, 3..5 = mu_e hi/mid/lo, 6..7 = 0.  The contraction index may be visited in any
-// order, so lane (g, t) of a warp takes the 16-byte chunks t, t+4, t+8, ... of rows g and g+8 straight
-// from the staged tile (no transposition, no conversion) and the right-hand side uses the same order.
-// Requires block % 16 == 0 and at most four episodic blocks per tile.  `pp`/`invs` staging as in pass_b;
-// behind the staged floats `pp` also holds the split right-hand sides [nblk][8][D] in bf16.
-template <int D>
-__device__ __forceinline__ void pass_b_mma(const FusedArgs& A, int u, int tile_idx, const unsigned char* tile, float* pp,
-                                           float* invs, uint32_t* mmk, uint64_t* full, uint32_t parity,
-                                           int* abort_flag, const volatile Item* next, int next_seq,
-                                           Prefetched& pre) {
-    using G = Geo<__nv_bfloat16, D>;
-    constexpr int kSteps = D / 16;        // k-steps of the MMA
-    constexpr int kCh = D / 32;           // 16-byte chunks per lane and row
-    const int N = A.K.N, b = A.sp.block, nb = A.sp.nblocks;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-    const int i0 = tile_idx * G::kTile;
-    const int blk0 = i0 / b;
-    const int nblk = min(nb - blk0, G::kTile / b);
-    __nv_bfloat16* rhs = reinterpret_cast<__nv_bfloat16*>(pp + 5 * D);   // [nblk][8][D]
-
-    if (tid < D) {
-        float mu, me[4], aux = 0.f;
-        if (pre.have && pre.unit == u && pre.tile == tile_idx) {
-            mu = pre.mu;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) me[q] = pre.me[q];
-            aux = pre.aux;
-        } else {
-            const int* ready = A.ctrl + kCtrlHeader + A.units + u;
-            bool ok = ld_acquire(ready) != 0;
-            if (!ok && *reinterpret_cast<volatile int*>(abort_flag) == 0) {
-                const unsigned long long t0 = now_ns();
-                for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
-                    if (ld_acquire(ready) != 0) {
-                        ok = true;
-                        break;
-                    }
-                    __nanosleep(64);
-                    if ((spin & 63u) == 63u && now_ns() - t0 > kWaitLimitNs) break;
-                }
-            }
-            if (!ok) {
-                set_status(A.status, NKV_ERR_TIMEOUT, 505);
-                *abort_flag = 1;
-            }
-            mu = __ldcg(A.mu_s + (int64_t)u * D + tid);
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-                me[q] = q < nblk ? __ldcg(A.block_sums + ((int64_t)u * nb + blk0 + q) * D + tid) : 0.f;
-            if (tid == 0) aux = __ldcg(A.inv_s + u);
-            else if (tid <= nblk) aux = __ldcg(A.inv_e + (int64_t)u * nb + blk0 + tid - 1);
-        }
-        if (tid <= nblk) invs[tid] = aux;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            if (q < nblk) {
-                __nv_bfloat16* r = rhs + (size_t)q * 8 * D + tid;
-                split3_bf16(mu, r, D);
-                split3_bf16(me[q], r + 3 * D, D);
-                r[6 * D] = __float2bfloat16_rn(0.f);
-                r[7 * D] = __float2bfloat16_rn(0.f);
-            }
-        }
-    }
-    bar_sync(kBarCompute, G::kThreads);
-    prefetch_flag<__nv_bfloat16, D>(A, next, next_seq, pre);
-
-    const int rows = min(N, i0 + G::kTile) - i0;
-    const float rs = invs[0];
-    // each lane finishes one of the four results of its quad: t=0: a_s(row g), t=1: a_e(row g),
-    // t=2: a_s(row g+8), t=3: a_e(row g+8); its key's reciprocal norm is fetched before the copy is awaited
-    constexpr int kWarps = G::kThreads / 32;
-    constexpr int kIters = (G::kTile / 16 + kWarps - 1) / kWarps;
-    const int row_in_block = g + ((t & 2) ? 8 : 0);
-    float inv_pre[kIters];
-#pragma unroll
-    for (int it = 0; it < kIters; ++it) {
-        const int gi = i0 + (warp + it * kWarps) * 16 + row_in_block;
-        inv_pre[it] = (warp + it * kWarps) * 16 < rows && gi < N ? __ldcg(A.inv_norm + (int64_t)u * N + gi) : 0.f;
-    }
-    if (!mbar_wait(full, parity, abort_flag)) {
-        set_status(A.status, NKV_ERR_TIMEOUT, 503);
-        *abort_flag = 1;
-    }
-    float lo_s = INFINITY, hi_s = -INFINITY, lo_e = INFINITY, hi_e = -INFINITY;
-#pragma unroll
-    for (int it = 0; it < kIters; ++it) {
-        const int rb = warp + it * kWarps;
-        if (rb * 16 >= rows) break;
-        const int r0 = rb * 16;
-        const int q = min((i0 + r0) / b, nb - 1) - blk0;
-        const float re = invs[1 + q];
-        const int my_row = r0 + row_in_block;
-        const float inv_mine = inv_pre[it];
-        float c[4] = {0.f, 0.f, 0.f, 0.f};
-        const unsigned char* row_lo = tile + (size_t)(r0 + g) * G::kRowBytes;
-        const unsigned char* row_hi = row_lo + 8 * G::kRowBytes;
-        const __nv_bfloat16* rq = rhs + ((size_t)q * 8 + g) * D;
-#pragma unroll
-        for (int j = 0; j < kCh; ++j) {
-            const uint4 x = *reinterpret_cast<const uint4*>(row_lo + (t + 4 * j) * 16);
-            const uint4 y = *reinterpret_cast<const uint4*>(row_hi + (t + 4 * j) * 16);
-            const uint4 w = *reinterpret_cast<const uint4*>(rq + (t + 4 * j) * 8);
-            const uint32_t a_first[4] = {x.x, y.x, x.y, y.y};
-            const uint32_t a_second[4] = {x.z, y.z, x.w, y.w};
-            mma_bf16_16816(c, a_first, w.x, w.y);
-            mma_bf16_16816(c, a_second, w.z, w.w);
-        }
-        static_assert(kSteps == 2 * kCh, "two k-steps per chunk");
-        // columns: 0,1 (t=0) and 2 (t=1, c[0]) belong to mu_s; 3 (t=1, c[1]) and 4,5 (t=2) to mu_e
-        float xs_lo = t == 0 ? c[0] + c[1] : (t == 1 ? c[0] : 0.f);
-        float xe_lo = t == 1 ? c[1] : (t == 2 ? c[0] + c[1] : 0.f);
-        float xs_hi = t == 0 ? c[2] + c[3] : (t == 1 ? c[2] : 0.f);
-        float xe_hi = t == 1 ? c[3] : (t == 2 ? c[2] + c[3] : 0.f);
-#pragma unroll
-        for (int o = 1; o <= 2; o <<= 1) {
-            xs_lo += __shfl_xor_sync(0xffffffffu, xs_lo, o);
-            xe_lo += __shfl_xor_sync(0xffffffffu, xe_lo, o);
-            xs_hi += __shfl_xor_sync(0xffffffffu, xs_hi, o);
-            xe_hi += __shfl_xor_sync(0xffffffffu, xe_hi, o);
-        }
-        const float dot = t == 0 ? xs_lo : (t == 1 ? xe_lo : (t == 2 ? xs_hi : xe_hi));
-        const float a = -(dot * inv_mine) * ((t & 1) ? re : rs) + 0.f;
-        if (i0 + my_row < N) {
-            A.a_raw[((int64_t)u * 3 + (t & 1)) * N + i0 + my_row] = a;
-            if (t & 1) {
-                lo_e = fminf(lo_e, a);
-                hi_e = fmaxf(hi_e, a);
-            } else {
-                lo_s = fminf(lo_s, a);
-                hi_s = fmaxf(hi_s, a);
-            }
-        }
-    }
-    prefetch_data<__nv_bfloat16, D>(A, pre);
-    lo_s = warp_min(lo_s);
-    hi_s = warp_max(hi_s);
-    lo_e = warp_min(lo_e);
-    hi_e = warp_max(hi_e);
-    if (lane == 0) {
-        if (lo_s <= hi_s) {
-            atomicMin(&mmk[0], ord_key(lo_s));
-            atomicMax(&mmk[1], ord_key(hi_s));
-        }
-        if (lo_e <= hi_e) {
-            atomicMin(&mmk[2], ord_key(lo_e));
-            atomicMax(&mmk[3], ord_key(hi_e));
         }
     }
 }
@@ -843,290 +755,7 @@ __device__ __forceinline__ void finalize_head(const FusedArgs& A, int u, float* 
     if (tid == 0) st_release(A.ctrl + kCtrlHeader + A.units + u, 1);
 }
 
-// ---------------------------------------------------------------------------- the persistent kernel
-// Small shared-memory state after the big arrays (byte offsets inside `small`):
-//   0  item[2]      descriptors of the items in the two tile buffers
-//   32 mmk[2][6]    per-item ordered min/max keys (double buffered like the tiles)
-//   80 fin[2]       head whose anchors this CTA owes after item k (or -1), written by the control warp
-//   88 abort_flag   a bounded wait ran out somewhere in this CTA
-//   92 book_seq     index of the last item whose bookkeeping is complete
-//   96 full[2]      mbarriers of the two tile buffers
-template <typename T, int D>
-struct Ctl {
-    using G = Geo<T, D>;
-    const FusedArgs& A;
-    unsigned char* tiles;
-    Item* item;
-    uint64_t* full;
-    int* abort_flag;
-    int tiles_per_unit;
-    long long per_step, total;
-    uint64_t pol_a, pol_b;
-
-    // ticket number -> item; kind 2 with pad 1 means "this ticket names no item, take another"
-    __device__ __forceinline__ Item decode(unsigned long long t) const {
-        Item it;
-        it.kind = 2;
-        it.unit = it.tile = it.pad = 0;
-        if ((long long)t >= total) return it;
-        const long long step = (long long)(t / (unsigned long long)per_step);
-        const int j = (int)(t - (unsigned long long)step * (unsigned long long)per_step);
-        const int strips = (int)(per_step / 2);
-        if (j < strips) {
-            if (step < A.units) {
-                it.kind = 0;
-                it.unit = (int)step;
-                it.tile = j * A.strip;   // first tile of the strip
-                return it;
-            }
-        } else if (step >= A.lag) {
-            it.kind = 1;
-            it.unit = (int)(step - A.lag);
-            it.tile = (j - strips) * A.strip;
-            return it;
-        }
-        it.pad = 1;
-        return it;
-    }
-    __device__ __forceinline__ unsigned long long take_ticket() {
-        return atomicAdd(reinterpret_cast<unsigned long long*>(A.ctrl), 1ULL);
-    }
-    // the item of ticket t, or of the next ticket that names one (steps at both ends of the order
-    // have no pass-A or no pass-B head)
-    __device__ __forceinline__ Item item_from(unsigned long long t) {
-        Item it = decode(t);
-        while (it.kind == 2 && it.pad == 1 && *reinterpret_cast<volatile int*>(abort_flag) == 0) it = decode(take_ticket());
-        it.pad = 0;
-        return it;
-    }
-    __device__ __forceinline__ Item fetch() { return item_from(take_ticket()); }
-    // tiles that follow `it` in its strip
-    __device__ __forceinline__ int rest_of_strip(const Item& it) const {
-        return it.kind == 2 ? 0 : min(A.strip, tiles_per_unit - it.tile) - 1;
-    }
-    // publish `it` as item number `seq` in `slot` and start its copy
-    __device__ __forceinline__ void issue(int slot, Item it, int seq) {
-        volatile Item* d = item + slot;
-        d->pad = -1;
-        __threadfence_block();
-        d->kind = it.kind;
-        d->unit = it.unit;
-        d->tile = it.tile;
-        __threadfence_block();
-        d->pad = seq;   // readers that find `seq` here may trust the other fields
-        if (it.kind == 2) return;
-        const int N = A.K.N;
-        const int g = it.unit / A.K.H, h = it.unit % A.K.H;
-        const unsigned char* base = reinterpret_cast<const unsigned char*>(A.K.ptr) +
-                                    ((int64_t)g * A.K.stride_g + (int64_t)h * A.K.stride_h) * (int64_t)sizeof(T);
-        const int i0 = it.tile * G::kTile;
-        unsigned char* dst = tiles + (size_t)slot * G::kTileBytes;
-        int r0, r1;
-        if (it.kind == 0) {   // pass A stages the 64 rows in front of the tile as well
-            r0 = max(0, i0 - kHalo);
-            r1 = min(N, i0 + G::kTile);
-            dst += (size_t)(r0 - (i0 - kHalo)) * G::kRowBytes;
-        } else {
-            r0 = i0;
-            r1 = min(N, i0 + G::kTile);
-        }
-        const uint32_t bytes = (uint32_t)(r1 - r0) * G::kRowBytes;
-        const unsigned char* src = base + (int64_t)r0 * G::kRowBytes;
-        fence_async_smem();
-        mbar_expect_tx(&full[slot], bytes);
-        for (uint32_t off = 0; off < bytes; off += 32768u)
-            bulk_load(dst + off, src + off, min(32768u, bytes - off), &full[slot], it.kind == 0 ? pol_a : pol_b);
-    }
-};
-
-template <typename T, int D>
-__global__ void __launch_bounds__(Geo<T, D>::kThreads + 32, 1) fused_scan_kernel(FusedArgs A) {
-    using G = Geo<T, D>;
-    extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char* tiles = smem;
-    float* pp = reinterpret_cast<float*>(smem + 2 * G::kTileBytes);          // [kSegs][D]
-    float* invs = pp + G::kSegs * D;                                         // [kRows]
-    unsigned char* small = reinterpret_cast<unsigned char*>(invs + G::kRows);
-    Item* item = reinterpret_cast<Item*>(small);
-    uint32_t* mmk = reinterpret_cast<uint32_t*>(small + 32);
-    int* fin = reinterpret_cast<int*>(small + 80);
-    int* abort_flag = reinterpret_cast<int*>(small + 88);
-    int* book_seq = reinterpret_cast<int*>(small + 92);
-    uint64_t* full = reinterpret_cast<uint64_t*>(small + 96);
-
-    const int N = A.K.N;
-    const int tiles_per_unit = (N + G::kTile - 1) / G::kTile;
-    const int tid = threadIdx.x;
-    constexpr int kAll = G::kThreads + 32;
-
-    if (tid == 0) {
-        mbar_init(&full[0], 1);
-        mbar_init(&full[1], 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        for (int i = 0; i < 12; ++i) mmk[i] = (i & 1) ? 0u : 0xffffffffu;
-        fin[0] = fin[1] = -1;
-        *abort_flag = 0;
-        *book_seq = -1;
-    }
-    __syncthreads();
-
-    if (tid >= G::kThreads) {
-        // ------------------------------------------------------------------ control warp
-        // All 32 lanes run the loop together (the per-item barrier is warp-aligned); lane 0 works.
-        const int lane = tid - G::kThreads;
-        const long long strips = (tiles_per_unit + A.strip - 1) / A.strip;
-        Ctl<T, D> C{A, tiles, item, full, abort_flag, tiles_per_unit, 2LL * strips,
-                    ((long long)A.units + A.lag) * 2LL * strips,
-                    A.hints ? l2_policy_keep() : l2_policy_normal(), A.hints ? l2_policy_stream() : l2_policy_normal()};
-        Item nxt;   // the ticket after the two in flight, fetched ahead of time (lane 0)
-        nxt.kind = 2;
-        nxt.unit = nxt.tile = nxt.pad = 0;
-        int left = 0;   // tiles that follow `nxt` in its strip
-        auto advance = [&]() {   // nxt <- the item after nxt (blocking ticket fetch when the strip is used up)
-            if (left > 0) {
-                ++nxt.tile;
-                --left;
-            } else {
-                nxt = C.fetch();
-                left = C.rest_of_strip(nxt);
-            }
-        };
-        if (lane == 0) {
-            advance();
-            C.issue(0, nxt, 0);
-            advance();
-            C.issue(1, nxt, 1);
-            advance();
-        }
-        __syncwarp();
-        bar_sync(kBarEnd, kAll);   // start: both descriptors are visible
-        bool prev_done = false;
-        for (int k = 0;; ++k) {
-            const Item cur = item[k & 1];
-            bar_sync(kBarEnd, kAll);   // the compute threads have finished item k
-            const bool done = cur.kind == 2;
-            if (done && prev_done) break;
-            prev_done = done;
-            if (lane == 0) {
-                C.issue(k & 1, nxt, k + 2);   // item k + 2 goes into the buffer that item k has released
-                // Two global atomics per item, both in flight at once: the next ticket (needed at the
-                // next item barrier) and the tile counter of the head (needed now).  No fence here: the
-                // compute threads fence their block sums before the item barrier.
-                const bool in_strip = left > 0;
-                const bool more = !in_strip && nxt.kind != 2 && *reinterpret_cast<volatile int*>(abort_flag) == 0;
-                unsigned long long t_raw = ~0ULL;
-                if (more) t_raw = C.take_ticket();
-                int fin_unit = -1;
-                if (cur.kind == 0) {
-                    const int prev = atomicAdd(A.ctrl + kCtrlHeader + cur.unit, 1);
-                    if (prev == tiles_per_unit - 1) fin_unit = cur.unit;
-                }
-                *reinterpret_cast<volatile int*>(&fin[k & 1]) = fin_unit;
-                __threadfence_block();
-                *reinterpret_cast<volatile int*>(book_seq) = k;
-                if (!done) {   // publish the tile's min/max and re-arm the slots
-                    uint32_t* m = mmk + (k & 1) * 6;
-                    const int q0 = cur.kind == 0 ? 4 : 0, q1 = cur.kind == 0 ? 6 : 4;
-                    for (int q = q0; q < q1; ++q) {
-                        const uint32_t v = m[q];
-                        if (q & 1) {
-                            if (v != 0u) atomicMax(&A.mm[(int64_t)cur.unit * 6 + q], v);
-                            m[q] = 0u;
-                        } else {
-                            if (v != 0xffffffffu) atomicMin(&A.mm[(int64_t)cur.unit * 6 + q], v);
-                            m[q] = 0xffffffffu;
-                        }
-                    }
-                }
-                if (in_strip) {
-                    ++nxt.tile;
-                    --left;
-                } else if (more) {
-                    nxt = C.item_from(t_raw);
-                    left = C.rest_of_strip(nxt);
-                } else {
-                    nxt.kind = 2;
-                }
-            }
-            __syncwarp();
-        }
-        return;
-    }
-
-    // ---------------------------------------------------------------------- compute threads
-    bar_sync(kBarEnd, kAll);   // start
-    bool prev_done = false;
-    int prev_kind = 2;
-    Prefetched pre;
-    pre.have = 0;
-    for (int k = 0;; ++k) {
-        const Item cur = item[k & 1];
-        const int buf = k & 1;
-        const volatile Item* next = item + ((k + 1) & 1);
-        const uint32_t parity = (uint32_t)((k >> 1) & 1);
-        unsigned char* tile = tiles + (size_t)buf * G::kTileBytes;
-        // A pass-B item may have to wait for anchors.  This CTA must not wait while it still owes
-        // some head its anchors, so first learn whether the previous pass-A item completed a head.
-        bool owed_paid = false;
-        if (cur.kind == 1 && prev_kind == 0) {
-            if (tid == 0) {
-                const unsigned long long t0 = now_ns();
-                for (uint32_t spin = 0; *reinterpret_cast<volatile int*>(book_seq) < k - 1; ++spin) {
-                    if ((spin & 63u) == 63u && now_ns() - t0 > kWaitLimitNs) {
-                        set_status(A.status, NKV_ERR_TIMEOUT, 504);
-                        *abort_flag = 1;
-                        break;
-                    }
-                }
-            }
-            bar_sync(kBarCompute, G::kThreads);
-            const int f = *reinterpret_cast<volatile int*>(&fin[(k - 1) & 1]);
-            if (f >= 0 && *reinterpret_cast<volatile int*>(book_seq) >= k - 1) {
-                finalize_head<T, D>(A, f, pp, invs);
-                owed_paid = true;
-            }
-        }
-        prev_kind = cur.kind;
-        if (cur.kind == 0) pass_a<T, D>(A, cur.unit, cur.tile, tile, pp, invs, mmk + buf * 6, &full[buf], parity, abort_flag,
-                                       next, k + 1, pre);
-        else if (cur.kind == 1) {
-            bool on_tensor_cores = false;
-            if constexpr (sizeof(T) == 2) {
-                if (A.sp.block % 16 == 0 && G::kTile / A.sp.block <= 4) {
-                    on_tensor_cores = true;
-                    pass_b_mma<D>(A, cur.unit, cur.tile, tile, pp, invs, mmk + buf * 6, &full[buf], parity, abort_flag,
-                                  next, k + 1, pre);
-                }
-            }
-            if (!on_tensor_cores)
-                pass_b<T, D>(A, cur.unit, cur.tile, tile, pp, invs, mmk + buf * 6, &full[buf], parity, abort_flag,
-                             next, k + 1, pre);
-        }
-        bar_sync(kBarEnd, kAll);   // end of item k
-        const bool done = cur.kind == 2;
-        if (done && prev_done) break;
-        prev_done = done;
-        if (k >= 1 && !owed_paid) {
-            const int f = fin[(k - 1) & 1];
-            if (f >= 0) finalize_head<T, D>(A, f, pp, invs);
-        }
-    }
-}
-
-__global__ void fused_init_kernel(int units, uint32_t* mm, int* ctrl) {
-    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < (long long)units * 6) mm[i] = (i & 1) ? 0u : 0xffffffffu;
-    if (i < (long long)kCtrlHeader + 2LL * units) ctrl[i] = 0;
-}
-
-template <typename T, int D>
-cudaError_t launch_one(const FusedArgs& A, int sm_count, cudaStream_t stream) {
-    using G = Geo<T, D>;
-    const long long tiles = (long long)A.units * ((A.K.N + G::kTile - 1) / G::kTile);
-    const unsigned grid = (unsigned)(2 * tiles < sm_count ? 2 * tiles : sm_count);
-    fused_scan_kernel<T, D><<<grid, G::kThreads + 32, G::kSmem, stream>>>(A);
-    return cudaGetLastError();
-}
+//@@KERNEL@@
 
 }  // namespace
 
