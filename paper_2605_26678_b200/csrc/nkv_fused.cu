@@ -7,19 +7,18 @@
 //                              CTA that finishes the head's last pass-A tile
 //   pass B (needs the anchors) a_s(i), a_e(i) and their per-head min/max
 //
-// Work items are handed out in ticket order: for every step s, the tiles of A(head s), then the tiles
-// of B(head s - lag).  A pass-B item waits (bounded) for its head's anchors; every pass-A item it
-// depends on carries an earlier ticket and never waits, and a CTA pays the anchors it owes before it
-// waits itself, so the order cannot deadlock.
+// Pass-A tiles are handed out in ticket order (strips of consecutive tiles of one head) to the pass-A
+// threads of the persistent CTAs; a control warp per CTA takes the tickets, issues the bulk copies into
+// two tile buffers (one is always in flight) and does the per-item bookkeeping, so the compute threads
+// never wait for a global atomic.  Pass B runs beside it on its own warp group with its own ticket
+// counter and buffer: it waits (bounded) for a head's anchors and therefore trails pass A by as little
+// as the anchors allow, which is what keeps its reads in L2.  Pass A never waits for pass B, so the two
+// cannot deadlock.
 //
-// A row of d elements is split over 8 lanes (16-byte chunks l, l+8, ...), so a quarter warp reads 128
-// contiguous bytes of shared memory.  Each 8-lane group owns one 8-row segment; per-token partial
-// sums are combined with a transposed shuffle reduction that leaves token l with lane l, which then
-// writes its result straight to global memory (32 contiguous bytes per group).  The sliding-window
-// sum is a running sum over the 8 tokens of a group, seeded from exact segment sums, so no long
-// prefix is ever differenced.  Key tiles are staged with bulk asynchronous copies, double buffered,
-// issued by a control warp that also does the per-item bookkeeping (tickets, tile counters, min/max
-// publication) so that the compute threads never wait for a global atomic.
+// Pass A: a row of d elements is split over 8 or 16 lanes (16-byte chunks), each lane group owns one
+// 8-row segment; per-token partial sums are combined with a transposed shuffle reduction.  The
+// sliding-window sum is a running sum over the 8 tokens of a group, seeded from exact segment sums, so
+// no long prefix is ever differenced.
 #include "nkv_common.cuh"
 
 namespace nkv {
@@ -30,8 +29,8 @@ constexpr int kHalo = kMaxWindow;
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr unsigned long long kWaitLimitNs = 2000000000ULL;   // every device-side wait gives up after 2 s
 
-// control words (ints) in the workspace: [0..1] 64-bit ticket counter, [8 + u] tiles of head u
-// finished by pass A, [8 + units + u] anchors of head u published
+// control words (ints) in the workspace: [0..1] 64-bit ticket counter of pass A, [2..3] of pass B,
+// [8 + u] tiles of head u finished by pass A, [8 + units + u] anchors of head u published
 constexpr int kCtrlHeader = 8;
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -450,7 +449,7 @@ struct BGeo {
     using G = Geo<T, D>;
     static constexpr int kBytes = G::kRowBytes >= 512 ? 16384 : 32768;   // private buffer of the group
     static constexpr int kRows = kBytes / G::kRowBytes;                  // rows per sub-tile
-    static constexpr int kAnchorBytes = 4 * 8 * D * 2;                   // split right-hand sides [4][8][D] bf16
+    static constexpr int kAnchorBytes = sizeof(T) == 2 ? 4 * 8 * D * 2 : 0;   // split right-hand sides [4][8][D] bf16
 };
 
 template <typename T, int D>
@@ -465,7 +464,8 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
     const long long total = (long long)A.units * tiles_per_unit;
     unsigned long long* ticket = reinterpret_cast<unsigned long long*>(A.ctrl + 2);
     const uint64_t policy = A.hints ? l2_policy_stream() : l2_policy_normal();
-    const bool mma_path = sizeof(T) == 2 && b % 16 == 0 && B::kRows <= 4 * b;
+    // a sub-tile overlaps at most ceil(kRows / b) + 1 blocks; the staged right-hand sides hold four
+    const bool mma_path = sizeof(T) == 2 && b % 16 == 0 && (B::kRows + b - 1) / b + 1 <= 4;
     uint32_t copies = 0;   // copies awaited so far (mbarrier parity)
 
     for (;;) {
@@ -523,7 +523,7 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
             if (mma_path) {
                 if constexpr (sizeof(T) == 2) {
                     // split right-hand sides of the sub-tile's blocks, one anchor column per thread
-                    const int nblk = min(nb - blk0, max(1, B::kRows / b));
+                    const int nblk = min(nb - 1, (r0 + rows - 1) / b) - blk0 + 1;
                     if (bt < D) {
                         const float mu = __ldcg(A.mu_s + (int64_t)u * D + bt);
                         for (int q = 0; q < nblk; ++q) {
@@ -755,7 +755,222 @@ __device__ __forceinline__ void finalize_head(const FusedArgs& A, int u, float* 
     if (tid == 0) st_release(A.ctrl + kCtrlHeader + A.units + u, 1);
 }
 
-//@@KERNEL@@
+// ---------------------------------------------------------------------------- the persistent kernel
+// Thread roles: [0, kThreads) pass A; one control warp (tickets, copies and bookkeeping of pass A);
+// kBThreads threads of pass B.  Small shared-memory state after the big arrays (byte offsets in `small`):
+//   0  item[2]      descriptors of the pass-A items in the two tile buffers
+//   32 mmk[2][6]    per-item ordered min/max keys (double buffered like the tiles; slots 4, 5 are used)
+//   80 fin[2]       head whose anchors this CTA owes after item k (or -1), written by the control warp
+//   88 abort_flag   a bounded wait ran out somewhere in this CTA
+//   96 full[2]      mbarriers of the two pass-A tile buffers
+//   112 mbarB       mbarrier of the pass-B buffer
+//   120 bslot[2]    head and tile of the pass-B group's current ticket
+//   128 bsc[8]      1/||mu_e|| of the blocks of the current pass-B sub-tile
+template <typename T, int D>
+struct Ctl {
+    using G = Geo<T, D>;
+    const FusedArgs& A;
+    unsigned char* tiles;
+    Item* item;
+    uint64_t* full;
+    int* abort_flag;
+    int tiles_per_unit, strips;
+    long long total;   // strip tickets of pass A
+    uint64_t policy;
+
+    __device__ __forceinline__ unsigned long long take_ticket() {
+        return atomicAdd(reinterpret_cast<unsigned long long*>(A.ctrl), 1ULL);
+    }
+    // ticket number -> first tile of its strip (kind 2 when the tickets are used up)
+    __device__ __forceinline__ Item decode(unsigned long long t) const {
+        Item it;
+        it.kind = 2;
+        it.unit = it.tile = it.pad = 0;
+        if ((long long)t >= total || *reinterpret_cast<volatile int*>(abort_flag) != 0) return it;
+        it.kind = 0;
+        it.unit = (int)(t / (unsigned long long)strips);
+        it.tile = (int)(t - (unsigned long long)it.unit * strips) * A.strip;
+        return it;
+    }
+    // tiles that follow `it` in its strip
+    __device__ __forceinline__ int rest_of_strip(const Item& it) const {
+        return it.kind == 2 ? 0 : min(A.strip, tiles_per_unit - it.tile) - 1;
+    }
+    // publish `it` in `slot` and start its copy (tile rows plus the 64 rows in front of them)
+    __device__ __forceinline__ void issue(int slot, Item it) {
+        item[slot] = it;
+        if (it.kind == 2) return;
+        const int N = A.K.N;
+        const int g = it.unit / A.K.H, h = it.unit % A.K.H;
+        const unsigned char* base = reinterpret_cast<const unsigned char*>(A.K.ptr) +
+                                    ((int64_t)g * A.K.stride_g + (int64_t)h * A.K.stride_h) * (int64_t)sizeof(T);
+        const int i0 = it.tile * G::kTile;
+        const int r0 = max(0, i0 - kHalo), r1 = min(N, i0 + G::kTile);
+        unsigned char* dst = tiles + (size_t)slot * G::kTileBytes + (size_t)(r0 - (i0 - kHalo)) * G::kRowBytes;
+        const uint32_t bytes = (uint32_t)(r1 - r0) * G::kRowBytes;
+        const unsigned char* src = base + (int64_t)r0 * G::kRowBytes;
+        fence_async_smem();
+        mbar_expect_tx(&full[slot], bytes);
+        for (uint32_t off = 0; off < bytes; off += 32768u)
+            bulk_load(dst + off, src + off, min(32768u, bytes - off), &full[slot], policy);
+    }
+};
+
+template <typename T, int D>
+constexpr size_t fused_smem_bytes() {
+    using G = Geo<T, D>;
+    return 2 * G::kTileBytes + BGeo<T, D>::kBytes + (size_t)G::kSegs * D * 4 + (size_t)G::kRows * 4 +
+           BGeo<T, D>::kAnchorBytes + 256;
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(Geo<T, D>::kThreads + 32 + kBThreads, 1) fused_scan_kernel(FusedArgs A) {
+    using G = Geo<T, D>;
+    using B = BGeo<T, D>;
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* tiles = smem;
+    unsigned char* tileB = smem + 2 * G::kTileBytes;
+    float* pp = reinterpret_cast<float*>(tileB + B::kBytes);                 // [kSegs][D]
+    float* invs = pp + G::kSegs * D;                                         // [kRows]
+    __nv_bfloat16* rhs = reinterpret_cast<__nv_bfloat16*>(invs + G::kRows);
+    unsigned char* small = reinterpret_cast<unsigned char*>(rhs) + B::kAnchorBytes;
+    Item* item = reinterpret_cast<Item*>(small);
+    uint32_t* mmk = reinterpret_cast<uint32_t*>(small + 32);
+    int* fin = reinterpret_cast<int*>(small + 80);
+    int* abort_flag = reinterpret_cast<int*>(small + 88);
+    uint64_t* full = reinterpret_cast<uint64_t*>(small + 96);
+    uint64_t* mbarB = reinterpret_cast<uint64_t*>(small + 112);
+    int* bslot = reinterpret_cast<int*>(small + 120);
+    float* bsc = reinterpret_cast<float*>(small + 128);
+
+    const int N = A.K.N;
+    const int tiles_per_unit = (N + G::kTile - 1) / G::kTile;
+    const int tid = threadIdx.x;
+    constexpr int kAll = G::kThreads + 32;   // pass-A threads and the control warp share the item barrier
+
+    if (tid == 0) {
+        mbar_init(&full[0], 1);
+        mbar_init(&full[1], 1);
+        mbar_init(mbarB, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        for (int i = 0; i < 12; ++i) mmk[i] = (i & 1) ? 0u : 0xffffffffu;
+        fin[0] = fin[1] = -1;
+        *abort_flag = 0;
+    }
+    __syncthreads();
+
+    if (tid >= kAll) {
+        pass_b_group<T, D>(A, tileB, rhs, bsc, bslot, mbarB, abort_flag);
+        return;
+    }
+
+    if (tid >= G::kThreads) {
+        // ------------------------------------------------------------------ control warp
+        // All 32 lanes run the loop together (the per-item barrier is warp-aligned); lane 0 works.
+        const int lane = tid - G::kThreads;
+        const int strips = (tiles_per_unit + A.strip - 1) / A.strip;
+        Ctl<T, D> C{A, tiles, item, full, abort_flag, tiles_per_unit, strips, (long long)A.units * strips,
+                    A.hints ? l2_policy_keep() : l2_policy_normal()};
+        Item nxt;   // the next item to issue (lane 0), fetched ahead of time
+        nxt.kind = 2;
+        nxt.unit = nxt.tile = nxt.pad = 0;
+        int left = 0;   // tiles that follow `nxt` in its strip
+        auto advance = [&]() {
+            if (left > 0) {
+                ++nxt.tile;
+                --left;
+            } else {
+                nxt = C.decode(C.take_ticket());
+                left = C.rest_of_strip(nxt);
+            }
+        };
+        if (lane == 0) {
+            advance();
+            C.issue(0, nxt);
+            advance();
+            C.issue(1, nxt);
+            advance();
+        }
+        __syncwarp();
+        bar_sync(kBarEnd, kAll);   // start: both descriptors are visible
+        bool prev_done = false;
+        for (int k = 0;; ++k) {
+            const Item cur = item[k & 1];
+            bar_sync(kBarEnd, kAll);   // the pass-A threads have finished item k
+            const bool done = cur.kind == 2;
+            if (done && prev_done) break;
+            prev_done = done;
+            if (lane == 0) {
+                C.issue(k & 1, nxt);   // item k + 2 goes into the buffer that item k has released
+                // Two global atomics, both in flight at once: the next ticket (needed at the next item
+                // barrier) and the tile counter of the head.  No fence here: the pass-A threads fence
+                // their block sums before the item barrier.
+                const bool in_strip = left > 0;
+                const bool more = !in_strip && nxt.kind != 2;
+                unsigned long long t_raw = ~0ULL;
+                if (more) t_raw = C.take_ticket();
+                int fin_unit = -1;
+                if (cur.kind == 0) {
+                    const int prev = atomicAdd(A.ctrl + kCtrlHeader + cur.unit, 1);
+                    if (prev == tiles_per_unit - 1) fin_unit = cur.unit;
+                    // publish the tile's min/max of a_c and re-arm the slots
+                    uint32_t* m = mmk + (k & 1) * 6;
+                    if (m[4] != 0xffffffffu) atomicMin(&A.mm[(int64_t)cur.unit * 6 + 4], m[4]);
+                    if (m[5] != 0u) atomicMax(&A.mm[(int64_t)cur.unit * 6 + 5], m[5]);
+                    m[4] = 0xffffffffu;
+                    m[5] = 0u;
+                }
+                fin[k & 1] = fin_unit;
+                if (in_strip) {
+                    ++nxt.tile;
+                    --left;
+                } else if (more) {
+                    nxt = C.decode(t_raw);
+                    left = C.rest_of_strip(nxt);
+                } else {
+                    nxt.kind = 2;
+                }
+            }
+            __syncwarp();
+        }
+        return;
+    }
+
+    // ---------------------------------------------------------------------- pass-A threads
+    bar_sync(kBarEnd, kAll);   // start
+    bool prev_done = false;
+    for (int k = 0;; ++k) {
+        const Item cur = item[k & 1];
+        const int buf = k & 1;
+        if (cur.kind == 0)
+            pass_a<T, D>(A, cur.unit, cur.tile, tiles + (size_t)buf * G::kTileBytes, pp, invs, mmk + buf * 6, &full[buf],
+                         (uint32_t)((k >> 1) & 1), abort_flag);
+        bar_sync(kBarEnd, kAll);   // end of item k
+        const bool done = cur.kind == 2;
+        if (done && prev_done) break;
+        prev_done = done;
+        // the head completed by item k - 1 (known since the control warp passed this barrier) gets its anchors
+        if (k >= 1) {
+            const int f = fin[(k - 1) & 1];
+            if (f >= 0) finalize_head<T, D>(A, f, pp, invs);
+        }
+    }
+}
+
+__global__ void fused_init_kernel(int units, uint32_t* mm, int* ctrl) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < (long long)units * 6) mm[i] = (i & 1) ? 0u : 0xffffffffu;
+    if (i < (long long)kCtrlHeader + 2LL * units) ctrl[i] = 0;
+}
+
+template <typename T, int D>
+cudaError_t launch_one(const FusedArgs& A, int sm_count, cudaStream_t stream) {
+    using G = Geo<T, D>;
+    const long long tiles = (long long)A.units * ((A.K.N + G::kTile - 1) / G::kTile);
+    const unsigned grid = (unsigned)(tiles < sm_count ? tiles : sm_count);
+    fused_scan_kernel<T, D><<<grid, G::kThreads + 32 + kBThreads, fused_smem_bytes<T, D>(), stream>>>(A);
+    return cudaGetLastError();
+}
 
 }  // namespace
 
@@ -773,7 +988,7 @@ cudaError_t configure_fused_kernels() {
 #define CALL(T, D)                                                                                          \
     if (e == cudaSuccess)                                                                                   \
     e = cudaFuncSetAttribute(fused_scan_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,          \
-                             (int)Geo<T, D>::kSmem)
+                             (int)fused_smem_bytes<T, D>())
     CALL(__nv_bfloat16, 64);
     CALL(__nv_bfloat16, 128);
     CALL(float, 64);
