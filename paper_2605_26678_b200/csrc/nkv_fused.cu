@@ -458,45 +458,49 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
     using G = Geo<T, D>;
     using B = BGeo<T, D>;
     constexpr int NP = G::kNP, L = G::kL;
+    constexpr int kHalfRows = B::kRows / 2;                       // rows per sub-tile (one half of the buffer)
+    constexpr int kHalfBytes = B::kBytes / 2;
     const int N = A.K.N, b = A.sp.block, nb = A.sp.nblocks;
     const int bt = threadIdx.x - (G::kThreads + 32), warp = bt >> 5, lane = bt & 31;
     const int tiles_per_unit = (N + G::kTile - 1) / G::kTile;
     const long long total = (long long)A.units * tiles_per_unit;
     unsigned long long* ticket = reinterpret_cast<unsigned long long*>(A.ctrl + 2);
     const uint64_t policy = A.hints ? l2_policy_stream() : l2_policy_normal();
-    // a sub-tile overlaps at most ceil(kRows / b) + 1 blocks; the staged right-hand sides hold four
-    const bool mma_path = sizeof(T) == 2 && b % 16 == 0 && (B::kRows + b - 1) / b + 1 <= 4;
-    uint32_t copies = 0;   // copies awaited so far (mbarrier parity)
+    // a sub-tile overlaps at most ceil(kHalfRows / b) + 1 blocks; the staged right-hand sides hold four
+    const bool mma_path = sizeof(T) == 2 && b % 16 == 0 && (kHalfRows + b - 1) / b + 1 <= 4;
+    uint32_t used[2] = {0u, 0u};   // copies awaited so far per half (mbarrier parity)
+    unsigned long long next_t = 0;
+    if (bt == 0) next_t = atomicAdd(ticket, 1ULL);   // always one ticket ahead
+    int staged_u = -1, staged_blk0 = -1, staged_n = 0;
 
     for (;;) {
         if (bt == 0) {
             int u = -1, tile = 0;
-            if (*reinterpret_cast<volatile int*>(abort_flag) == 0) {
-                const unsigned long long t = atomicAdd(ticket, 1ULL);
-                if ((long long)t < total) {
-                    u = (int)(t / (unsigned long long)tiles_per_unit);
-                    tile = (int)(t - (unsigned long long)u * tiles_per_unit);
-                    // wait (bounded) until the head's anchors have been published
-                    const int* ready = A.ctrl + kCtrlHeader + A.units + u;
-                    bool ok = ld_acquire(ready) != 0;
-                    if (!ok) {
-                        const unsigned long long t0 = now_ns();
-                        for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
-                            if (ld_acquire(ready) != 0) {
-                                ok = true;
-                                break;
-                            }
-                            __nanosleep(256);
-                            if ((spin & 15u) == 15u && (*reinterpret_cast<volatile int*>(abort_flag) != 0 ||
-                                                        now_ns() - t0 > kWaitLimitNs))
-                                break;
+            const unsigned long long t = next_t;
+            if ((long long)t < total && *reinterpret_cast<volatile int*>(abort_flag) == 0) {
+                next_t = atomicAdd(ticket, 1ULL);
+                u = (int)(t / (unsigned long long)tiles_per_unit);
+                tile = (int)(t - (unsigned long long)u * tiles_per_unit);
+                // wait (bounded) until the head's anchors have been published
+                const int* ready = A.ctrl + kCtrlHeader + A.units + u;
+                bool ok = ld_acquire(ready) != 0;
+                if (!ok) {
+                    const unsigned long long t0 = now_ns();
+                    for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+                        if (ld_acquire(ready) != 0) {
+                            ok = true;
+                            break;
                         }
+                        __nanosleep(256);
+                        if ((spin & 15u) == 15u &&
+                            (*reinterpret_cast<volatile int*>(abort_flag) != 0 || now_ns() - t0 > kWaitLimitNs))
+                            break;
                     }
-                    if (!ok) {
-                        set_status(A.status, NKV_ERR_TIMEOUT, 502);
-                        *abort_flag = 1;
-                        u = -1;
-                    }
+                }
+                if (!ok) {
+                    set_status(A.status, NKV_ERR_TIMEOUT, 502);
+                    *abort_flag = 1;
+                    u = -1;
                 }
             }
             bslot[0] = u;
@@ -510,52 +514,72 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
                                     ((int64_t)g * A.K.stride_g + (int64_t)h * A.K.stride_h) * (int64_t)sizeof(T);
         float lo_s = INFINITY, hi_s = -INFINITY, lo_e = INFINITY, hi_e = -INFINITY;
         const float rs = __ldcg(A.inv_s + u);
+        const int row_begin = tile_idx * G::kTile, row_end = min(N, (tile_idx + 1) * G::kTile);
+        auto issue = [&](int r0, int half) {   // thread 0 of the group
+            const uint32_t bytes = (uint32_t)(min(row_end, r0 + kHalfRows) - r0) * G::kRowBytes;
+            fence_async_smem();
+            mbar_expect_tx(&mbarB[half], bytes);
+            bulk_load(tileB + (size_t)half * kHalfBytes, base + (int64_t)r0 * G::kRowBytes, bytes, &mbarB[half], policy);
+        };
+        if (bt == 0) issue(row_begin, 0);
 
-        for (int r0 = tile_idx * G::kTile; r0 < min(N, (tile_idx + 1) * G::kTile); r0 += B::kRows) {
-            const int rows = min(N, r0 + B::kRows) - r0;
-            if (bt == 0) {
-                const uint32_t bytes = (uint32_t)rows * G::kRowBytes;
-                fence_async_smem();
-                mbar_expect_tx(mbarB, bytes);
-                bulk_load(tileB, base + (int64_t)r0 * G::kRowBytes, bytes, mbarB, policy);
-            }
+        int sub = 0;
+        for (int r0 = row_begin; r0 < row_end; r0 += kHalfRows, ++sub) {
+            const int half = sub & 1;
+            const int rows = min(row_end, r0 + kHalfRows) - r0;
+            // the other half was released by the barrier that ended the previous sub-tile
+            if (bt == 0 && r0 + kHalfRows < row_end) issue(r0 + kHalfRows, half ^ 1);
+            const unsigned char* buf = tileB + (size_t)half * kHalfBytes;
             const int blk0 = r0 / b;
-            if (mma_path) {
-                if constexpr (sizeof(T) == 2) {
-                    // split right-hand sides of the sub-tile's blocks, one anchor column per thread
-                    const int nblk = min(nb - 1, (r0 + rows - 1) / b) - blk0 + 1;
-                    if (bt < D) {
-                        const float mu = __ldcg(A.mu_s + (int64_t)u * D + bt);
-                        for (int q = 0; q < nblk; ++q) {
-                            __nv_bfloat16* r = rhs + (size_t)q * 8 * D + bt;
-                            split3_bf16(mu, r, D);
-                            split3_bf16(__ldcg(A.block_sums + ((int64_t)u * nb + blk0 + q) * D + bt), r + 3 * D, D);
-                            r[6 * D] = __float2bfloat16_rn(0.f);
-                            r[7 * D] = __float2bfloat16_rn(0.f);
-                        }
-                        if (bt < nblk) bsc[bt] = __ldcg(A.inv_e + (int64_t)u * nb + blk0 + bt);
-                    }
-                }
-            }
-            bar_sync(kBarB, kBThreads);   // right-hand sides visible
-            if (!mbar_wait(mbarB, copies & 1u, abort_flag)) {
-                set_status(A.status, NKV_ERR_TIMEOUT, 503);
-                *abort_flag = 1;
-            }
-            ++copies;
             if (mma_path) {
                 if constexpr (sizeof(T) == 2) {
                     constexpr int kCh = D / 32;
                     const int gq = lane >> 2, t = lane & 3;
                     const int row_in_block = gq + ((t & 2) ? 8 : 0);
-                    for (int rb = warp; rb * 16 < rows; rb += kBThreads / 32) {
-                        const int rr = rb * 16;
+                    // split right-hand sides of the sub-tile's blocks (restaged only when they change)
+                    const int nblk = min(nb - 1, (r0 + rows - 1) / b) - blk0 + 1;
+                    const bool restage = u != staged_u || blk0 != staged_blk0 || nblk > staged_n;
+                    if (restage) {
+                        if (bt < D) {
+                            const float mu = __ldcg(A.mu_s + (int64_t)u * D + bt);
+                            for (int q = 0; q < nblk; ++q) {
+                                __nv_bfloat16* r = rhs + (size_t)q * 8 * D + bt;
+                                split3_bf16(mu, r, D);
+                                split3_bf16(__ldcg(A.block_sums + ((int64_t)u * nb + blk0 + q) * D + bt), r + 3 * D, D);
+                                r[6 * D] = __float2bfloat16_rn(0.f);
+                                r[7 * D] = __float2bfloat16_rn(0.f);
+                            }
+                            if (bt < nblk) bsc[bt] = __ldcg(A.inv_e + (int64_t)u * nb + blk0 + bt);
+                        }
+                        staged_u = u;
+                        staged_blk0 = blk0;
+                        staged_n = nblk;
+                    }
+                    // reciprocal norm of the key this lane finishes, fetched before the copy is awaited
+                    constexpr int kIters = (kHalfRows / 16 + kBThreads / 32 - 1) / (kBThreads / 32);
+                    float inv_pre[kIters];
+#pragma unroll
+                    for (int it = 0; it < kIters; ++it) {
+                        const int gi = r0 + (warp + it * (kBThreads / 32)) * 16 + row_in_block;
+                        inv_pre[it] = (warp + it * (kBThreads / 32)) * 16 < rows && gi < N
+                                          ? __ldcg(A.inv_norm + (int64_t)u * N + gi)
+                                          : 0.f;
+                    }
+                    if (restage) bar_sync(kBarB, kBThreads);   // right-hand sides visible (uniform condition)
+                    if (!mbar_wait(&mbarB[half], used[half] & 1u, abort_flag)) {
+                        set_status(A.status, NKV_ERR_TIMEOUT, 503);
+                        *abort_flag = 1;
+                    }
+                    ++used[half];
+#pragma unroll
+                    for (int it = 0; it < kIters; ++it) {
+                        const int rr = (warp + it * (kBThreads / 32)) * 16;
+                        if (rr >= rows) break;
                         const int q = min((r0 + rr) / b, nb - 1) - blk0;
                         const float re = bsc[q];
                         const int gi = r0 + rr + row_in_block;
-                        const float inv_mine = gi < N ? __ldcg(A.inv_norm + (int64_t)u * N + gi) : 0.f;
                         float c[4] = {0.f, 0.f, 0.f, 0.f};
-                        const unsigned char* row_lo = tileB + (size_t)(rr + gq) * G::kRowBytes;
+                        const unsigned char* row_lo = buf + (size_t)(rr + gq) * G::kRowBytes;
                         const unsigned char* row_hi = row_lo + 8 * G::kRowBytes;
                         const __nv_bfloat16* rq = rhs + ((size_t)q * 8 + gq) * D;
 #pragma unroll
@@ -583,7 +607,7 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
                         // each lane finishes one of its quad's four results: t=0: a_s(row g), t=1: a_e(row g),
                         // t=2: a_s(row g+8), t=3: a_e(row g+8)
                         const float dot = t == 0 ? xs_lo : (t == 1 ? xe_lo : (t == 2 ? xs_hi : xe_hi));
-                        const float a = -(dot * inv_mine) * ((t & 1) ? re : rs) + 0.f;
+                        const float a = -(dot * inv_pre[it]) * ((t & 1) ? re : rs) + 0.f;
                         if (gi < N) {
                             A.a_raw[((int64_t)u * 3 + (t & 1)) * N + gi] = a;
                             if (t & 1) {
@@ -598,7 +622,12 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
                 }
             } else {
                 // packed FMAs: an L-lane group walks 8 rows; whole warps run every iteration (groups past
-                // the end compute on stale rows and write nothing)
+                // the end compute on stale rows and write nothing); anchors come from L2
+                if (!mbar_wait(&mbarB[half], used[half] & 1u, abort_flag)) {
+                    set_status(A.status, NKV_ERR_TIMEOUT, 503);
+                    *abort_flag = 1;
+                }
+                ++used[half];
                 const int grp = bt / L, l = bt % L;
                 F2 ms[NP];
                 G::load_vec(A.mu_s + (int64_t)u * D, l, ms);
@@ -612,11 +641,11 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
                     const int o_mine = L == 16 ? (l >> 1) : l;
                     const float inv_mine = gi0 + o_mine < N ? __ldcg(A.inv_norm + (int64_t)u * N + gi0 + o_mine) : 0.f;
                     float part[16];
-                    const int seg_c = min(seg, B::kRows / kSeg - 1);   // stay inside the buffer
+                    const int seg_c = min(seg, kHalfRows / kSeg - 1);   // stay inside the buffer
 #pragma unroll
                     for (int o = 0; o < kSeg; ++o) {
                         F2 kn[NP];
-                        G::load_row(tileB + (size_t)(seg_c * kSeg + o) * G::kRowBytes, l, kn);
+                        G::load_row(buf + (size_t)(seg_c * kSeg + o) * G::kRowBytes, l, kn);
                         F2 ds = pack2(0.f, 0.f), de = pack2(0.f, 0.f);
 #pragma unroll
                         for (int p = 0; p < NP; ++p) {
@@ -655,7 +684,7 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
                     }
                 }
             }
-            bar_sync(kBarB, kBThreads);   // the buffer and the right-hand sides may be overwritten
+            bar_sync(kBarB, kBThreads);   // this half (and, next time they change, the right-hand sides) is free
         }
         lo_s = warp_min(lo_s);
         hi_s = warp_max(hi_s);
@@ -763,9 +792,9 @@ __device__ __forceinline__ void finalize_head(const FusedArgs& A, int u, float* 
 //   80 fin[2]       head whose anchors this CTA owes after item k (or -1), written by the control warp
 //   88 abort_flag   a bounded wait ran out somewhere in this CTA
 //   96 full[2]      mbarriers of the two pass-A tile buffers
-//   112 mbarB       mbarrier of the pass-B buffer
-//   120 bslot[2]    head and tile of the pass-B group's current ticket
-//   128 bsc[8]      1/||mu_e|| of the blocks of the current pass-B sub-tile
+//   112 mbarB[2]    mbarriers of the two halves of the pass-B buffer
+//   128 bslot[2]    head and tile of the pass-B group's current ticket
+//   136 bsc[8]      1/||mu_e|| of the blocks of the current pass-B sub-tile
 template <typename T, int D>
 struct Ctl {
     using G = Geo<T, D>;
@@ -840,8 +869,8 @@ __global__ void __launch_bounds__(Geo<T, D>::kThreads + 32 + kBThreads, 1) fused
     int* abort_flag = reinterpret_cast<int*>(small + 88);
     uint64_t* full = reinterpret_cast<uint64_t*>(small + 96);
     uint64_t* mbarB = reinterpret_cast<uint64_t*>(small + 112);
-    int* bslot = reinterpret_cast<int*>(small + 120);
-    float* bsc = reinterpret_cast<float*>(small + 128);
+    int* bslot = reinterpret_cast<int*>(small + 128);
+    float* bsc = reinterpret_cast<float*>(small + 136);
 
     const int N = A.K.N;
     const int tiles_per_unit = (N + G::kTile - 1) / G::kTile;
@@ -851,7 +880,8 @@ __global__ void __launch_bounds__(Geo<T, D>::kThreads + 32 + kBThreads, 1) fused
     if (tid == 0) {
         mbar_init(&full[0], 1);
         mbar_init(&full[1], 1);
-        mbar_init(mbarB, 1);
+        mbar_init(&mbarB[0], 1);
+        mbar_init(&mbarB[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         for (int i = 0; i < 12; ++i) mmk[i] = (i & 1) ? 0u : 0xffffffffu;
         fin[0] = fin[1] = -1;
