@@ -523,20 +523,24 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
         float lo_s = INFINITY, hi_s = -INFINITY, lo_e = INFINITY, hi_e = -INFINITY;
         const float rs = __ldcg(A.inv_s + u);
         const int row_begin = tile_idx * G::kTile, row_end = min(N, (tile_idx + 1) * G::kTile);
-        // thread 0: copy one sub-tile of ticket `t` starting at row `r` into the next ring slot
-        auto issue_at = [&](unsigned long long t, int r) {
-            const int uu = (int)(t / (unsigned long long)tiles_per_unit);
-            const int tl = (int)(t - (unsigned long long)uu * tiles_per_unit);
-            const int end = min(N, (tl + 1) * G::kTile);
-            const unsigned char* src = reinterpret_cast<const unsigned char*>(A.K.ptr) +
-                                       ((int64_t)(uu / A.K.H) * A.K.stride_g + (int64_t)(uu % A.K.H) * A.K.stride_h) *
-                                           (int64_t)sizeof(T) +
-                                       (int64_t)r * G::kRowBytes;
+        // thread 0: the next ticket's tile, decoded once (64-bit divisions are slow for a single thread)
+        const unsigned char* next_base = nullptr;
+        int next_begin = 0, next_end = 0;
+        if (bt == 0 && (long long)next_t < total) {
+            const int uu = (int)(next_t / (unsigned long long)tiles_per_unit);
+            const int tl = (int)(next_t - (unsigned long long)uu * tiles_per_unit);
+            next_base = reinterpret_cast<const unsigned char*>(A.K.ptr) +
+                        ((int64_t)(uu / A.K.H) * A.K.stride_g + (int64_t)(uu % A.K.H) * A.K.stride_h) * (int64_t)sizeof(T);
+            next_begin = tl * G::kTile;
+            next_end = min(N, (tl + 1) * G::kTile);
+        }
+        // thread 0: copy one sub-tile (rows r .. of a tile ending at `end`) into the next ring slot
+        auto issue_at = [&](const unsigned char* tile_base, int r, int end) {
             const uint32_t bytes = (uint32_t)(min(end, r + kHalfRows) - r) * G::kRowBytes;
             const int slot = (int)(issued % kStages);
             fence_async_smem();
             mbar_expect_tx(&mbarB[slot], bytes);
-            bulk_load(tileB + (size_t)slot * kHalfBytes, src, bytes, &mbarB[slot], policy);
+            bulk_load(tileB + (size_t)slot * kHalfBytes, tile_base + (int64_t)r * G::kRowBytes, bytes, &mbarB[slot], policy);
             ++issued;
         };
         // thread 0: keep up to kStages - 1 copies in flight; the cursor walks this tile, then the next ticket's
@@ -547,17 +551,18 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
                 cursor_valid = true;
             }
             while (issued - consumed < (uint32_t)(kStages - 1)) {
-                const unsigned long long t = cursor_on_next ? next_t : cur_t;
-                if ((long long)t >= total) break;
-                const int tl = (int)(t % (unsigned long long)tiles_per_unit);
-                const int end = min(N, (tl + 1) * G::kTile);
-                if (cursor_row >= end) {
-                    if (cursor_on_next) break;   // both tiles fully issued
+                if (!cursor_on_next) {
+                    if (cursor_row < row_end) {
+                        issue_at(base, cursor_row, row_end);
+                        cursor_row += kHalfRows;
+                        continue;
+                    }
+                    if (next_base == nullptr) break;
                     cursor_on_next = 1;
-                    cursor_row = (int)(next_t % (unsigned long long)tiles_per_unit) * G::kTile;
-                    continue;
+                    cursor_row = next_begin;
                 }
-                issue_at(t, cursor_row);
+                if (cursor_row >= next_end) break;   // both tiles fully issued
+                issue_at(next_base, cursor_row, next_end);
                 cursor_row += kHalfRows;
             }
         };
