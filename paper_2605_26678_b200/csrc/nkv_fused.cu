@@ -567,6 +567,7 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
             }
         };
 
+        float inv_next[(kHalfRows / 16 + kBThreads / 32 - 1) / (kBThreads / 32)] = {};
         for (int r0 = row_begin; r0 < row_end; r0 += kHalfRows) {
             const int half = (int)(consumed % kStages);
             const int rows = min(row_end, r0 + kHalfRows) - r0;
@@ -597,15 +598,21 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
                         staged_blk0 = blk0;
                         staged_n = nblk;
                     }
-                    // reciprocal norm of the key this lane finishes, fetched before the copy is awaited
+                    // reciprocal norm of the key this lane finishes: the values of this sub-tile were fetched
+                    // while the previous one was being worked on (directly at the first sub-tile of a tile)
                     constexpr int kIters = (kHalfRows / 16 + kBThreads / 32 - 1) / (kBThreads / 32);
                     float inv_pre[kIters];
 #pragma unroll
                     for (int it = 0; it < kIters; ++it) {
-                        const int gi = r0 + (warp + it * (kBThreads / 32)) * 16 + row_in_block;
-                        inv_pre[it] = (warp + it * (kBThreads / 32)) * 16 < rows && gi < N
-                                          ? __ldcg(A.inv_norm + (int64_t)u * N + gi)
-                                          : 0.f;
+                        const int off = (warp + it * (kBThreads / 32)) * 16 + row_in_block;
+                        if (r0 == row_begin) {
+                            const int gi = r0 + off;
+                            inv_pre[it] = off < rows && gi < N ? __ldcg(A.inv_norm + (int64_t)u * N + gi) : 0.f;
+                        } else {
+                            inv_pre[it] = inv_next[it];
+                        }
+                        const int gn = r0 + kHalfRows + off;   // same lane, next sub-tile of this tile
+                        inv_next[it] = gn < row_end ? __ldcg(A.inv_norm + (int64_t)u * N + gn) : 0.f;
                     }
                     if (restage) bar_sync(kBarB, kBThreads);   // right-hand sides visible (uniform condition)
                     if (!mbar_wait(&mbarB[half], (consumed / kStages) & 1u, abort_flag)) {
