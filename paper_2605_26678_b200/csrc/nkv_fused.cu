@@ -567,7 +567,8 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
             }
         };
 
-        float inv_next[(kHalfRows / 16 + kBThreads / 32 - 1) / (kBThreads / 32)] = {};
+        constexpr int kItersB = kHalfRows >= 16 ? (kHalfRows / 16 + kBThreads / 32 - 1) / (kBThreads / 32) : 1;
+        float inv_next[kItersB] = {};
         for (int r0 = row_begin; r0 < row_end; r0 += kHalfRows) {
             const int half = (int)(consumed % kStages);
             const int rows = min(row_end, r0 + kHalfRows) - r0;
@@ -600,7 +601,7 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
                     }
                     // reciprocal norm of the key this lane finishes: the values of this sub-tile were fetched
                     // while the previous one was being worked on (directly at the first sub-tile of a tile)
-                    constexpr int kIters = (kHalfRows / 16 + kBThreads / 32 - 1) / (kBThreads / 32);
+                    constexpr int kIters = kItersB;
                     float inv_pre[kIters];
 #pragma unroll
                     for (int it = 0; it < kIters; ++it) {
