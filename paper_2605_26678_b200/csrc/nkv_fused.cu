@@ -458,9 +458,8 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
     using G = Geo<T, D>;
     using B = BGeo<T, D>;
     constexpr int NP = G::kNP, L = G::kL;
-    constexpr int kStages = 4;                                    // ring of sub-tile buffers, three copies in flight
-    constexpr int kHalfRows = B::kRows / kStages;                 // rows per sub-tile
-    constexpr int kHalfBytes = B::kBytes / kStages;
+    constexpr int kHalfRows = B::kRows / 2;                       // rows per sub-tile (one half of the buffer)
+    constexpr int kHalfBytes = B::kBytes / 2;
     const int N = A.K.N, b = A.sp.block, nb = A.sp.nblocks;
     const int bt = threadIdx.x - (G::kThreads + 32), warp = bt >> 5, lane = bt & 31;
     const int tiles_per_unit = (N + G::kTile - 1) / G::kTile;
@@ -469,24 +468,17 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
     const uint64_t policy = A.hints ? l2_policy_stream() : l2_policy_normal();
     // a sub-tile overlaps at most ceil(kHalfRows / b) + 1 blocks; the staged right-hand sides hold four
     const bool mma_path = sizeof(T) == 2 && b % 16 == 0 && (kHalfRows + b - 1) / b + 1 <= 4;
-    uint32_t consumed = 0;   // sub-tiles consumed so far: slot = consumed % kStages, parity = (consumed / kStages) & 1
-    // thread 0 only: the copy cursor runs up to three sub-tiles ahead of consumption, across tile boundaries
-    // (the copies do not depend on the anchors, only the arithmetic does)
-    unsigned long long cur_t = 0, next_t = 0;
-    uint32_t issued = 0;
-    int cursor_on_next = 0, cursor_row = 0;   // where the next copy starts: in the current or the next ticket's tile
-    bool cursor_valid = false;
-    if (bt == 0) {
-        cur_t = atomicAdd(ticket, 1ULL);
-        next_t = atomicAdd(ticket, 1ULL);
-    }
+    uint32_t used[2] = {0u, 0u};   // copies awaited so far per half (mbarrier parity)
+    unsigned long long next_t = 0;
+    if (bt == 0) next_t = atomicAdd(ticket, 1ULL);   // always one ticket ahead
     int staged_u = -1, staged_blk0 = -1, staged_n = 0;
 
     for (;;) {
         if (bt == 0) {
             int u = -1, tile = 0;
-            const unsigned long long t = cur_t;
+            const unsigned long long t = next_t;
             if ((long long)t < total && *reinterpret_cast<volatile int*>(abort_flag) == 0) {
+                next_t = atomicAdd(ticket, 1ULL);
                 u = (int)(t / (unsigned long long)tiles_per_unit);
                 tile = (int)(t - (unsigned long long)u * tiles_per_unit);
                 // wait (bounded) until the head's anchors have been published
@@ -523,56 +515,20 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
         float lo_s = INFINITY, hi_s = -INFINITY, lo_e = INFINITY, hi_e = -INFINITY;
         const float rs = __ldcg(A.inv_s + u);
         const int row_begin = tile_idx * G::kTile, row_end = min(N, (tile_idx + 1) * G::kTile);
-        // thread 0: the next ticket's tile, decoded once (64-bit divisions are slow for a single thread)
-        const unsigned char* next_base = nullptr;
-        int next_begin = 0, next_end = 0;
-        if (bt == 0 && (long long)next_t < total) {
-            const int uu = (int)(next_t / (unsigned long long)tiles_per_unit);
-            const int tl = (int)(next_t - (unsigned long long)uu * tiles_per_unit);
-            next_base = reinterpret_cast<const unsigned char*>(A.K.ptr) +
-                        ((int64_t)(uu / A.K.H) * A.K.stride_g + (int64_t)(uu % A.K.H) * A.K.stride_h) * (int64_t)sizeof(T);
-            next_begin = tl * G::kTile;
-            next_end = min(N, (tl + 1) * G::kTile);
-        }
-        // thread 0: copy one sub-tile (rows r .. of a tile ending at `end`) into the next ring slot
-        auto issue_at = [&](const unsigned char* tile_base, int r, int end) {
-            const uint32_t bytes = (uint32_t)(min(end, r + kHalfRows) - r) * G::kRowBytes;
-            const int slot = (int)(issued % kStages);
+        auto issue = [&](int r0, int half) {   // thread 0 of the group
+            const uint32_t bytes = (uint32_t)(min(row_end, r0 + kHalfRows) - r0) * G::kRowBytes;
             fence_async_smem();
-            mbar_expect_tx(&mbarB[slot], bytes);
-            bulk_load(tileB + (size_t)slot * kHalfBytes, tile_base + (int64_t)r * G::kRowBytes, bytes, &mbarB[slot], policy);
-            ++issued;
+            mbar_expect_tx(&mbarB[half], bytes);
+            bulk_load(tileB + (size_t)half * kHalfBytes, base + (int64_t)r0 * G::kRowBytes, bytes, &mbarB[half], policy);
         };
-        // thread 0: keep up to kStages - 1 copies in flight; the cursor walks this tile, then the next ticket's
-        auto top_up = [&]() {
-            if (!cursor_valid) {   // (re)start: at the first sub-tile not yet issued
-                cursor_on_next = 0;
-                cursor_row = row_begin;
-                cursor_valid = true;
-            }
-            while (issued - consumed < (uint32_t)(kStages - 1)) {
-                if (!cursor_on_next) {
-                    if (cursor_row < row_end) {
-                        issue_at(base, cursor_row, row_end);
-                        cursor_row += kHalfRows;
-                        continue;
-                    }
-                    if (next_base == nullptr) break;
-                    cursor_on_next = 1;
-                    cursor_row = next_begin;
-                }
-                if (cursor_row >= next_end) break;   // both tiles fully issued
-                issue_at(next_base, cursor_row, next_end);
-                cursor_row += kHalfRows;
-            }
-        };
+        if (bt == 0) issue(row_begin, 0);
 
-        constexpr int kItersB = kHalfRows >= 16 ? (kHalfRows / 16 + kBThreads / 32 - 1) / (kBThreads / 32) : 1;
-        float inv_next[kItersB] = {};
-        for (int r0 = row_begin; r0 < row_end; r0 += kHalfRows) {
-            const int half = (int)(consumed % kStages);
+        int sub = 0;
+        for (int r0 = row_begin; r0 < row_end; r0 += kHalfRows, ++sub) {
+            const int half = sub & 1;
             const int rows = min(row_end, r0 + kHalfRows) - r0;
-            if (bt == 0) top_up();
+            // the other half was released by the barrier that ended the previous sub-tile
+            if (bt == 0 && r0 + kHalfRows < row_end) issue(r0 + kHalfRows, half ^ 1);
             const unsigned char* buf = tileB + (size_t)half * kHalfBytes;
             const int blk0 = r0 / b;
             if (mma_path) {
@@ -599,27 +555,22 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
                         staged_blk0 = blk0;
                         staged_n = nblk;
                     }
-                    // reciprocal norm of the key this lane finishes: the values of this sub-tile were fetched
-                    // while the previous one was being worked on (directly at the first sub-tile of a tile)
-                    constexpr int kIters = kItersB;
+                    // reciprocal norm of the key this lane finishes, fetched before the copy is awaited
+                    constexpr int kIters = (kHalfRows / 16 + kBThreads / 32 - 1) / (kBThreads / 32);
                     float inv_pre[kIters];
 #pragma unroll
                     for (int it = 0; it < kIters; ++it) {
-                        const int off = (warp + it * (kBThreads / 32)) * 16 + row_in_block;
-                        if (r0 == row_begin) {
-                            const int gi = r0 + off;
-                            inv_pre[it] = off < rows && gi < N ? __ldcg(A.inv_norm + (int64_t)u * N + gi) : 0.f;
-                        } else {
-                            inv_pre[it] = inv_next[it];
-                        }
-                        const int gn = r0 + kHalfRows + off;   // same lane, next sub-tile of this tile
-                        inv_next[it] = gn < row_end ? __ldcg(A.inv_norm + (int64_t)u * N + gn) : 0.f;
+                        const int gi = r0 + (warp + it * (kBThreads / 32)) * 16 + row_in_block;
+                        inv_pre[it] = (warp + it * (kBThreads / 32)) * 16 < rows && gi < N
+                                          ? __ldcg(A.inv_norm + (int64_t)u * N + gi)
+                                          : 0.f;
                     }
                     if (restage) bar_sync(kBarB, kBThreads);   // right-hand sides visible (uniform condition)
-                    if (!mbar_wait(&mbarB[half], (consumed / kStages) & 1u, abort_flag)) {
+                    if (!mbar_wait(&mbarB[half], used[half] & 1u, abort_flag)) {
                         set_status(A.status, NKV_ERR_TIMEOUT, 503);
                         *abort_flag = 1;
                     }
+                    ++used[half];
 #pragma unroll
                     for (int it = 0; it < kIters; ++it) {
                         const int rr = (warp + it * (kBThreads / 32)) * 16;
@@ -672,10 +623,11 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
             } else {
                 // packed FMAs: an L-lane group walks 8 rows; whole warps run every iteration (groups past
                 // the end compute on stale rows and write nothing); anchors come from L2
-                if (!mbar_wait(&mbarB[half], (consumed / kStages) & 1u, abort_flag)) {
+                if (!mbar_wait(&mbarB[half], used[half] & 1u, abort_flag)) {
                     set_status(A.status, NKV_ERR_TIMEOUT, 503);
                     *abort_flag = 1;
                 }
+                ++used[half];
                 const int grp = bt / L, l = bt % L;
                 F2 ms[NP];
                 G::load_vec(A.mu_s + (int64_t)u * D, l, ms);
@@ -732,14 +684,7 @@ __device__ __forceinline__ void pass_b_group(const FusedArgs& A, unsigned char* 
                     }
                 }
             }
-            bar_sync(kBarB, kBThreads);   // this slot (and, next time they change, the right-hand sides) is free
-            ++consumed;
-        }
-        if (bt == 0) {   // the next ticket becomes the current one; keep one ticket ahead
-            cur_t = next_t;
-            next_t = (long long)cur_t < total ? atomicAdd(ticket, 1ULL) : cur_t;
-            if (cursor_on_next) cursor_on_next = 0;   // the cursor is already inside the new current tile
-            else cursor_valid = false;
+            bar_sync(kBarB, kBThreads);   // this half (and, next time they change, the right-hand sides) is free
         }
         lo_s = warp_min(lo_s);
         hi_s = warp_max(hi_s);
@@ -847,9 +792,9 @@ __device__ __forceinline__ void finalize_head(const FusedArgs& A, int u, float* 
 //   80 fin[2]       head whose anchors this CTA owes after item k (or -1), written by the control warp
 //   88 abort_flag   a bounded wait ran out somewhere in this CTA
 //   96 full[2]      mbarriers of the two pass-A tile buffers
-//   112 mbarB[4]    mbarriers of the pass-B ring
-//   144 bslot[2]    head and tile of the pass-B group's current ticket
-//   152 bsc[8]      1/||mu_e|| of the blocks of the current pass-B sub-tile
+//   112 mbarB[2]    mbarriers of the two halves of the pass-B buffer
+//   128 bslot[2]    head and tile of the pass-B group's current ticket
+//   136 bsc[8]      1/||mu_e|| of the blocks of the current pass-B sub-tile
 template <typename T, int D>
 struct Ctl {
     using G = Geo<T, D>;
@@ -924,8 +869,8 @@ __global__ void __launch_bounds__(Geo<T, D>::kThreads + 32 + kBThreads, 1) fused
     int* abort_flag = reinterpret_cast<int*>(small + 88);
     uint64_t* full = reinterpret_cast<uint64_t*>(small + 96);
     uint64_t* mbarB = reinterpret_cast<uint64_t*>(small + 112);
-    int* bslot = reinterpret_cast<int*>(small + 144);
-    float* bsc = reinterpret_cast<float*>(small + 152);
+    int* bslot = reinterpret_cast<int*>(small + 128);
+    float* bsc = reinterpret_cast<float*>(small + 136);
 
     const int N = A.K.N;
     const int tiles_per_unit = (N + G::kTile - 1) / G::kTile;
@@ -935,7 +880,8 @@ __global__ void __launch_bounds__(Geo<T, D>::kThreads + 32 + kBThreads, 1) fused
     if (tid == 0) {
         mbar_init(&full[0], 1);
         mbar_init(&full[1], 1);
-        for (int i = 0; i < 4; ++i) mbar_init(&mbarB[i], 1);
+        mbar_init(&mbarB[0], 1);
+        mbar_init(&mbarB[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         for (int i = 0; i < 12; ++i) mmk[i] = (i & 1) ? 0u : 0xffffffffu;
         fin[0] = fin[1] = -1;
