@@ -294,7 +294,7 @@ __device__ __forceinline__ float block_reduce_f(SelectShared& S, float v, int op
 // result is always exact.
 // ------------------------------------------------------------------------------------------
 constexpr int kSampleMin = 1024, kSampleMax = 32768;   // sample positions: n / 8, clamped
-constexpr int kCandSmall = 3072;                       // bracket capacity of the per-head kernels
+constexpr int kCandSmall = 4096;                       // bracket capacity of the per-head kernels
 constexpr int kCandLarge = 12288;                      // ... of the per-group kernel (dynamic shared memory)
 
 template <int CAP>
@@ -473,6 +473,126 @@ __device__ void block_select_bracket(SelectShared& S, BracketShared<CAP>& X, con
     }
 }
 
+// Sums of the m largest and of the m smallest of a[0..n) with both tails bracketed from one sample
+// histogram and collected in one pass (the two halves of X.cand hold the two brackets).  Returns false,
+// having computed nothing, when a bracket misses or the two overlap; the caller then selects each tail
+// on its own.  lo0 / sc0: value-linear binning of the whole range.
+template <int CAP>
+__device__ bool two_tail_sums(SelectShared& S, BracketShared<CAP>& X, const float* __restrict__ a, int n, int m,
+                              float lo0, float sc0, int* status, float* top_sum, float* bot_sum) {
+    constexpr int kHalf = CAP / 2;
+    __shared__ int sh_n[2], sh_cnt[2], sh_ok;
+    __shared__ float sh_piv[4], sh_sum[2], sh_res[2];
+    const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
+    if (n <= CAP || 2 * m >= n) return false;
+    // 1. histogram of a strided sample
+    const int positions = min(max(n / 8, kSampleMin), kSampleMax);
+    for (int b = tid; b < kBins; b += nt) S.hist[b] = 0;
+    __syncthreads();
+    for (int i = tid; i < positions; i += nt) atomicAdd(&S.hist[bin_of(a[(int)(((long long)i * n) / positions)], lo0, sc0)], 1);
+    __syncthreads();
+    const int sn = positions;
+    // 2. four pivots: ranks (counted from the top) around m and around n - m + 1
+    const float qt = (float)m * (float)sn / (float)n, qb = (float)(n - m + 1) * (float)sn / (float)n;
+    const float sdt = sqrtf(fmaxf(qt * (1.0f - qt / (float)sn), 1.0f)), sdb = sqrtf(fmaxf(qb * (1.0f - qb / (float)sn), 1.0f));
+    const int r[4] = {(int)floorf(qt - 4.0f * sdt - 4.0f), (int)ceilf(qt + 4.0f * sdt + 4.0f),
+                      (int)floorf(qb - 4.0f * sdb - 4.0f), (int)ceilf(qb + 4.0f * sdb + 4.0f)};
+    if (tid == 0) {
+        sh_piv[0] = INFINITY;    // top bracket: (piv[1], piv[0]]
+        sh_piv[3] = -INFINITY;   // bottom bracket: [piv[3], piv[2])
+    }
+    if (r[1] > sn || r[2] < 1) return false;   // uniform: depends on n and m only
+    __syncthreads();
+    for (int k = 0; k < 4; ++k) {
+        if (r[k] >= 1 && r[k] <= sn) {
+            find_bin_desc(S, r[k]);
+            __syncthreads();
+            // upper pivots take the upper edge of their bin, lower pivots the lower edge
+            if (tid == 0) sh_piv[k] = lo0 + (float)(S.bin + ((k & 1) ? 0 : 1)) / sc0;
+            __syncthreads();
+        }
+    }
+    const float pt_hi = sh_piv[0], pt_lo = sh_piv[1], pb_hi = sh_piv[2], pb_lo = sh_piv[3];
+    if (!(pt_lo > pb_hi)) return false;   // uniform
+    // 3. one pass: count and sum beyond the brackets, collect inside them
+    if (tid == 0) sh_n[0] = sh_n[1] = 0;
+    __syncthreads();
+    int cnt_t = 0, cnt_b = 0;
+    float sum_t = 0.f, sum_b = 0.f;
+    for (int j0 = 0; j0 < n; j0 += nt) {
+        const int j = j0 + tid;
+        const bool in = j < n;
+        const float v = in ? a[j] : 0.f;
+        const bool above = in && v > pt_hi, below = in && v < pb_lo;
+        const bool in_t = in && !above && v >= pt_lo, in_b = in && !below && v <= pb_hi;
+        cnt_t += above;
+        cnt_b += below;
+        if (above) sum_t += v;
+        if (below) sum_b += v;
+#pragma unroll
+        for (int side = 0; side < 2; ++side) {
+            const bool mine = side == 0 ? in_t : in_b;
+            const unsigned ballot = __ballot_sync(0xffffffffu, mine);
+            if (ballot) {
+                int base = 0;
+                if (lane == 0) base = atomicAdd(&sh_n[side], __popc(ballot));
+                base = __shfl_sync(0xffffffffu, base, 0);
+                const int pos = base + __popc(ballot & ((1u << lane) - 1u));
+                if (mine && pos < kHalf) X.cand[side * kHalf + pos] = v;
+            }
+        }
+    }
+    cnt_t = block_sum_int(S, cnt_t);
+    __syncthreads();
+    cnt_b = block_sum_int(S, cnt_b);
+    __syncthreads();
+    sum_t = block_reduce_f(S, sum_t, 0);
+    sum_b = block_reduce_f(S, sum_b, 0);
+    if (tid == 0) {
+        const int rt = m - cnt_t, rb = m - cnt_b;   // ranks wanted inside the brackets (largest / smallest)
+        sh_ok = sh_n[0] <= kHalf && sh_n[1] <= kHalf && rt >= 1 && rt <= sh_n[0] && rb >= 1 && rb <= sh_n[1];
+        sh_cnt[0] = cnt_t;
+        sh_cnt[1] = cnt_b;
+        sh_sum[0] = sum_t;
+        sh_sum[1] = sum_b;
+    }
+    __syncthreads();
+    if (!sh_ok) return false;
+    // 4. finish exactly inside each bracket
+    for (int side = 0; side < 2; ++side) {
+        const int cn = sh_n[side];
+        const float* c = X.cand + side * kHalf;
+        const int want = m - sh_cnt[side];
+        const int rank_desc = side == 0 ? want : cn - want + 1;
+        const float blo = side == 0 ? pt_lo : pb_lo, bhi = side == 0 ? pt_hi : pb_hi, width = bhi - blo;
+        const bool own = width > 0.f && isfinite(width) && isfinite(blo);
+        SmemSrc csrc{c};
+        block_select_desc(S, csrc, cn, rank_desc, own ? blo : lo0, own ? (float)kBins / width : sc0, status);
+        const uint32_t theta = S.theta;
+        __syncthreads();
+        float part = 0.f;
+        int beyond = 0;   // bracket elements strictly beyond theta on this side
+        for (int j = tid; j < cn; j += nt) {
+            const uint32_t key = ord_key(c[j]);
+            const bool b = side == 0 ? key > theta : key < theta;
+            if (b) {
+                part += c[j];
+                ++beyond;
+            }
+        }
+        const float inner = block_reduce_f(S, part, 0);
+        beyond = block_sum_int(S, beyond);
+        if (tid == 0) sh_res[side] = sh_sum[side] + inner + (float)(want - beyond) * ord_float(theta);
+        __syncthreads();
+    }
+    if (tid == 0) {
+        *top_sum = sh_res[0];
+        *bot_sum = sh_res[1];
+    }
+    __syncthreads();
+    return true;
+}
+
 // Layout of the per-head statistics scratch written by scale_stats_kernel (floats per head).
 constexpr int kHeadStat = 8;   // Delta_s, Delta_e, Delta_c, min s, max s, sum s, unused, unused
 constexpr int kStatThreads = 256;
@@ -506,17 +626,22 @@ __global__ void __launch_bounds__(kStatThreads, 4) scale_stats_kernel(int N, Sco
         const float* ak = k == 0 ? a[0] : (k == 1 ? a[1] : a[2]);
         float gap = 0.f;
         if (rk > 0.f) {
-            float side_sum[2];
-            for (int side = 0; side < 2; ++side) {
-                ScaleSrc src{ak, side == 0 ? 1.f : -1.f};
-                const float lo0 = side == 0 ? lok : -(lok + rk);
-                block_select_bracket(S, X, src, N, (long long)N, m, lo0, (float)kBins / rk, status, &sh_above);
-                __syncthreads();
-                side_sum[side] = sh_above + (float)(m - S.gt) * ord_float(S.theta);
-                __syncthreads();
+            __shared__ float sh_top, sh_bot;
+            if (two_tail_sums(S, X, ak, N, m, lok, (float)kBins / rk, status, &sh_top, &sh_bot)) {
+                gap = (sh_top - sh_bot) / ((float)m * rk);
+            } else {
+                float side_sum[2];
+                for (int side = 0; side < 2; ++side) {
+                    ScaleSrc src{ak, side == 0 ? 1.f : -1.f};
+                    const float lo0 = side == 0 ? lok : -(lok + rk);
+                    block_select_bracket(S, X, src, N, (long long)N, m, lo0, (float)kBins / rk, status, &sh_above);
+                    __syncthreads();
+                    side_sum[side] = sh_above + (float)(m - S.gt) * ord_float(S.theta);
+                    __syncthreads();
+                }
+                // side 1 summed the negated values: top_sum - bot_sum = side_sum[0] + side_sum[1]
+                gap = (side_sum[0] + side_sum[1]) / ((float)m * rk);
             }
-            // side 1 summed the negated values: top_sum - bot_sum = side_sum[0] + side_sum[1]
-            gap = (side_sum[0] + side_sum[1]) / ((float)m * rk);
         }
         if (threadIdx.x == 0) out[k] = gap;
     } else {
