@@ -256,6 +256,16 @@ NKV_API int64_t nkv_launch_count(const nkv_handle* h);
  * either setting. */
 NKV_API int nkv_set_scan_options(nkv_handle* h, int lag, int l2_hints);
 
+/* Choice of the kernel that makes the first key pass of nkv_compress (Sections 2.1-2.3: 1/||k||,
+ * the block sums of normalised keys, and the current-memory anomaly a_c).  NKV_FIRST_PASS_FMA walks
+ * the sliding window with fp32 FMAs.  NKV_FIRST_PASS_TENSOR (bf16 keys, d = 128, W = 64 only) takes
+ * k_hat_i . S_i and ||S_i||^2 as sums over a band of the keys' Gram matrix, which the tensor cores
+ * form, one CTA per head; a request that the inputs do not allow falls back to the FMA kernel.
+ * NKV_FIRST_PASS_AUTO (default) takes whichever measures faster on B200, today the FMA kernel.  The
+ * two forms agree to fp32 rounding. */
+enum { NKV_FIRST_PASS_AUTO = 0, NKV_FIRST_PASS_FMA = 1, NKV_FIRST_PASS_TENSOR = 2 };
+NKV_API int nkv_set_first_pass(nkv_handle* h, int mode);
+
 /*
  * nkv_budget for callers that cannot allocate device memory (the paper has no
  * counterpart: this is a packaging variant of nkv_budget, same arithmetic,

@@ -15,6 +15,7 @@ struct nkv_handle {
     int64_t launches;
     int timing;
     int timing_valid;
+    int first_pass;   // NKV_FIRST_PASS_*: which kernel makes the first key pass
     int scan_lag;     // heads between the two passes of the fused scan (0: use the separate passes)
     int scan_hints;   // L2 eviction hints on the key loads of the fused scan
     cudaEvent_t ev[NKV_NUM_STAGES + 1];
@@ -218,8 +219,9 @@ int nkv_create(nkv_handle** out, int device) {
     h->l2_bytes = prop.l2CacheSize;
     h->scan_lag = 0;   // the separate passes are faster today; see nkv_set_scan_options
     h->scan_hints = 1;
+    h->first_pass = NKV_FIRST_PASS_AUTO;
     if (configure_scan_kernels() != cudaSuccess || configure_stream_kernels() != cudaSuccess ||
-        configure_fused_kernels() != cudaSuccess || configure_select_kernels() != cudaSuccess) {
+        configure_fused_kernels() != cudaSuccess || configure_gram_kernels() != cudaSuccess || configure_select_kernels() != cudaSuccess) {
         delete h;
         return NKV_ERR_CUDA;
     }
@@ -406,8 +408,15 @@ int nkv_compress(nkv_handle* h, const nkv_tensor* K, const nkv_tensor* V, double
         CU(mark());
     } else if (stream_path_supported(sp)) {
         // pass A: norms, block sums and the current-memory anomaly; pass B: the two anchor anomalies
-        CU(launch_stream_a(kv, K->dtype, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm),
-                           at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));
+        // the FMA form measures faster today, so the default choice takes it
+        const bool use_tensor = h->first_pass == NKV_FIRST_PASS_TENSOR && gram_pass_supported(kv, K->dtype, sp);
+        if (use_tensor)
+            CU(launch_gram_pass(kv, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm), at<float>(ws, L.a_raw),
+                                at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));
+        else
+            CU(launch_stream_a(kv, K->dtype, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm),
+                               at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), status, h->sm_count, st,
+                               &h->launches));
         CU(launch_anchor_means(units, N, d, sp, at<float>(ws, L.mu_e), at<float>(ws, L.mu_s), st, &h->launches));
         CU(launch_anchor_norms(units, d, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_s),
                                at<float>(ws, L.inv_e), nullptr, st, &h->launches));
@@ -573,6 +582,12 @@ int nkv_set_scan_options(nkv_handle* h, int lag, int l2_hints) {
     if (!h || lag < 0 || lag > 64) return NKV_ERR_INVALID_ARG;
     h->scan_lag = lag;
     h->scan_hints = l2_hints ? 1 : 0;
+    return NKV_OK;
+}
+
+int nkv_set_first_pass(nkv_handle* h, int mode) {
+    if (!h || mode < NKV_FIRST_PASS_AUTO || mode > NKV_FIRST_PASS_TENSOR) return NKV_ERR_INVALID_ARG;
+    h->first_pass = mode;
     return NKV_OK;
 }
 

@@ -1,0 +1,535 @@
+// First key pass on the tensor cores (bf16 keys, d = 128, window W = 64).
+//
+// What the pass computes (Sections 2.1-2.3): 1/||k_i||, the sums of normalised keys of every episodic
+// block, and the current-memory anomaly a_c(i) = -cos(k_hat_i, mu_c(i)) with its per-head min/max, where
+// mu_c(i) is the mean of the last W normalised keys.  With S_i the sum of that window,
+//     k_hat_i . S_i = sum_{j in window(i)} g_ij          g_ij = k_hat_i . k_hat_j
+//     ||S_i||^2     = sum_{j, l in window(i)} g_jl
+// so both are sums over a band of the Gram matrix of the keys.  The raw Gram entries G_ij = k_i . k_j are
+// products of bf16 numbers summed in fp32, which is what tcgen05.mma does, so the band comes out of the
+// tensor cores at no cost in instruction issue: g_ij = w_i w_j G_ij with w_i = 1/||k_i||.
+//
+// One CTA walks a head front to back in tiles of 128 keys.  Keys are staged by TMA in slabs of 64 rows
+// (128-byte swizzle, two 64-column halves) in a ring of eight slabs, so every key is fetched once.  For
+// tile t the MMA warp forms D = K[tile rows] x K[64 rows before .. 64 rows after]^T (128 x 256, fp32 in
+// tensor memory, double buffered).  Row r of D gives
+//     c_r = sum of g over the 64 columns ending at the diagonal       (= k_hat . S, backward band)
+//     f_r = sum of g over the 64 columns starting at the diagonal     (forward band)
+// and ||S_i||^2 follows from T_i = T_{i-1} + (2 c_i - g_ii) - (2 f_{i-W} - g_{i-W,i-W}), a prefix sum over
+// the tile that restarts every tile from an exact value (the sum of the 64 x 64 Gram block that ends at
+// the previous tile's last row, which is in that tile's D).  The norms and the block sums need the key
+// values themselves and stay on the FMA pipes.
+//
+// The CTA is a pipeline of warp groups, each one tile behind the previous one:
+//     producer (1 thread)  TMA loads of the slabs
+//     norms    (8 warps)   1/||k||, g_ii and the sums of normalised keys, 64 rows ahead of the tile
+//     mma      (1 thread)  the Gram rectangle of the tile
+//     band     (8 warps)   c_r, f_r and the row's part of the next exact restart value from D
+//     scan     (4 warps)   prefix sum, a_c, outputs, min/max
+// Groups hand work to each other through mbarriers; every wait is bounded and a group that gives up
+// records where and leaves, which makes the others give up in turn.
+#include "nkv_sm100.cuh"
+
+namespace nkv {
+
+namespace {
+
+using namespace sm100;
+
+constexpr int kD = 128;                       // head dimension
+constexpr int kTile = 128;                    // keys per tile (rows of D)
+constexpr int kSlabRows = 64;                 // rows per staged slab
+constexpr int kRing = 8;                      // slabs in the ring
+constexpr int kSlabHalfBytes = kSlabRows * 128;             // one 64-column half of a slab
+constexpr int kHalfBytes = kRing * kSlabHalfBytes;          // all slabs of one half are contiguous
+constexpr int kRingBytes = 2 * kHalfBytes;
+constexpr int kBandThreads = 256, kNormThreads = 256, kScanThreads = 128;
+constexpr int kBandWarp0 = 0, kNormWarp0 = 8, kScanWarp0 = 16, kProducerWarp = 20, kMmaWarp = 21;
+constexpr int kThreads = 22 * 32;
+constexpr int kWRing = 2048;                  // per-row scalars kept in rings of 2048 rows
+constexpr int kCfRing = 4;                    // band -> scan hand-over buffers
+constexpr int kWReady = 8;                    // norms -> band hand-over barriers
+constexpr uint32_t kTmemCols = 512;           // two accumulators of 256 columns
+constexpr int kBarNorm = 1, kBarBand = 2, kBarScan = 3;   // named barriers
+
+struct Smem {
+    float pp[2][16 * kD];        // sums of normalised keys of the 16 eight-row segments of a span
+    float w[kWRing];             // 1/||k|| by row (0 outside the head)
+    float g[kWRing];             // g_ii by row
+    float c[kCfRing][kTile];     // backward band sums of a tile
+    float f[kCfRing][kTile];     // forward band sums of a tile
+    float bp[kCfRing][kTile];    // row's share of the Gram block of the tile's last 64 rows
+    float anchor[2];             // exact ||S||^2 at the last row of the previous tile
+    float wtot[2][4];            // per-warp totals of a tile's prefix sum
+    float apart[2][4];           // per-warp parts of the next anchor
+    float red[16];               // min/max reduction at the end of a head
+    uint64_t full[kRing];        // slab landed
+    uint64_t sfree[kRing];       // slab no longer needed (one arrival from the MMAs, one from the norms group)
+    uint64_t tfull[2];           // accumulator written
+    uint64_t tempty[2];          // accumulator read
+    uint64_t wready[kWReady];    // norms of a span written
+    uint64_t cready[kCfRing];    // band sums of a tile written
+    uint64_t cfree[kCfRing];     // band sums of a tile consumed
+    uint32_t tmem_base;
+};
+constexpr size_t kSmemBytes = 1024 + kRingBytes + sizeof(Smem);
+
+// Slab q of a CTA's slab sequence sits at ring position p and is the fc-th use of that position.
+// Positions are handed out so that the two slabs of a tile's own rows are adjacent (even, odd).
+__device__ __forceinline__ void slab_slot(long long q, int& p, uint32_t& fc) {
+    const long long Q = q + 7;
+    p = (int)(Q & 7);
+    fc = (uint32_t)(Q >> 3) - (p != 7 ? 1u : 0u);
+}
+
+// Transposed reduction of V per-lane partial values over a group of L lanes (L, V powers of two, V <= L):
+// afterwards lane l holds in v[0] the complete sum of value l / (L/V).
+template <int V, int L>
+__device__ __forceinline__ void treduce(float* v, int l) {
+    int n = V;
+#pragma unroll
+    for (int o = L / 2; o >= 1; o >>= 1) {
+        if (n > 1) {
+            const int half = n / 2;
+            const bool up = (l & o) != 0;
+#pragma unroll
+            for (int j = 0; j < V / 2; ++j) {
+                if (j < half) {
+                    const float send = up ? v[j] : v[j + half];
+                    const float keep = up ? v[j + half] : v[j];
+                    v[j] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+                }
+            }
+            n = half;
+        } else {
+            v[0] += __shfl_xor_sync(0xffffffffu, v[0], o);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------- producer and MMA
+// TMA producer (one thread): the slabs of every head of this CTA, in order.  Slab lam of a head holds
+// rows [64 (lam - 1), 64 lam); rows outside [0, N) arrive as zeros.
+__device__ void producer_role(const CUtensorMap* tmap, unsigned char* ring, Smem* s, int units, int H, int T,
+                              int* status) {
+    long long q = 0;
+    for (int u = blockIdx.x; u < units; u += gridDim.x) {
+        const int g = u / H, h = u - g * H;
+        for (int lam = 0; lam < 2 * T + 2; ++lam, ++q) {
+            int p;
+            uint32_t fc;
+            slab_slot(q, p, fc);
+            if (fc > 0 && !mbar_wait(&s->sfree[p], (fc - 1) & 1u, status, 701)) return;
+            mbar_expect_tx(&s->full[p], 2 * kSlabHalfBytes);
+            unsigned char* dst = ring + (size_t)p * kSlabHalfBytes;
+            tma_load_4d(dst, tmap, 0, kSlabRows * (lam - 1), h, g, &s->full[p]);
+            tma_load_4d(dst + kHalfBytes, tmap, 64, kSlabRows * (lam - 1), h, g, &s->full[p]);
+        }
+    }
+}
+
+// MMA issuer (one thread).  Tile tau of a head: A = slabs 2 tau + 1, 2 tau + 2 (the tile's rows),
+// B = slabs 2 tau .. 2 tau + 3, four MMAs of N = 64 per 16-wide K step.
+__device__ void mma_role(unsigned char* ring, Smem* s, uint32_t tmem_base, int units, int T, int* status) {
+    constexpr uint32_t idesc = umma_idesc_bf16(kTile, 64);
+    const uint32_t ring_addr = smem_addr(ring);
+    long long hb = 0, gt = 0;
+    for (int u = blockIdx.x; u < units; u += gridDim.x) {
+        for (int tau = 0; tau < T; ++tau, ++gt) {
+            int p;
+            uint32_t fc;
+            for (int lam = tau == 0 ? 0 : 2 * tau + 2; lam <= 2 * tau + 3; ++lam) {
+                slab_slot(hb + lam, p, fc);
+                if (!mbar_wait(&s->full[p], fc & 1u, status, 702)) return;
+            }
+            const int st = (int)(gt & 1);
+            if (!mbar_wait(&s->tempty[st], (uint32_t)(((gt >> 1) & 1) ^ 1), status, 703)) return;
+            tc_fence_after();
+            int pa;
+            slab_slot(hb + 2 * tau + 1, pa, fc);
+#pragma unroll
+            for (int n = 0; n < 4; ++n) {
+                int pb;
+                slab_slot(hb + 2 * tau + n, pb, fc);
+#pragma unroll
+                for (int kk = 0; kk < kD / 16; ++kk) {
+                    const uint32_t koff = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
+                    const uint64_t adesc = umma_desc_sw128(ring_addr + (uint32_t)pa * kSlabHalfBytes + koff);
+                    const uint64_t bdesc = umma_desc_sw128(ring_addr + (uint32_t)pb * kSlabHalfBytes + koff);
+                    umma_bf16(tmem_base + (uint32_t)st * 256u + (uint32_t)n * 64u, adesc, bdesc, idesc, kk > 0);
+                }
+            }
+            umma_commit(&s->tfull[st]);
+            for (int lam = 2 * tau; lam <= (tau == T - 1 ? 2 * tau + 3 : 2 * tau + 1); ++lam) {
+                slab_slot(hb + lam, p, fc);
+                umma_commit(&s->sfree[p]);
+            }
+        }
+        hb += 2 * T + 2;
+    }
+}
+
+// ---------------------------------------------------------------------------- norms group
+// Norms and segment sums of the 128 rows [R1, R1 + 128) held by ring positions p0 (first 64 rows) and
+// p1.  Lane group grp (16 lanes, 8 columns per lane) takes the 8 rows of segment grp.
+__device__ __forceinline__ void span_norms_and_sums(const unsigned char* ring, int p0, int p1, Smem* s, float* pp, int R1,
+                                                    int N, int grp, int l) {
+    F2 acc[4];
+#pragma unroll
+    for (int p = 0; p < 4; ++p) acc[p] = pack2(0.f, 0.f);
+    const int pos = grp < 8 ? p0 : p1;
+    const unsigned char* base = ring + (size_t)(l >> 3) * kHalfBytes + (size_t)pos * kSlabHalfBytes;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        F2 x[4][4];
+        float n2[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int rs = (grp & 7) * 8 + half * 4 + r;   // row inside the slab
+            const uint4 q = *reinterpret_cast<const uint4*>(base + rs * 128 + (((l & 7) ^ (rs & 7)) << 4));
+            unpack_bf16x8(q, x[r]);
+            F2 sq = pack2(0.f, 0.f);
+#pragma unroll
+            for (int p = 0; p < 4; ++p) sq = fma2(x[r][p], x[r][p], sq);
+            n2[r] = hsum2(sq);
+        }
+        treduce<4, 16>(n2, l);
+        // lane l now owns the squared norm of row l / 4 of this half
+        const int row = R1 + grp * 8 + half * 4 + (l >> 2);
+        const bool inside = row >= 0 && row < N;
+        const float inv = inside ? 1.0f / fmaxf(sqrtf(n2[0]), kEps) : 0.f;
+        if ((l & 3) == 0) {
+            s->w[(row + 64) & (kWRing - 1)] = inv;
+            s->g[(row + 64) & (kWRing - 1)] = inv * inv * n2[0];
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const float ir = __shfl_sync(0xffffffffu, inv, r * 4, 16);
+            const F2 ir2 = pack2(ir, ir);
+#pragma unroll
+            for (int p = 0; p < 4; ++p) acc[p] = fma2(x[r][p], ir2, acc[p]);
+        }
+    }
+    float* dst = pp + grp * kD + l * 8;
+    float4 o0, o1;
+    unpack2(acc[0], o0.x, o0.y);
+    unpack2(acc[1], o0.z, o0.w);
+    unpack2(acc[2], o1.x, o1.y);
+    unpack2(acc[3], o1.z, o1.w);
+    *reinterpret_cast<float4*>(dst) = o0;
+    *reinterpret_cast<float4*>(dst + 4) = o1;
+}
+
+// Span tau of a head covers rows [128 tau + 64, 128 tau + 192), tau = -1 .. T-1: always 64 rows ahead of
+// what the band sums of tile tau need.
+__device__ void norms_role(const unsigned char* ring, Smem* s, ScoreParams sp, int units, int N, int T,
+                           float* __restrict__ block_sums, int* status) {
+    const int t = threadIdx.x - kNormWarp0 * 32;
+    const int grp = t >> 4, l = t & 15;
+    const int b = sp.block;
+    long long hb = 0, gs = 0;
+    for (int u = blockIdx.x; u < units; u += gridDim.x) {
+        float run = 0.f;   // running block sum of column t (t < 128)
+        for (int tau = -1; tau < T; ++tau, ++gs) {
+            int p0, p1;
+            uint32_t fc0, fc1;
+            slab_slot(hb + 2 * tau + 2, p0, fc0);
+            slab_slot(hb + 2 * tau + 3, p1, fc1);
+            bool ok = mbar_wait(&s->full[p0], fc0 & 1u, status, 704);
+            ok = ok && mbar_wait(&s->full[p1], fc1 & 1u, status, 704);
+            const int R1 = kTile * tau + 64;
+            float* pp = s->pp[gs & 1];
+            span_norms_and_sums(ring, p0, p1, s, pp, R1, N, grp, l);
+            if (bar_or(kBarNorm, kNormThreads, !ok)) return;
+            if (t == 0) {   // every thread is done with the two slabs and has written its norms
+                mbar_arrive(&s->sfree[p0]);
+                mbar_arrive(&s->sfree[p1]);
+                mbar_arrive(&s->wready[gs & (kWReady - 1)]);
+            }
+            if (t < kD) {
+                // block sums: segments in order, flushed when a segment closes a block or the head
+                for (int sg = 0; sg < 16; ++sg) {
+                    const int row0 = R1 + sg * kSeg;
+                    if (row0 < 0 || row0 >= N) continue;
+                    run += pp[sg * kD + t];
+                    if ((row0 + kSeg) % b == 0 || row0 + kSeg >= N) {
+                        block_sums[((int64_t)u * sp.nblocks + row0 / b) * kD + t] = run;
+                        run = 0.f;
+                    }
+                }
+            }
+        }
+        hb += 2 * T + 2;
+    }
+}
+
+// ---------------------------------------------------------------------------- band group
+// Band sums of one row of D.  The thread's row has its diagonal at column 64 + r.  side 0 sums the 64
+// columns that end at the diagonal, side 1 the 64 columns that start there; both live in three
+// 32-column chunks starting at column `taddr` points to, of which the first and the last are cut by the
+// diagonal: column o of the first chunk counts when o >= thr, column o of the last when o < thr.
+// Returns the three chunk sums, every column weighted by its key's 1/||k||; row0 is the key of the
+// first column.
+__device__ __forceinline__ void band_sums(uint32_t taddr, const float* wring, int row0, int thr, float& X, float& Y,
+                                          float& Z) {
+    const float* wA = wring + ((row0 + 64) & (kWRing - 1));
+    const float* wB = wring + ((row0 + 96) & (kWRing - 1));
+    const float* wC = wring + ((row0 + 128) & (kWRing - 1));
+    X = 0.f;
+    Y = 0.f;
+    Z = 0.f;
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        float a[16], c[16];
+        tmem_ld16(taddr + 16 * hh, a);
+        tmem_ld16(taddr + 64 + 16 * hh, c);
+        tmem_wait_ld();
+#pragma unroll
+        for (int o4 = 0; o4 < 4; ++o4) {
+            const float4 wa = *reinterpret_cast<const float4*>(wA + 16 * hh + 4 * o4);
+            const float4 wc = *reinterpret_cast<const float4*>(wC + 16 * hh + 4 * o4);
+            const float was[4] = {wa.x, wa.y, wa.z, wa.w}, wcs[4] = {wc.x, wc.y, wc.z, wc.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int o = 4 * o4 + e;
+                const bool first = 16 * hh + o >= thr;
+                X = fmaf(first ? a[o] : 0.f, was[e], X);
+                Z = fmaf(first ? 0.f : c[o], wcs[e], Z);
+            }
+        }
+    }
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        float a[16];
+        tmem_ld16(taddr + 32 + 16 * hh, a);
+        tmem_wait_ld();
+#pragma unroll
+        for (int o4 = 0; o4 < 4; ++o4) {
+            const float4 wb = *reinterpret_cast<const float4*>(wB + 16 * hh + 4 * o4);
+            Y = fmaf(a[4 * o4], wb.x, Y);
+            Y = fmaf(a[4 * o4 + 1], wb.y, Y);
+            Y = fmaf(a[4 * o4 + 2], wb.z, Y);
+            Y = fmaf(a[4 * o4 + 3], wb.w, Y);
+        }
+    }
+}
+
+__device__ void band_role(Smem* s, uint32_t tmem_base, int units, int T, int* status) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int q = warp & 3, side = warp >> 2;   // quarter of the tile's rows, backward / forward band
+    const int r = q * 32 + lane;                // row of the tile
+    long long sb = 0, gt = 0;
+    for (int u = blockIdx.x; u < units; u += gridDim.x) {
+        for (int tau = 0; tau < T; ++tau, ++gt) {
+            const long long gs = sb + tau + 1;   // the span that completes this tile's norms
+            const int st = (int)(gt & 1), cb = (int)(gt & (kCfRing - 1));
+            bool ok = mbar_wait(&s->wready[gs & (kWReady - 1)], (uint32_t)((gs >> 3) & 1), status, 705);
+            ok = ok && mbar_wait(&s->cfree[cb], (uint32_t)(((gt >> 2) & 1) ^ 1), status, 706);
+            ok = ok && mbar_wait(&s->tfull[st], (uint32_t)((gt >> 1) & 1), status, 707);
+            tc_fence_after();
+            const int R0 = kTile * tau;
+            const int cA = 32 * q + 64 * side;   // first column of the first chunk
+            const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(st * 256 + cA);
+            float X, Y, Z;
+            band_sums(taddr, s->w, R0 - 64 + cA, lane + (side == 0 ? 1 : 0), X, Y, Z);
+            tc_fence_before();
+            const float wi = s->w[(R0 + r + 64) & (kWRing - 1)];
+            if (side == 0) {
+                s->c[cb][r] = wi * (X + Y + Z);
+                // Gram block of the tile's last 64 rows: columns 128 .. diagonal of rows 64 .. 127
+                s->bp[cb][r] = q == 2 ? wi * Z : q == 3 ? wi * (Y + Z) : 0.f;
+            } else {
+                s->f[cb][r] = wi * (X + Y + Z);
+            }
+            if (bar_or(kBarBand, kBandThreads, !ok)) return;
+            if (tid == 0) {
+                mbar_arrive(&s->tempty[st]);
+                mbar_arrive(&s->cready[cb]);
+            }
+        }
+        sb += T + 1;
+    }
+}
+
+// ---------------------------------------------------------------------------- scan group
+// Thread r owns row r of the tile: T_i = anchor + prefix of (2 c_i - g_ii) - (2 f_{i-64} - g_{i-64,i-64}).
+__device__ void scan_role(Smem* s, int units, int N, int T, float* __restrict__ inv_norm, float* __restrict__ a_raw,
+                          uint32_t* __restrict__ mm, int* status) {
+    const int r = threadIdx.x - kScanWarp0 * 32;
+    const int q = r >> 5, lane = r & 31;
+    long long gt = 0;
+    for (int u = blockIdx.x; u < units; u += gridDim.x) {
+        float lo = INFINITY, hi = -INFINITY;
+        if (r == 0) s->anchor[gt & 1] = 0.f;
+        for (int tau = 0; tau < T; ++tau, ++gt) {
+            const int cb = (int)(gt & (kCfRing - 1)), pb = (int)((gt - 1) & (kCfRing - 1)), par = (int)(gt & 1);
+            const bool ok = mbar_wait(&s->cready[cb], (uint32_t)((gt >> 2) & 1), status, 708);
+            const int R0 = kTile * tau;
+            const float gi = s->g[(R0 + r + 64) & (kWRing - 1)];
+            const float wi = s->w[(R0 + r + 64) & (kWRing - 1)];
+            const float ci = s->c[cb][r];
+            float rem = 0.f;
+            if (r >= 64) rem = 2.f * s->f[cb][r - 64] - s->g[(R0 + r) & (kWRing - 1)];
+            else if (tau > 0) rem = 2.f * s->f[pb][r + 64] - s->g[(R0 + r) & (kWRing - 1)];
+            float x = 2.f * ci - gi - rem;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const float y = __shfl_up_sync(0xffffffffu, x, o);
+                if (lane >= o) x += y;
+            }
+            const float ap = warp_sum(q >= 2 ? 2.f * s->bp[cb][r] - gi : 0.f);
+            if (lane == 31) s->wtot[par][q] = x;
+            if (lane == 0) s->apart[par][q] = ap;
+            if (bar_or(kBarScan, kScanThreads, !ok)) return;
+            // the previous tile's forward sums have been read by now
+            if (r == 0 && gt > 0) mbar_arrive(&s->cfree[pb]);
+            float base = s->anchor[par];
+            for (int w = 0; w < q; ++w) base += s->wtot[par][w];
+            const float Ti = base + x;
+            const int i = R0 + r;
+            if (i < N) {
+                const float a_c = -ci / fmaxf(sqrtf(fmaxf(Ti, 0.f)), kEps) + 0.f;
+                a_raw[((int64_t)u * 3 + 2) * N + i] = a_c;
+                inv_norm[(int64_t)u * N + i] = wi;
+                lo = fminf(lo, a_c);
+                hi = fmaxf(hi, a_c);
+            }
+            if (r == 0) s->anchor[par ^ 1] = s->apart[par][2] + s->apart[par][3];
+        }
+        // ---- per-head min/max of a_c
+        lo = warp_min(lo);
+        hi = warp_max(hi);
+        if (lane == 0) {
+            s->red[2 * q] = lo;
+            s->red[2 * q + 1] = hi;
+        }
+        bar_sync(kBarScan, kScanThreads);
+        if (r == 0) {
+            for (int w = 1; w < 4; ++w) {
+                lo = fminf(lo, s->red[2 * w]);
+                hi = fmaxf(hi, s->red[2 * w + 1]);
+            }
+            if (lo <= hi) {
+                atomicMin(&mm[(int64_t)u * 6 + 4], ord_key(lo));
+                atomicMax(&mm[(int64_t)u * 6 + 5], ord_key(hi));
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+gram_pass_kernel(const __grid_constant__ CUtensorMap tmap, ScoreParams sp, int units, int H, int N,
+                 float* __restrict__ block_sums, float* __restrict__ inv_norm, float* __restrict__ a_raw,
+                 uint32_t* __restrict__ mm, int* status) {
+    extern __shared__ unsigned char smem_raw[];
+    // the swizzle atoms (8 rows x 128 bytes) must start on 1024-byte boundaries
+    unsigned char* ring = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
+    Smem* s = reinterpret_cast<Smem*>(ring + kRingBytes);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int T = (N + kTile - 1) / kTile;
+
+    if (tid == 0) {
+        for (int i = 0; i < kRing; ++i) {
+            mbar_init(&s->full[i], 1);
+            mbar_init(&s->sfree[i], 2);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&s->tfull[i], 1);
+            mbar_init(&s->tempty[i], 1);
+        }
+        for (int i = 0; i < kWReady; ++i) mbar_init(&s->wready[i], 1);
+        for (int i = 0; i < kCfRing; ++i) {
+            mbar_init(&s->cready[i], 1);
+            mbar_init(&s->cfree[i], 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kMmaWarp) tmem_alloc(&s->tmem_base, kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = s->tmem_base;
+
+    if (warp == kProducerWarp) {
+        if (lane == 0) producer_role(&tmap, ring, s, units, H, T, status);
+        __syncwarp();
+    } else if (warp == kMmaWarp) {
+        if (lane == 0) mma_role(ring, s, tmem_base, units, T, status);
+        __syncwarp();
+    } else if (warp >= kScanWarp0) {
+        scan_role(s, units, N, T, inv_norm, a_raw, mm, status);
+    } else if (warp >= kNormWarp0) {
+        norms_role(ring, s, sp, units, N, T, block_sums, status);
+    } else {
+        band_role(s, tmem_base, units, T, status);
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kMmaWarp) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// reset of the per-head min/max keys
+__global__ void gram_init_kernel(int units, uint32_t* mm) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < units * 6) mm[i] = (i & 1) ? 0u : 0xffffffffu;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up once (the library does not link against the driver).
+EncodeTiledFn tensor_map_encoder() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+}  // namespace
+
+cudaError_t configure_gram_kernels() {
+    return cudaFuncSetAttribute(gram_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+}
+
+// bf16 keys of 128 columns, the paper's window of 64, a block size the segment sums can follow, and
+// strides a tensor map accepts (multiples of 16 bytes, base 16-byte aligned).
+bool gram_pass_supported(const TensorView& K, int dtype, const ScoreParams& sp) {
+    if (dtype != NKV_BF16 || K.d != kD || sp.window != 64 || sp.block % kSeg != 0) return false;
+    if (reinterpret_cast<uintptr_t>(K.ptr) % 16 != 0) return false;
+    if (K.stride_h % 8 != 0 || K.stride_g % 8 != 0) return false;
+    if (K.stride_h < (int64_t)K.N * kD || K.stride_g < K.stride_h) return false;
+    return true;
+}
+
+cudaError_t launch_gram_pass(const TensorView& K, int G, const ScoreParams& sp, float* block_sums, float* inv_norm,
+                             float* a_raw, uint32_t* mm, int* status, int sm_count, cudaStream_t stream,
+                             int64_t* launches) {
+    EncodeTiledFn encode = tensor_map_encoder();
+    if (!encode) return cudaErrorNotSupported;
+    const int units = G * K.H;
+    alignas(64) CUtensorMap tmap;
+    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)K.N, (cuuint64_t)K.H, (cuuint64_t)G};
+    const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)K.stride_h * 2, (cuuint64_t)K.stride_g * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)kSlabRows, 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(K.ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
+    gram_init_kernel<<<(units * 6 + 255) / 256, 256, 0, stream>>>(units, mm);
+    ++*launches;
+    const unsigned grid = (unsigned)(units < sm_count ? units : sm_count);
+    gram_pass_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tmap, sp, units, K.H, K.N, block_sums, inv_norm, a_raw, mm,
+                                                             status);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace nkv

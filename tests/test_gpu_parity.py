@@ -177,6 +177,27 @@ def test_fused_compress_end_to_end(N, d, dtype, H, layers, r, scan_lag):
     assert rep.swapped_tokens <= max(2, rep.heads)   # near-tie swaps are rare at fp32 accuracy
 
 
+@pytest.mark.parametrize("N,H,layers,r", [
+    (100, 2, 1, 0.5), (777, 1, 3, 0.9), (2500, 8, 2, 0.95), (4096, 4, 1, 0.75), (8200, 3, 1, 0.75)])
+def test_tensor_core_first_pass_end_to_end(N, H, layers, r):
+    """The first key pass as band sums of the keys' Gram matrix (tcgen05) against the oracle."""
+    K, V = _cache(N, 128, "bf16", H=H, layers=layers)
+    p = nkv.nkv_default_params()
+    ws = nkv.alloc_workspace(K, p)
+    before = nkv.nkv_launch_count()
+    nkv.nkv_set_first_pass("tensor")
+    try:
+        res = nkv.nkv_compress(K, V, r, p, ws=ws, want_a_star=True)
+    finally:
+        nkv.nkv_set_first_pass("auto")
+    assert nkv.nkv_last_device_status(ws) == nkv.NKV_OK
+    assert nkv.nkv_launch_count() > before
+    rep = pr.SwapReport()
+    for g in range(K.shape[0]):
+        pr.check_group_against_oracle(K, V, res, g, r, p, rep)
+    assert rep.swapped_tokens <= max(2, rep.heads)
+
+
 def test_identical_keys_take_the_tie_path():
     """All keys equal: every score is 0 and every selection is decided by position alone."""
     K = torch.ones((1, 2, 3000, 64), dtype=torch.bfloat16, device=DEV)
