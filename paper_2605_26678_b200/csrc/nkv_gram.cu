@@ -82,6 +82,11 @@ __device__ __forceinline__ void slab_slot(long long q, int& p, uint32_t& fc) {
     fc = (uint32_t)(Q >> 3) - (p != 7 ? 1u : 0u);
 }
 
+// The per-row rings (1/||k||, g_ii) are indexed by a row count that keeps running from head to head, so
+// that the first rows of a head never land on entries the last tiles of the previous head still read.
+// A head uses rows -64 .. 128 T + 127.
+__device__ __forceinline__ int ring_advance(int T) { return kTile * (T + 2); }
+
 // Transposed reduction of V per-lane partial values over a group of L lanes (L, V powers of two, V <= L):
 // afterwards lane l holds in v[0] the complete sum of value l / (L/V).
 template <int V, int L>
@@ -173,7 +178,7 @@ __device__ void mma_role(unsigned char* ring, Smem* s, uint32_t tmem_base, int u
 // Norms and segment sums of the 128 rows [R1, R1 + 128) held by ring positions p0 (first 64 rows) and
 // p1.  Lane group grp (16 lanes, 8 columns per lane) takes the 8 rows of segment grp.
 __device__ __forceinline__ void span_norms_and_sums(const unsigned char* ring, int p0, int p1, Smem* s, float* pp, int R1,
-                                                    int N, int grp, int l) {
+                                                    int N, int rb, int grp, int l) {
     F2 acc[4];
 #pragma unroll
     for (int p = 0; p < 4; ++p) acc[p] = pack2(0.f, 0.f);
@@ -199,8 +204,8 @@ __device__ __forceinline__ void span_norms_and_sums(const unsigned char* ring, i
         const bool inside = row >= 0 && row < N;
         const float inv = inside ? 1.0f / fmaxf(sqrtf(n2[0]), kEps) : 0.f;
         if ((l & 3) == 0) {
-            s->w[(row + 64) & (kWRing - 1)] = inv;
-            s->g[(row + 64) & (kWRing - 1)] = inv * inv * n2[0];
+            s->w[(rb + row) & (kWRing - 1)] = inv;
+            s->g[(rb + row) & (kWRing - 1)] = inv * inv * n2[0];
         }
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
@@ -228,8 +233,10 @@ __device__ void norms_role(const unsigned char* ring, Smem* s, ScoreParams sp, i
     const int grp = t >> 4, l = t & 15;
     const int b = sp.block;
     long long hb = 0, gs = 0;
+    int rb = 64;   // ring index of the head's row 0 (see ring_advance)
     for (int u = blockIdx.x; u < units; u += gridDim.x) {
         float run = 0.f;   // running block sum of column t (t < 128)
+        int blk = 0, blk_end = min(b, N);   // block being summed and the row it ends before
         for (int tau = -1; tau < T; ++tau, ++gs) {
             int p0, p1;
             uint32_t fc0, fc1;
@@ -239,7 +246,7 @@ __device__ void norms_role(const unsigned char* ring, Smem* s, ScoreParams sp, i
             ok = ok && mbar_wait(&s->full[p1], fc1 & 1u, status, 704);
             const int R1 = kTile * tau + 64;
             float* pp = s->pp[gs & 1];
-            span_norms_and_sums(ring, p0, p1, s, pp, R1, N, grp, l);
+            span_norms_and_sums(ring, p0, p1, s, pp, R1, N, rb, grp, l);
             if (bar_or(kBarNorm, kNormThreads, !ok)) return;
             if (t == 0) {   // every thread is done with the two slabs and has written its norms
                 mbar_arrive(&s->sfree[p0]);
@@ -248,18 +255,26 @@ __device__ void norms_role(const unsigned char* ring, Smem* s, ScoreParams sp, i
             }
             if (t < kD) {
                 // block sums: segments in order, flushed when a segment closes a block or the head
+                float v[16];
+#pragma unroll
+                for (int sg = 0; sg < 16; ++sg) v[sg] = pp[sg * kD + t];
+#pragma unroll
                 for (int sg = 0; sg < 16; ++sg) {
                     const int row0 = R1 + sg * kSeg;
-                    if (row0 < 0 || row0 >= N) continue;
-                    run += pp[sg * kD + t];
-                    if ((row0 + kSeg) % b == 0 || row0 + kSeg >= N) {
-                        block_sums[((int64_t)u * sp.nblocks + row0 / b) * kD + t] = run;
-                        run = 0.f;
+                    if (row0 >= 0 && row0 < N) {
+                        run += v[sg];
+                        if (row0 + kSeg >= blk_end) {
+                            block_sums[((int64_t)u * sp.nblocks + blk) * kD + t] = run;
+                            run = 0.f;
+                            ++blk;
+                            blk_end = min(blk_end + b, N);
+                        }
                     }
                 }
             }
         }
         hb += 2 * T + 2;
+        rb = (rb + ring_advance(T)) & (kWRing - 1);
     }
 }
 
@@ -268,50 +283,49 @@ __device__ void norms_role(const unsigned char* ring, Smem* s, ScoreParams sp, i
 // columns that end at the diagonal, side 1 the 64 columns that start there; both live in three
 // 32-column chunks starting at column `taddr` points to, of which the first and the last are cut by the
 // diagonal: column o of the first chunk counts when o >= thr, column o of the last when o < thr.
-// Returns the three chunk sums, every column weighted by its key's 1/||k||; row0 is the key of the
-// first column.
+// Returns the three chunk sums, every column weighted by its key's 1/||k||; row0 is the ring index of
+// the first column's key.
 __device__ __forceinline__ void band_sums(uint32_t taddr, const float* wring, int row0, int thr, float& X, float& Y,
                                           float& Z) {
-    const float* wA = wring + ((row0 + 64) & (kWRing - 1));
-    const float* wB = wring + ((row0 + 96) & (kWRing - 1));
-    const float* wC = wring + ((row0 + 128) & (kWRing - 1));
-    X = 0.f;
-    Y = 0.f;
-    Z = 0.f;
-#pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-        float a[16], c[16];
-        tmem_ld16(taddr + 16 * hh, a);
-        tmem_ld16(taddr + 64 + 16 * hh, c);
-        tmem_wait_ld();
+    const float* wA = wring + (row0 & (kWRing - 1));
+    const float* wB = wring + ((row0 + 32) & (kWRing - 1));
+    const float* wC = wring + ((row0 + 64) & (kWRing - 1));
+    // sum of v[o] * w[o] over 16 columns, two accumulators; MODE 0: all, 1: columns >= thr, 2: columns < thr
+    auto dot16 = [&](const float* v, const float* w, int col0, int mode, float& s0, float& s1) {
 #pragma unroll
         for (int o4 = 0; o4 < 4; ++o4) {
-            const float4 wa = *reinterpret_cast<const float4*>(wA + 16 * hh + 4 * o4);
-            const float4 wc = *reinterpret_cast<const float4*>(wC + 16 * hh + 4 * o4);
-            const float was[4] = {wa.x, wa.y, wa.z, wa.w}, wcs[4] = {wc.x, wc.y, wc.z, wc.w};
+            const float4 ww = *reinterpret_cast<const float4*>(w + 4 * o4);
+            const float ws[4] = {ww.x, ww.y, ww.z, ww.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int o = 4 * o4 + e;
-                const bool first = 16 * hh + o >= thr;
-                X = fmaf(first ? a[o] : 0.f, was[e], X);
-                Z = fmaf(first ? 0.f : c[o], wcs[e], Z);
+                const bool keep = mode == 0 || (mode == 1 ? col0 + o >= thr : col0 + o < thr);
+                float& acc = (e & 1) ? s1 : s0;
+                acc = fmaf(keep ? v[o] : 0.f, ws[e], acc);
             }
         }
-    }
-#pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-        float a[16];
-        tmem_ld16(taddr + 32 + 16 * hh, a);
-        tmem_wait_ld();
-#pragma unroll
-        for (int o4 = 0; o4 < 4; ++o4) {
-            const float4 wb = *reinterpret_cast<const float4*>(wB + 16 * hh + 4 * o4);
-            Y = fmaf(a[4 * o4], wb.x, Y);
-            Y = fmaf(a[4 * o4 + 1], wb.y, Y);
-            Y = fmaf(a[4 * o4 + 2], wb.z, Y);
-            Y = fmaf(a[4 * o4 + 3], wb.w, Y);
-        }
-    }
+    };
+    float x0 = 0.f, x1 = 0.f, y0 = 0.f, y1 = 0.f, z0 = 0.f, z1 = 0.f;
+    float p0[16], p1[16], p2[16], p3[16];
+    // the loads of the next pair of 16-column pieces are in flight while the current pair is summed
+    tmem_ld16(taddr, p0);
+    tmem_ld16(taddr + 16, p1);
+    tmem_wait_ld(p0, p1);
+    tmem_ld16(taddr + 32, p2);
+    tmem_ld16(taddr + 48, p3);
+    dot16(p0, wA, 0, 1, x0, x1);
+    dot16(p1, wA + 16, 16, 1, x0, x1);
+    tmem_wait_ld(p2, p3);
+    tmem_ld16(taddr + 64, p0);
+    tmem_ld16(taddr + 80, p1);
+    dot16(p2, wB, 0, 0, y0, y1);
+    dot16(p3, wB + 16, 16, 0, y0, y1);
+    tmem_wait_ld(p0, p1);
+    dot16(p0, wC, 0, 2, z0, z1);
+    dot16(p1, wC + 16, 16, 2, z0, z1);
+    X = x0 + x1;
+    Y = y0 + y1;
+    Z = z0 + z1;
 }
 
 __device__ void band_role(Smem* s, uint32_t tmem_base, int units, int T, int* status) {
@@ -319,6 +333,7 @@ __device__ void band_role(Smem* s, uint32_t tmem_base, int units, int T, int* st
     const int q = warp & 3, side = warp >> 2;   // quarter of the tile's rows, backward / forward band
     const int r = q * 32 + lane;                // row of the tile
     long long sb = 0, gt = 0;
+    int rb = 64;
     for (int u = blockIdx.x; u < units; u += gridDim.x) {
         for (int tau = 0; tau < T; ++tau, ++gt) {
             const long long gs = sb + tau + 1;   // the span that completes this tile's norms
@@ -331,9 +346,9 @@ __device__ void band_role(Smem* s, uint32_t tmem_base, int units, int T, int* st
             const int cA = 32 * q + 64 * side;   // first column of the first chunk
             const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(st * 256 + cA);
             float X, Y, Z;
-            band_sums(taddr, s->w, R0 - 64 + cA, lane + (side == 0 ? 1 : 0), X, Y, Z);
+            band_sums(taddr, s->w, rb + R0 - 64 + cA, lane + (side == 0 ? 1 : 0), X, Y, Z);
             tc_fence_before();
-            const float wi = s->w[(R0 + r + 64) & (kWRing - 1)];
+            const float wi = s->w[(rb + R0 + r) & (kWRing - 1)];
             if (side == 0) {
                 s->c[cb][r] = wi * (X + Y + Z);
                 // Gram block of the tile's last 64 rows: columns 128 .. diagonal of rows 64 .. 127
@@ -348,6 +363,7 @@ __device__ void band_role(Smem* s, uint32_t tmem_base, int units, int T, int* st
             }
         }
         sb += T + 1;
+        rb = (rb + ring_advance(T)) & (kWRing - 1);
     }
 }
 
@@ -358,6 +374,7 @@ __device__ void scan_role(Smem* s, int units, int N, int T, float* __restrict__ 
     const int r = threadIdx.x - kScanWarp0 * 32;
     const int q = r >> 5, lane = r & 31;
     long long gt = 0;
+    int rb = 64;
     for (int u = blockIdx.x; u < units; u += gridDim.x) {
         float lo = INFINITY, hi = -INFINITY;
         if (r == 0) s->anchor[gt & 1] = 0.f;
@@ -365,12 +382,12 @@ __device__ void scan_role(Smem* s, int units, int N, int T, float* __restrict__ 
             const int cb = (int)(gt & (kCfRing - 1)), pb = (int)((gt - 1) & (kCfRing - 1)), par = (int)(gt & 1);
             const bool ok = mbar_wait(&s->cready[cb], (uint32_t)((gt >> 2) & 1), status, 708);
             const int R0 = kTile * tau;
-            const float gi = s->g[(R0 + r + 64) & (kWRing - 1)];
-            const float wi = s->w[(R0 + r + 64) & (kWRing - 1)];
+            const float gi = s->g[(rb + R0 + r) & (kWRing - 1)];
+            const float wi = s->w[(rb + R0 + r) & (kWRing - 1)];
             const float ci = s->c[cb][r];
             float rem = 0.f;
-            if (r >= 64) rem = 2.f * s->f[cb][r - 64] - s->g[(R0 + r) & (kWRing - 1)];
-            else if (tau > 0) rem = 2.f * s->f[pb][r + 64] - s->g[(R0 + r) & (kWRing - 1)];
+            if (r >= 64) rem = 2.f * s->f[cb][r - 64] - s->g[(rb + R0 + r - 64) & (kWRing - 1)];
+            else if (tau > 0) rem = 2.f * s->f[pb][r + 64] - s->g[(rb + R0 + r - 64) & (kWRing - 1)];
             float x = 2.f * ci - gi - rem;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -414,6 +431,7 @@ __device__ void scan_role(Smem* s, int units, int N, int T, float* __restrict__ 
                 atomicMax(&mm[(int64_t)u * 6 + 5], ord_key(hi));
             }
         }
+        rb = (rb + ring_advance(T)) & (kWRing - 1);
     }
 }
 
