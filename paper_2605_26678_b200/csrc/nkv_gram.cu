@@ -176,44 +176,48 @@ __device__ void mma_role(unsigned char* ring, Smem* s, uint32_t tmem_base, int u
 
 // ---------------------------------------------------------------------------- norms group
 // Norms and segment sums of the 128 rows [R1, R1 + 128) held by ring positions p0 (first 64 rows) and
-// p1.  Lane group grp (16 lanes, 8 columns per lane) takes the 8 rows of segment grp.
+// p1.  Lane group grp (16 lanes, 8 columns per lane) takes the 8 rows of segment grp, twice: the rows
+// are cheap to fetch again from shared memory and keeping them would serialise the two halves.
 __device__ __forceinline__ void span_norms_and_sums(const unsigned char* ring, int p0, int p1, Smem* s, float* pp, int R1,
                                                     int N, int rb, int grp, int l) {
+    const int pos = grp < 8 ? p0 : p1;
+    const unsigned char* base = ring + (size_t)(l >> 3) * kHalfBytes + (size_t)pos * kSlabHalfBytes;
+    // first sweep: squared norms of the eight rows (nothing is kept, so the rows overlap in flight)
+    float n2[8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+        const int rs = (grp & 7) * 8 + r;   // row inside the slab
+        const uint4 q = *reinterpret_cast<const uint4*>(base + rs * 128 + (((l & 7) ^ (rs & 7)) << 4));
+        F2 x[4];
+        unpack_bf16x8(q, x);
+        F2 sq = pack2(0.f, 0.f);
+#pragma unroll
+        for (int p = 0; p < 4; ++p) sq = fma2(x[p], x[p], sq);
+        n2[r] = hsum2(sq);
+    }
+    treduce<8, 16>(n2, l);
+    // lane l now owns the squared norm of row l / 2
+    const int row = R1 + grp * 8 + (l >> 1);
+    const bool inside = row >= 0 && row < N;
+    const float inv = inside ? 1.0f / fmaxf(sqrtf(n2[0]), kEps) : 0.f;
+    if ((l & 1) == 0) {
+        s->w[(rb + row) & (kWRing - 1)] = inv;
+        s->g[(rb + row) & (kWRing - 1)] = inv * inv * n2[0];
+    }
+    // second sweep: the rows again, scaled and summed
     F2 acc[4];
 #pragma unroll
     for (int p = 0; p < 4; ++p) acc[p] = pack2(0.f, 0.f);
-    const int pos = grp < 8 ? p0 : p1;
-    const unsigned char* base = ring + (size_t)(l >> 3) * kHalfBytes + (size_t)pos * kSlabHalfBytes;
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
-        F2 x[4][4];
-        float n2[4];
+    for (int r = 0; r < 8; ++r) {
+        const int rs = (grp & 7) * 8 + r;
+        const uint4 q = *reinterpret_cast<const uint4*>(base + rs * 128 + (((l & 7) ^ (rs & 7)) << 4));
+        F2 x[4];
+        unpack_bf16x8(q, x);
+        const float ir = __shfl_sync(0xffffffffu, inv, r * 2, 16);
+        const F2 ir2 = pack2(ir, ir);
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const int rs = (grp & 7) * 8 + half * 4 + r;   // row inside the slab
-            const uint4 q = *reinterpret_cast<const uint4*>(base + rs * 128 + (((l & 7) ^ (rs & 7)) << 4));
-            unpack_bf16x8(q, x[r]);
-            F2 sq = pack2(0.f, 0.f);
-#pragma unroll
-            for (int p = 0; p < 4; ++p) sq = fma2(x[r][p], x[r][p], sq);
-            n2[r] = hsum2(sq);
-        }
-        treduce<4, 16>(n2, l);
-        // lane l now owns the squared norm of row l / 4 of this half
-        const int row = R1 + grp * 8 + half * 4 + (l >> 2);
-        const bool inside = row >= 0 && row < N;
-        const float inv = inside ? 1.0f / fmaxf(sqrtf(n2[0]), kEps) : 0.f;
-        if ((l & 3) == 0) {
-            s->w[(rb + row) & (kWRing - 1)] = inv;
-            s->g[(rb + row) & (kWRing - 1)] = inv * inv * n2[0];
-        }
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const float ir = __shfl_sync(0xffffffffu, inv, r * 4, 16);
-            const F2 ir2 = pack2(ir, ir);
-#pragma unroll
-            for (int p = 0; p < 4; ++p) acc[p] = fma2(x[r][p], ir2, acc[p]);
-        }
+        for (int p = 0; p < 4; ++p) acc[p] = fma2(x[p], ir2, acc[p]);
     }
     float* dst = pp + grp * kD + l * 8;
     float4 o0, o1;
@@ -223,6 +227,18 @@ __device__ __forceinline__ void span_norms_and_sums(const unsigned char* ring, i
     unpack2(acc[3], o1.z, o1.w);
     *reinterpret_cast<float4*>(dst) = o0;
     *reinterpret_cast<float4*>(dst + 4) = o1;
+}
+
+// sum of v[sg] over a <= sg < b (16 segment sums in registers), as a tree
+__device__ __forceinline__ float segment_range_sum(const float* v, int a, int b) {
+    float p[16];
+#pragma unroll
+    for (int sg = 0; sg < 16; ++sg) p[sg] = (sg >= a && sg < b) ? v[sg] : 0.f;
+#pragma unroll
+    for (int w = 8; w >= 1; w >>= 1)
+#pragma unroll
+        for (int sg = 0; sg < w; ++sg) p[sg] += p[sg + w];
+    return p[0];
 }
 
 // Span tau of a head covers rows [128 tau + 64, 128 tau + 192), tau = -1 .. T-1: always 64 rows ahead of
@@ -254,23 +270,22 @@ __device__ void norms_role(const unsigned char* ring, Smem* s, ScoreParams sp, i
                 mbar_arrive(&s->wready[gs & (kWReady - 1)]);
             }
             if (t < kD) {
-                // block sums: segments in order, flushed when a segment closes a block or the head
+                // block sums of column t: a block that closes inside this span is written out, the
+                // rest of the span starts the next one (rows outside the head are zeros)
                 float v[16];
 #pragma unroll
                 for (int sg = 0; sg < 16; ++sg) v[sg] = pp[sg * kD + t];
-#pragma unroll
-                for (int sg = 0; sg < 16; ++sg) {
-                    const int row0 = R1 + sg * kSeg;
-                    if (row0 >= 0 && row0 < N) {
-                        run += v[sg];
-                        if (row0 + kSeg >= blk_end) {
-                            block_sums[((int64_t)u * sp.nblocks + blk) * kD + t] = run;
-                            run = 0.f;
-                            ++blk;
-                            blk_end = min(blk_end + b, N);
-                        }
-                    }
+                int s0 = 0;   // first segment not yet added
+                while (blk < sp.nblocks && blk_end <= R1 + kTile) {
+                    const int s1 = (blk_end - R1 + kSeg - 1) / kSeg;   // segments [s0, s1) close the block
+                    run += segment_range_sum(v, s0, s1);
+                    block_sums[((int64_t)u * sp.nblocks + blk) * kD + t] = run;
+                    run = 0.f;
+                    ++blk;
+                    blk_end = min(blk_end + b, N);
+                    s0 = s1;
                 }
+                run += segment_range_sum(v, s0, 16);
             }
         }
         hb += 2 * T + 2;
