@@ -305,39 +305,51 @@ __device__ __forceinline__ void band_sums(uint32_t taddr, const float* wring, in
     const float* wA = wring + (row0 & (kWRing - 1));
     const float* wB = wring + ((row0 + 32) & (kWRing - 1));
     const float* wC = wring + ((row0 + 64) & (kWRing - 1));
-    // sum of v[o] * w[o] over 16 columns, two accumulators; MODE 0: all, 1: columns >= thr, 2: columns < thr
-    auto dot16 = [&](const float* v, const float* w, int col0, int mode, float& s0, float& s1) {
+    // 16 columns of the first chunk and the 16 columns 64 further on share the diagonal test: column o
+    // of the first chunk counts exactly when column o of the last one does not
+    auto cut16 = [&](const float* a, const float* c, const float* wa, const float* wc, int col0, float& xa, float& xb,
+                     float& za, float& zb) {
 #pragma unroll
         for (int o4 = 0; o4 < 4; ++o4) {
-            const float4 ww = *reinterpret_cast<const float4*>(w + 4 * o4);
-            const float ws[4] = {ww.x, ww.y, ww.z, ww.w};
+            const float4 fa = *reinterpret_cast<const float4*>(wa + 4 * o4);
+            const float4 fc = *reinterpret_cast<const float4*>(wc + 4 * o4);
+            const float was[4] = {fa.x, fa.y, fa.z, fa.w}, wcs[4] = {fc.x, fc.y, fc.z, fc.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int o = 4 * o4 + e;
-                const bool keep = mode == 0 || (mode == 1 ? col0 + o >= thr : col0 + o < thr);
-                float& acc = (e & 1) ? s1 : s0;
-                acc = fmaf(keep ? v[o] : 0.f, ws[e], acc);
+                float& x = (e & 1) ? xb : xa;
+                float& z = (e & 1) ? zb : za;
+                if (col0 + o >= thr) x = fmaf(a[o], was[e], x);
+                else z = fmaf(c[o], wcs[e], z);
             }
+        }
+    };
+    auto dot16 = [&](const float* v, const float* w, float& s0, float& s1) {
+#pragma unroll
+        for (int o4 = 0; o4 < 4; ++o4) {
+            const float4 ww = *reinterpret_cast<const float4*>(w + 4 * o4);
+            s0 = fmaf(v[4 * o4], ww.x, s0);
+            s1 = fmaf(v[4 * o4 + 1], ww.y, s1);
+            s0 = fmaf(v[4 * o4 + 2], ww.z, s0);
+            s1 = fmaf(v[4 * o4 + 3], ww.w, s1);
         }
     };
     float x0 = 0.f, x1 = 0.f, y0 = 0.f, y1 = 0.f, z0 = 0.f, z1 = 0.f;
     float p0[16], p1[16], p2[16], p3[16];
     // the loads of the next pair of 16-column pieces are in flight while the current pair is summed
     tmem_ld16(taddr, p0);
-    tmem_ld16(taddr + 16, p1);
+    tmem_ld16(taddr + 64, p1);
     tmem_wait_ld(p0, p1);
-    tmem_ld16(taddr + 32, p2);
-    tmem_ld16(taddr + 48, p3);
-    dot16(p0, wA, 0, 1, x0, x1);
-    dot16(p1, wA + 16, 16, 1, x0, x1);
+    tmem_ld16(taddr + 16, p2);
+    tmem_ld16(taddr + 80, p3);
+    cut16(p0, p1, wA, wC, 0, x0, x1, z0, z1);
     tmem_wait_ld(p2, p3);
-    tmem_ld16(taddr + 64, p0);
-    tmem_ld16(taddr + 80, p1);
-    dot16(p2, wB, 0, 0, y0, y1);
-    dot16(p3, wB + 16, 16, 0, y0, y1);
+    tmem_ld16(taddr + 32, p0);
+    tmem_ld16(taddr + 48, p1);
+    cut16(p2, p3, wA + 16, wC + 16, 16, x0, x1, z0, z1);
     tmem_wait_ld(p0, p1);
-    dot16(p0, wC, 0, 2, z0, z1);
-    dot16(p1, wC + 16, 16, 2, z0, z1);
+    dot16(p0, wB, y0, y1);
+    dot16(p1, wB + 16, y0, y1);
     X = x0 + x1;
     Y = y0 + y1;
     Z = z0 + z1;
