@@ -261,8 +261,9 @@ NKV_API int nkv_set_scan_options(nkv_handle* h, int lag, int l2_hints);
  * the sliding window with fp32 FMAs.  NKV_FIRST_PASS_TENSOR (bf16 keys, d = 128, W = 64 only) takes
  * k_hat_i . S_i and ||S_i||^2 as sums over a band of the keys' Gram matrix, which the tensor cores
  * form, one CTA per head; a request that the inputs do not allow falls back to the FMA kernel.
- * NKV_FIRST_PASS_AUTO (default) takes whichever measures faster on B200, today the FMA kernel.  The
- * two forms agree to fp32 rounding. */
+ * NKV_FIRST_PASS_AUTO (default) takes the tensor form when the inputs allow it and the call has at
+ * least half as many heads as the GPU has SMs, else the FMA kernel.  The two forms agree to fp32
+ * rounding. */
 enum { NKV_FIRST_PASS_AUTO = 0, NKV_FIRST_PASS_FMA = 1, NKV_FIRST_PASS_TENSOR = 2 };
 NKV_API int nkv_set_first_pass(nkv_handle* h, int mode);
 

@@ -408,8 +408,12 @@ int nkv_compress(nkv_handle* h, const nkv_tensor* K, const nkv_tensor* V, double
         CU(mark());
     } else if (stream_path_supported(sp)) {
         // pass A: norms, block sums and the current-memory anomaly; pass B: the two anchor anomalies
-        // the FMA form measures faster today, so the default choice takes it
-        const bool use_tensor = h->first_pass == NKV_FIRST_PASS_TENSOR && gram_pass_supported(kv, K->dtype, sp);
+        // the tensor-core form walks whole heads, one CTA each: by default it runs when there are enough
+        // heads to fill the GPU
+        const bool tensor_ok = gram_pass_supported(kv, K->dtype, sp);
+        const bool use_tensor = h->first_pass == NKV_FIRST_PASS_TENSOR
+                                    ? tensor_ok
+                                    : h->first_pass == NKV_FIRST_PASS_AUTO && tensor_ok && 2 * units >= h->sm_count;
         if (use_tensor)
             CU(launch_gram_pass(kv, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm), at<float>(ws, L.a_raw),
                                 at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));

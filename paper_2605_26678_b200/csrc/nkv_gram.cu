@@ -41,7 +41,9 @@ constexpr int kTile = 128;                    // keys per tile (rows of D)
 constexpr int kSlabRows = 64;                 // rows per staged slab
 constexpr int kRing = 8;                      // slabs in the ring
 constexpr int kSlabHalfBytes = kSlabRows * 128;             // one 64-column half of a slab
-constexpr int kHalfBytes = kRing * kSlabHalfBytes;          // all slabs of one half are contiguous
+constexpr int kHalfBytes = (kRing + 1) * kSlabHalfBytes;    // all slabs of one half are contiguous; position 8 is a
+                                                            // second copy of position 0, so that a pair of slabs
+                                                            // that starts at position 7 is contiguous too
 constexpr int kRingBytes = 2 * kHalfBytes;
 constexpr int kBandThreads = 256, kNormThreads = 256, kScanThreads = 128;
 constexpr int kBandWarp0 = 0, kNormWarp0 = 8, kScanWarp0 = 16, kProducerWarp = 20, kMmaWarp = 21;
@@ -125,18 +127,20 @@ __device__ void producer_role(const CUtensorMap* tmap, unsigned char* ring, Smem
             uint32_t fc;
             slab_slot(q, p, fc);
             if (fc > 0 && !mbar_wait(&s->sfree[p], (fc - 1) & 1u, status, 701)) return;
-            mbar_expect_tx(&s->full[p], 2 * kSlabHalfBytes);
-            unsigned char* dst = ring + (size_t)p * kSlabHalfBytes;
-            tma_load_4d(dst, tmap, 0, kSlabRows * (lam - 1), h, g, &s->full[p]);
-            tma_load_4d(dst + kHalfBytes, tmap, 64, kSlabRows * (lam - 1), h, g, &s->full[p]);
+            mbar_expect_tx(&s->full[p], (p == 0 ? 4 : 2) * kSlabHalfBytes);
+            for (int copy = 0; copy < (p == 0 ? 2 : 1); ++copy) {
+                unsigned char* dst = ring + (size_t)(copy ? kRing : p) * kSlabHalfBytes;
+                tma_load_4d(dst, tmap, 0, kSlabRows * (lam - 1), h, g, &s->full[p]);
+                tma_load_4d(dst + kHalfBytes, tmap, 64, kSlabRows * (lam - 1), h, g, &s->full[p]);
+            }
         }
     }
 }
 
 // MMA issuer (one thread).  Tile tau of a head: A = slabs 2 tau + 1, 2 tau + 2 (the tile's rows),
-// B = slabs 2 tau .. 2 tau + 3, four MMAs of N = 64 per 16-wide K step.
+// B = slabs 2 tau .. 2 tau + 3 as two pairs, two MMAs of N = 128 per 16-wide K step.
 __device__ void mma_role(unsigned char* ring, Smem* s, uint32_t tmem_base, int units, int T, int* status) {
-    constexpr uint32_t idesc = umma_idesc_bf16(kTile, 64);
+    constexpr uint32_t idesc = umma_idesc_bf16(kTile, 128);
     const uint32_t ring_addr = smem_addr(ring);
     long long hb = 0, gt = 0;
     for (int u = blockIdx.x; u < units; u += gridDim.x) {
@@ -153,15 +157,15 @@ __device__ void mma_role(unsigned char* ring, Smem* s, uint32_t tmem_base, int u
             int pa;
             slab_slot(hb + 2 * tau + 1, pa, fc);
 #pragma unroll
-            for (int n = 0; n < 4; ++n) {
-                int pb;
-                slab_slot(hb + 2 * tau + n, pb, fc);
+            for (int n = 0; n < 2; ++n) {
+                int pb;   // odd; the slab after position 7 is read from the copy at position 8
+                slab_slot(hb + 2 * tau + 2 * n, pb, fc);
 #pragma unroll
                 for (int kk = 0; kk < kD / 16; ++kk) {
                     const uint32_t koff = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
                     const uint64_t adesc = umma_desc_sw128(ring_addr + (uint32_t)pa * kSlabHalfBytes + koff);
                     const uint64_t bdesc = umma_desc_sw128(ring_addr + (uint32_t)pb * kSlabHalfBytes + koff);
-                    umma_bf16(tmem_base + (uint32_t)st * 256u + (uint32_t)n * 64u, adesc, bdesc, idesc, kk > 0);
+                    umma_bf16(tmem_base + (uint32_t)st * 256u + (uint32_t)n * 128u, adesc, bdesc, idesc, kk > 0);
                 }
             }
             umma_commit(&s->tfull[st]);
