@@ -256,16 +256,19 @@ NKV_API int64_t nkv_launch_count(const nkv_handle* h);
  * either setting. */
 NKV_API int nkv_set_scan_options(nkv_handle* h, int lag, int l2_hints);
 
-/* Choice of the kernel that makes the first key pass of nkv_compress (Sections 2.1-2.3: 1/||k||,
- * the block sums of normalised keys, and the current-memory anomaly a_c).  NKV_FIRST_PASS_FMA walks
- * the sliding window with fp32 FMAs.  NKV_FIRST_PASS_TENSOR (bf16 keys, d = 128, W = 64 only) takes
- * k_hat_i . S_i and ||S_i||^2 as sums over a band of the keys' Gram matrix, which the tensor cores
- * form, one CTA per head; a request that the inputs do not allow falls back to the FMA kernel.
- * NKV_FIRST_PASS_AUTO (default) takes the tensor form when the inputs allow it and the call has at
- * least half as many heads as the GPU has SMs, else the FMA kernel.  The two forms agree to fp32
- * rounding. */
-enum { NKV_FIRST_PASS_AUTO = 0, NKV_FIRST_PASS_FMA = 1, NKV_FIRST_PASS_TENSOR = 2 };
-NKV_API int nkv_set_first_pass(nkv_handle* h, int mode);
+/* Choice of the kernels that make the two key passes of nkv_compress (Sections 2.1-2.3).  The first
+ * pass yields 1/||k||, the block sums of normalised keys and the current-memory anomaly a_c; the
+ * second the anomalies a_s and a_e against the global and block anchors.
+ * NKV_KEY_PASS_FMA does both with fp32 FMAs on staged key tiles (any supported dtype and d).
+ * NKV_KEY_PASS_TENSOR (bf16 keys, d = 128) forms on the tensor cores what is a contraction: in the
+ * first pass (W = 64 only, one CTA per head) k_hat_i . S_i and ||S_i||^2 as sums over a band of the
+ * keys' Gram matrix, in the second pass the dots of the keys with the anchors, the fp32 anchors split
+ * three ways into bf16.  A pass whose inputs do not allow the tensor form runs the FMA kernel.
+ * NKV_KEY_PASS_AUTO (default) takes the tensor form of the second pass whenever it is allowed, and of
+ * the first pass when in addition the call has at least half as many heads as the GPU has SMs.
+ * The forms agree to fp32 rounding. */
+enum { NKV_KEY_PASS_AUTO = 0, NKV_KEY_PASS_FMA = 1, NKV_KEY_PASS_TENSOR = 2 };
+NKV_API int nkv_set_key_passes(nkv_handle* h, int mode);
 
 /*
  * nkv_budget for callers that cannot allocate device memory (the paper has no

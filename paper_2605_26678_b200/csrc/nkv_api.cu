@@ -15,7 +15,7 @@ struct nkv_handle {
     int64_t launches;
     int timing;
     int timing_valid;
-    int first_pass;   // NKV_FIRST_PASS_*: which kernel makes the first key pass
+    int key_pass;     // NKV_KEY_PASS_*: which kernels make the two key passes
     int scan_lag;     // heads between the two passes of the fused scan (0: use the separate passes)
     int scan_hints;   // L2 eviction hints on the key loads of the fused scan
     cudaEvent_t ev[NKV_NUM_STAGES + 1];
@@ -219,9 +219,9 @@ int nkv_create(nkv_handle** out, int device) {
     h->l2_bytes = prop.l2CacheSize;
     h->scan_lag = 0;   // the separate passes are faster today; see nkv_set_scan_options
     h->scan_hints = 1;
-    h->first_pass = NKV_FIRST_PASS_AUTO;
+    h->key_pass = NKV_KEY_PASS_AUTO;
     if (configure_scan_kernels() != cudaSuccess || configure_stream_kernels() != cudaSuccess ||
-        configure_fused_kernels() != cudaSuccess || configure_gram_kernels() != cudaSuccess || configure_select_kernels() != cudaSuccess) {
+        configure_fused_kernels() != cudaSuccess || configure_gram_kernels() != cudaSuccess || configure_dots_kernels() != cudaSuccess || configure_select_kernels() != cudaSuccess) {
         delete h;
         return NKV_ERR_CUDA;
     }
@@ -411,9 +411,9 @@ int nkv_compress(nkv_handle* h, const nkv_tensor* K, const nkv_tensor* V, double
         // the tensor-core form walks whole heads, one CTA each: by default it runs when there are enough
         // heads to fill the GPU
         const bool tensor_ok = gram_pass_supported(kv, K->dtype, sp);
-        const bool use_tensor = h->first_pass == NKV_FIRST_PASS_TENSOR
+        const bool use_tensor = h->key_pass == NKV_KEY_PASS_TENSOR
                                     ? tensor_ok
-                                    : h->first_pass == NKV_FIRST_PASS_AUTO && tensor_ok && 2 * units >= h->sm_count;
+                                    : h->key_pass == NKV_KEY_PASS_AUTO && tensor_ok && 2 * units >= h->sm_count;
         if (use_tensor)
             CU(launch_gram_pass(kv, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm), at<float>(ws, L.a_raw),
                                 at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));
@@ -425,9 +425,15 @@ int nkv_compress(nkv_handle* h, const nkv_tensor* K, const nkv_tensor* V, double
         CU(launch_anchor_norms(units, d, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_s),
                                at<float>(ws, L.inv_e), nullptr, st, &h->launches));
         CU(mark());
-        CU(launch_stream_b(kv, K->dtype, G, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e),
-                           at<float>(ws, L.inv_norm), at<float>(ws, L.inv_s), at<float>(ws, L.inv_e),
-                           at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));
+        if (h->key_pass != NKV_KEY_PASS_FMA && anchor_dots_supported(kv, K->dtype, sp))
+            CU(launch_anchor_dots(kv, G, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm),
+                                  at<float>(ws, L.inv_s), at<float>(ws, L.inv_e), at<float>(ws, L.a_raw),
+                                  at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));
+        else
+            CU(launch_stream_b(kv, K->dtype, G, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e),
+                               at<float>(ws, L.inv_norm), at<float>(ws, L.inv_s), at<float>(ws, L.inv_e),
+                               at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), status, h->sm_count, st,
+                               &h->launches));
     } else {
         CU(launch_anchor_sums(kv, K->dtype, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm), st,
                               &h->launches));
@@ -589,9 +595,9 @@ int nkv_set_scan_options(nkv_handle* h, int lag, int l2_hints) {
     return NKV_OK;
 }
 
-int nkv_set_first_pass(nkv_handle* h, int mode) {
-    if (!h || mode < NKV_FIRST_PASS_AUTO || mode > NKV_FIRST_PASS_TENSOR) return NKV_ERR_INVALID_ARG;
-    h->first_pass = mode;
+int nkv_set_key_passes(nkv_handle* h, int mode) {
+    if (!h || mode < NKV_KEY_PASS_AUTO || mode > NKV_KEY_PASS_TENSOR) return NKV_ERR_INVALID_ARG;
+    h->key_pass = mode;
     return NKV_OK;
 }
 

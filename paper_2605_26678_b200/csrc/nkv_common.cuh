@@ -139,6 +139,12 @@ cudaError_t configure_gram_kernels();
 cudaError_t launch_gram_pass(const TensorView& K, int G, const ScoreParams& sp, float* block_sums, float* inv_norm,
                              float* a_raw, uint32_t* mm, int* status, int sm_count, cudaStream_t stream,
                              int64_t* launches);
+// second key pass on the tensor cores (bf16 keys, d = 128): same outputs as launch_stream_b
+bool anchor_dots_supported(const TensorView& K, int dtype, const ScoreParams& sp);
+cudaError_t configure_dots_kernels();
+cudaError_t launch_anchor_dots(const TensorView& K, int G, const ScoreParams& sp, const float* mu_s, const float* mu_e,
+                               const float* inv_norm, const float* inv_s, const float* inv_e, float* a_raw,
+                               uint32_t* mm, int* status, int sm_count, cudaStream_t stream, int64_t* launches);
 // fused two-pass scan (one persistent kernel; the second pass reads the keys from L2)
 bool fused_scan_supported(const ScoreParams& sp, int dtype, int d);
 size_t fused_ctrl_bytes(int64_t units);

@@ -1,0 +1,280 @@
+// Second key pass on the tensor cores (bf16 keys, d = 128): a_s(i) = -cos(k_hat_i, mu_s) and
+// a_e(i) = -cos(k_hat_i, mu_e(block of i)) with their per-head min/max (Section 2.3).
+//
+// The dots of 128 keys with the anchors are one skinny product [128 x d] x [d x 16] per tile.  The fp32
+// anchors enter as three bf16 columns each (hi + mid + lo carries all 24 mantissa bits; products of bf16
+// numbers are exact in fp32 and tcgen05.mma accumulates in fp32), so a tile's right-hand side is
+//     columns 0..2  mu_s        3..5  mu_e of the block the tile starts in        6..8  mu_e of the next block
+// (a tile of 128 keys touches at most two blocks because a block has at least 128 keys).  Key tiles are
+// staged by TMA (128-byte swizzle) several tiles ahead; the tensor core reads them from shared memory
+// directly, so the SM issues a few dozen instructions per tile and the pass runs at the speed of the
+// copy.  Warp roles: TMA producer, MMA issuer, four warps that build the right-hand sides, four warps
+// that turn the accumulator into scores.  Every wait is bounded.
+#include "nkv_sm100.cuh"
+
+namespace nkv {
+
+namespace {
+
+using namespace sm100;
+
+constexpr int kD = 128;
+constexpr int kTile = 128;                        // keys per tile
+constexpr int kSlots = 5;                         // key tiles staged at once
+constexpr int kTileHalfBytes = kTile * 128;       // one 64-column half of a tile
+constexpr int kTileBytes = 2 * kTileHalfBytes;
+constexpr int kRhsHalfBytes = 16 * 128;           // 16 right-hand-side rows of 64 columns
+constexpr int kRhsBytes = 2 * kRhsHalfBytes;
+constexpr int kStages = 4;                        // accumulators of 32 columns (16 used)
+constexpr uint32_t kTmemCols = 128;
+constexpr int kPrepWarp0 = 0, kEpiWarp0 = 4, kProducerWarp = 8, kMmaWarp = 9;
+constexpr int kThreads = 10 * 32;
+
+struct Smem {
+    uint64_t full[kSlots];      // key tile landed
+    uint64_t rready[kSlots];    // right-hand side written (one arrival per building warp)
+    uint64_t kfree[kSlots];     // tile and right-hand side consumed by the MMAs
+    uint64_t tfull[kStages];    // accumulator written
+    uint64_t tempty[kStages];   // accumulator read (one arrival per reading warp)
+    uint32_t tmem_base;
+};
+constexpr size_t kSmemBytes = 1024 + (size_t)kSlots * (kTileBytes + kRhsBytes) + sizeof(Smem);
+
+struct TileRange {
+    long long first, last;      // this CTA's tiles [first, last)
+    int tiles_per_unit;
+};
+__device__ __forceinline__ TileRange my_tiles(int units, int N) {
+    TileRange r;
+    r.tiles_per_unit = (N + kTile - 1) / kTile;
+    const long long total = (long long)units * r.tiles_per_unit;
+    r.first = total * blockIdx.x / gridDim.x;
+    r.last = total * (blockIdx.x + 1) / gridDim.x;
+    return r;
+}
+
+// ---------------------------------------------------------------------------- roles
+__device__ void dots_producer(const CUtensorMap* tmap, unsigned char* tiles, Smem* s, TileRange tr, int H, int* status) {
+    long long n = 0;
+    for (long long t = tr.first; t < tr.last; ++t, ++n) {
+        const int slot = (int)(n % kSlots);
+        const long long fill = n / kSlots;
+        if (fill > 0 && !mbar_wait(&s->kfree[slot], (uint32_t)((fill - 1) & 1), status, 711)) return;
+        const int u = (int)(t / tr.tiles_per_unit);
+        const int i0 = (int)(t - (long long)u * tr.tiles_per_unit) * kTile;
+        const int g = u / H, h = u - g * H;
+        unsigned char* dst = tiles + (size_t)slot * kTileBytes;
+        mbar_expect_tx(&s->full[slot], kTileBytes);
+        tma_load_4d(dst, tmap, 0, i0, h, g, &s->full[slot]);
+        tma_load_4d(dst + kTileHalfBytes, tmap, 64, i0, h, g, &s->full[slot]);
+    }
+}
+
+__device__ void dots_mma(unsigned char* tiles, unsigned char* rhs, Smem* s, uint32_t tmem_base, TileRange tr,
+                         int* status) {
+    constexpr uint32_t idesc = umma_idesc_bf16(kTile, 16);
+    const uint32_t tiles_addr = smem_addr(tiles), rhs_addr = smem_addr(rhs);
+    long long n = 0;
+    for (long long t = tr.first; t < tr.last; ++t, ++n) {
+        const int slot = (int)(n % kSlots), stage = (int)(n % kStages);
+        const uint32_t fpar = (uint32_t)((n / kSlots) & 1), upar = (uint32_t)((n / kStages) & 1);
+        if (!mbar_wait(&s->full[slot], fpar, status, 712)) return;
+        if (!mbar_wait(&s->rready[slot], fpar, status, 713)) return;
+        if (!mbar_wait(&s->tempty[stage], upar ^ 1u, status, 714)) return;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < kD / 16; ++kk) {
+            const uint32_t a = tiles_addr + (uint32_t)slot * kTileBytes + (uint32_t)(kk >> 2) * kTileHalfBytes +
+                               (uint32_t)(kk & 3) * 32u;
+            const uint32_t b = rhs_addr + (uint32_t)slot * kRhsBytes + (uint32_t)(kk >> 2) * kRhsHalfBytes +
+                               (uint32_t)(kk & 3) * 32u;
+            umma_bf16(tmem_base + (uint32_t)stage * 32u, umma_desc_sw128(a), umma_desc_sw128(b), idesc, kk > 0);
+        }
+        umma_commit(&s->tfull[stage]);
+        umma_commit(&s->kfree[slot]);
+    }
+}
+
+// Thread k writes column k of the nine right-hand-side rows of every tile (rows 9..15 stay zero).
+__device__ void dots_prep(unsigned char* rhs, Smem* s, ScoreParams sp, TileRange tr, const float* __restrict__ mu_s,
+                          const float* __restrict__ mu_e, int* status) {
+    const int k = threadIdx.x - kPrepWarp0 * 32, lane = k & 31;
+    const int half = k >> 6, kk = k & 63;
+    long long n = 0;
+    for (long long t = tr.first; t < tr.last; ++t, ++n) {
+        const int slot = (int)(n % kSlots);
+        const long long fill = n / kSlots;
+        if (fill > 0 && !mbar_wait(&s->kfree[slot], (uint32_t)((fill - 1) & 1), status, 715)) return;
+        const int u = (int)(t / tr.tiles_per_unit);
+        const int i0 = (int)(t - (long long)u * tr.tiles_per_unit) * kTile;
+        const int blk0 = i0 / sp.block;
+        float v[3];
+        v[0] = mu_s[(int64_t)u * kD + k];
+        v[1] = mu_e[((int64_t)u * sp.nblocks + blk0) * kD + k];
+        v[2] = blk0 + 1 < sp.nblocks ? mu_e[((int64_t)u * sp.nblocks + blk0 + 1) * kD + k] : 0.f;
+        unsigned char* base = rhs + (size_t)slot * kRhsBytes + (size_t)half * kRhsHalfBytes + (kk & 7) * 2;
+#pragma unroll
+        for (int a = 0; a < 3; ++a) {
+            const __nv_bfloat16 hi = __float2bfloat16_rn(v[a]);
+            const float r1 = v[a] - __bfloat162float(hi);
+            const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+            const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+            const __nv_bfloat16 part[3] = {hi, mid, lo};
+#pragma unroll
+            for (int j = 0; j < 3; ++j) {
+                const int row = 3 * a + j;   // row of the right-hand side, 8-row groups 1024 bytes apart
+                *reinterpret_cast<__nv_bfloat16*>(base + (row >> 3) * 1024 + (row & 7) * 128 +
+                                                  ((((kk >> 3) ^ (row & 7))) << 4)) = part[j];
+            }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads these writes
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s->rready[slot]);
+    }
+}
+
+// Thread r reads row r of the accumulator: the key's dots with mu_s and with the two candidate mu_e.
+__device__ void dots_epilogue(Smem* s, uint32_t tmem_base, ScoreParams sp, TileRange tr, int N,
+                              const float* __restrict__ inv_norm, const float* __restrict__ inv_s,
+                              const float* __restrict__ inv_e, float* __restrict__ a_raw, uint32_t* __restrict__ mm,
+                              int* status) {
+    const int r = threadIdx.x - kEpiWarp0 * 32, q = r >> 5, lane = r & 31;
+    int cur_u = -1;
+    float rs = 0.f;
+    float lo_s = INFINITY, hi_s = -INFINITY, lo_e = INFINITY, hi_e = -INFINITY;
+    auto flush = [&]() {   // the warp's min/max of the head it has been working on
+        if (cur_u < 0) return;
+        lo_s = warp_min(lo_s);
+        hi_s = warp_max(hi_s);
+        lo_e = warp_min(lo_e);
+        hi_e = warp_max(hi_e);
+        if (lane == 0 && lo_s <= hi_s) {
+            atomicMin(&mm[(int64_t)cur_u * 6 + 0], ord_key(lo_s));
+            atomicMax(&mm[(int64_t)cur_u * 6 + 1], ord_key(hi_s));
+            atomicMin(&mm[(int64_t)cur_u * 6 + 2], ord_key(lo_e));
+            atomicMax(&mm[(int64_t)cur_u * 6 + 3], ord_key(hi_e));
+        }
+        lo_s = lo_e = INFINITY;
+        hi_s = hi_e = -INFINITY;
+    };
+    long long n = 0;
+    for (long long t = tr.first; t < tr.last; ++t, ++n) {
+        const int stage = (int)(n % kStages);
+        const int u = (int)(t / tr.tiles_per_unit);
+        const int i0 = (int)(t - (long long)u * tr.tiles_per_unit) * kTile;
+        if (u != cur_u) {
+            flush();
+            cur_u = u;
+            rs = inv_s[u];
+        }
+        const int blk0 = i0 / sp.block;
+        const int i = i0 + r;
+        const bool second = i >= (blk0 + 1) * sp.block;   // the key lies in the block after the tile's first
+        const int blk = min(blk0 + (second ? 1 : 0), sp.nblocks - 1);
+        const float inv_i = i < N ? inv_norm[(int64_t)u * N + i] : 0.f;
+        const float re = inv_e[(int64_t)u * sp.nblocks + blk];
+        if (!mbar_wait(&s->tfull[stage], (uint32_t)((n / kStages) & 1), status, 716)) return;
+        tc_fence_after();
+        float d[16];
+        tmem_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)stage * 32u, d);
+        tmem_wait_ld(d);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s->tempty[stage]);
+        const float ds = d[0] + d[1] + d[2];
+        const float de = second ? d[6] + d[7] + d[8] : d[3] + d[4] + d[5];
+        const float a_s = -(ds * inv_i) * rs + 0.f;
+        const float a_e = -(de * inv_i) * re + 0.f;
+        if (i < N) {
+            a_raw[((int64_t)u * 3 + 0) * N + i] = a_s;
+            a_raw[((int64_t)u * 3 + 1) * N + i] = a_e;
+            lo_s = fminf(lo_s, a_s);
+            hi_s = fmaxf(hi_s, a_s);
+            lo_e = fminf(lo_e, a_e);
+            hi_e = fmaxf(hi_e, a_e);
+        }
+    }
+    flush();
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+anchor_dots_kernel(const __grid_constant__ CUtensorMap tmap, ScoreParams sp, int units, int H, int N,
+                   const float* __restrict__ mu_s, const float* __restrict__ mu_e, const float* __restrict__ inv_norm,
+                   const float* __restrict__ inv_s, const float* __restrict__ inv_e, float* __restrict__ a_raw,
+                   uint32_t* __restrict__ mm, int* status) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* tiles = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
+    unsigned char* rhs = tiles + (size_t)kSlots * kTileBytes;
+    Smem* s = reinterpret_cast<Smem*>(rhs + (size_t)kSlots * kRhsBytes);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const TileRange tr = my_tiles(units, N);
+
+    if (tid == 0) {
+        for (int i = 0; i < kSlots; ++i) {
+            mbar_init(&s->full[i], 1);
+            mbar_init(&s->rready[i], 4);
+            mbar_init(&s->kfree[i], 1);
+        }
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(&s->tfull[i], 1);
+            mbar_init(&s->tempty[i], 4);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int i = tid; i < kSlots * kRhsBytes / 16; i += kThreads) reinterpret_cast<uint4*>(rhs)[i] = make_uint4(0, 0, 0, 0);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    if (warp == kMmaWarp) tmem_alloc(&s->tmem_base, kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = s->tmem_base;
+
+    if (warp == kProducerWarp) {
+        if (lane == 0) dots_producer(&tmap, tiles, s, tr, H, status);
+        __syncwarp();
+    } else if (warp == kMmaWarp) {
+        if (lane == 0) dots_mma(tiles, rhs, s, tmem_base, tr, status);
+        __syncwarp();
+    } else if (warp >= kEpiWarp0) {
+        dots_epilogue(s, tmem_base, sp, tr, N, inv_norm, inv_s, inv_e, a_raw, mm, status);
+    } else {
+        dots_prep(rhs, s, sp, tr, mu_s, mu_e, status);
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kMmaWarp) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+}  // namespace
+
+cudaError_t configure_dots_kernels() {
+    return cudaFuncSetAttribute(anchor_dots_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+}
+
+// Same input conditions as the tensor-core first pass, and blocks of at least 128 keys (a tile of 128
+// keys then touches at most two blocks).
+bool anchor_dots_supported(const TensorView& K, int dtype, const ScoreParams& sp) {
+    if (dtype != NKV_BF16 || K.d != kD || sp.block < kTile) return false;
+    if (reinterpret_cast<uintptr_t>(K.ptr) % 16 != 0) return false;
+    if (K.stride_h % 8 != 0 || K.stride_g % 8 != 0) return false;
+    if (K.stride_h < (int64_t)K.N * kD || K.stride_g < K.stride_h) return false;
+    return true;
+}
+
+cudaError_t launch_anchor_dots(const TensorView& K, int G, const ScoreParams& sp, const float* mu_s, const float* mu_e,
+                               const float* inv_norm, const float* inv_s, const float* inv_e, float* a_raw,
+                               uint32_t* mm, int* status, int sm_count, cudaStream_t stream, int64_t* launches) {
+    CUtensorMap tmap;
+    cudaError_t e = encode_key_map(K, G, kTile, &tmap);
+    if (e != cudaSuccess) return e;
+    const int units = G * K.H;
+    const long long total = (long long)units * ((K.N + kTile - 1) / kTile);
+    const unsigned grid = (unsigned)(total < sm_count ? total : sm_count);
+    anchor_dots_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tmap, sp, units, K.H, K.N, mu_s, mu_e, inv_norm, inv_s,
+                                                               inv_e, a_raw, mm, status);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace nkv

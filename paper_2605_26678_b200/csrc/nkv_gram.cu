@@ -524,6 +524,10 @@ __global__ void gram_init_kernel(int units, uint32_t* mm) {
     if (i < units * 6) mm[i] = (i & 1) ? 0u : 0xffffffffu;
 }
 
+}  // namespace
+
+namespace {
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -543,6 +547,21 @@ EncodeTiledFn tensor_map_encoder() {
 
 }  // namespace
 
+// Tensor map of the keys [G][H][N][128] bf16 for boxes of 64 columns x box_rows rows, 128-byte swizzle.
+cudaError_t encode_key_map(const TensorView& K, int G, int box_rows, CUtensorMap* out) {
+    EncodeTiledFn encode = tensor_map_encoder();
+    if (!encode) return cudaErrorNotSupported;
+    const cuuint64_t dims[4] = {(cuuint64_t)K.d, (cuuint64_t)K.N, (cuuint64_t)K.H, (cuuint64_t)G};
+    const cuuint64_t strides[3] = {(cuuint64_t)K.d * 2, (cuuint64_t)K.stride_h * 2, (cuuint64_t)K.stride_g * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(K.ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
+    return cudaSuccess;
+}
+
 cudaError_t configure_gram_kernels() {
     return cudaFuncSetAttribute(gram_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
 }
@@ -560,18 +579,10 @@ bool gram_pass_supported(const TensorView& K, int dtype, const ScoreParams& sp) 
 cudaError_t launch_gram_pass(const TensorView& K, int G, const ScoreParams& sp, float* block_sums, float* inv_norm,
                              float* a_raw, uint32_t* mm, int* status, int sm_count, cudaStream_t stream,
                              int64_t* launches) {
-    EncodeTiledFn encode = tensor_map_encoder();
-    if (!encode) return cudaErrorNotSupported;
     const int units = G * K.H;
-    alignas(64) CUtensorMap tmap;
-    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)K.N, (cuuint64_t)K.H, (cuuint64_t)G};
-    const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)K.stride_h * 2, (cuuint64_t)K.stride_g * 2};
-    const cuuint32_t box[4] = {64, (cuuint32_t)kSlabRows, 1, 1};
-    const cuuint32_t estr[4] = {1, 1, 1, 1};
-    if (encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(K.ptr), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return cudaErrorInvalidValue;
+    CUtensorMap tmap;
+    cudaError_t e = encode_key_map(K, G, kSlabRows, &tmap);
+    if (e != cudaSuccess) return e;
     gram_init_kernel<<<(units * 6 + 255) / 256, 256, 0, stream>>>(units, mm);
     ++*launches;
     const unsigned grid = (unsigned)(units < sm_count ? units : sm_count);

@@ -7,6 +7,10 @@
 #include "nkv_common.cuh"
 
 namespace nkv {
+
+// Tensor map of bf16 keys [G][H][N][128] for boxes of 64 columns x box_rows rows, 128-byte swizzle (host).
+cudaError_t encode_key_map(const TensorView& K, int G, int box_rows, CUtensorMap* out);
+
 namespace sm100 {
 
 constexpr uint32_t kSpinLimit = 1u << 22;
@@ -117,6 +121,13 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
 __device__ __forceinline__ void tmem_wait_ld(float* a, float* b) {
     asm volatile("tcgen05.wait::ld.sync.aligned;"
                  : "+f"(a[0]), "+f"(a[1]), "+f"(a[2]), "+f"(a[3]), "+f"(a[4]), "+f"(a[5]), "+f"(a[6]), "+f"(a[7]), "+f"(a[8]), "+f"(a[9]), "+f"(a[10]), "+f"(a[11]), "+f"(a[12]), "+f"(a[13]), "+f"(a[14]), "+f"(a[15]), "+f"(b[0]), "+f"(b[1]), "+f"(b[2]), "+f"(b[3]), "+f"(b[4]), "+f"(b[5]), "+f"(b[6]), "+f"(b[7]), "+f"(b[8]), "+f"(b[9]), "+f"(b[10]), "+f"(b[11]), "+f"(b[12]), "+f"(b[13]), "+f"(b[14]), "+f"(b[15])
+                 :
+                 : "memory");
+}
+
+__device__ __forceinline__ void tmem_wait_ld(float* a) {   // the same for one group of 16 values
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+f"(a[0]), "+f"(a[1]), "+f"(a[2]), "+f"(a[3]), "+f"(a[4]), "+f"(a[5]), "+f"(a[6]), "+f"(a[7]), "+f"(a[8]), "+f"(a[9]), "+f"(a[10]), "+f"(a[11]), "+f"(a[12]), "+f"(a[13]), "+f"(a[14]), "+f"(a[15])
                  :
                  : "memory");
 }

@@ -36,7 +36,7 @@ EXPORTS = (
     "nkv_keep_per_head", "nkv_safeguard_count", "nkv_top_count", "nkv_create", "nkv_destroy",
     "nkv_workspace_bytes", "nkv_anchors", "nkv_score", "nkv_budget", "nkv_select", "nkv_compact",
     "nkv_compress", "nkv_host_staging_bytes", "nkv_compress_host", "nkv_last_device_status",
-    "nkv_set_timing", "nkv_get_stage_ms", "nkv_launch_count", "nkv_budget_static", "nkv_set_scan_options", "nkv_set_first_pass",
+    "nkv_set_timing", "nkv_get_stage_ms", "nkv_launch_count", "nkv_budget_static", "nkv_set_scan_options", "nkv_set_key_passes",
 )
 
 
@@ -112,7 +112,7 @@ def load_library():
     L.nkv_launch_count.argtypes = [vp]
     L.nkv_launch_count.restype = i64
     L.nkv_set_scan_options.argtypes = [vp, ctypes.c_int, ctypes.c_int]
-    L.nkv_set_first_pass.argtypes = [vp, ctypes.c_int]
+    L.nkv_set_key_passes.argtypes = [vp, ctypes.c_int]
     L.nkv_budget_static.argtypes = [vp, i64, i64, i64, dbl, pp, vp, vp]
     _lib = L
     return L
@@ -420,13 +420,13 @@ def nkv_launch_count(h: Optional[Handle] = None) -> int:
     return int(h.lib.nkv_launch_count(h.h))
 
 
-FIRST_PASS = {"auto": 0, "fma": 1, "tensor": 2}
+KEY_PASS = {"auto": 0, "fma": 1, "tensor": 2}
 
 
-def nkv_set_first_pass(mode: str = "auto", h: Optional[Handle] = None) -> None:
-    """Kernel of the first key pass: "auto", "fma" or "tensor" (bf16, d = 128 only); see nkv.h."""
+def nkv_set_key_passes(mode: str = "auto", h: Optional[Handle] = None) -> None:
+    """Kernels of the two key passes: "auto", "fma" or "tensor" (bf16, d = 128 only); see nkv.h."""
     h = h or handle()
-    _check(h.lib.nkv_set_first_pass(h.h, FIRST_PASS[mode]), "nkv_set_first_pass")
+    _check(h.lib.nkv_set_key_passes(h.h, KEY_PASS[mode]), "nkv_set_key_passes")
 
 
 def nkv_set_scan_options(lag: int = 0, l2_hints: bool = True, h: Optional[Handle] = None) -> None:

@@ -179,17 +179,19 @@ def test_fused_compress_end_to_end(N, d, dtype, H, layers, r, scan_lag):
 
 @pytest.mark.parametrize("N,H,layers,r", [
     (100, 2, 1, 0.5), (777, 1, 3, 0.9), (2500, 8, 2, 0.95), (4096, 4, 1, 0.75), (8200, 3, 1, 0.75)])
-def test_tensor_core_first_pass_end_to_end(N, H, layers, r):
-    """The first key pass as band sums of the keys' Gram matrix (tcgen05) against the oracle."""
+@pytest.mark.parametrize("mode", ["tensor", "fma"])
+def test_key_pass_kernels_end_to_end(N, H, layers, r, mode):
+    """Both key passes on the tensor cores (tcgen05: band sums of the keys' Gram matrix, dots with the
+    split anchors) and both as FMA kernels, each against the oracle."""
     K, V = _cache(N, 128, "bf16", H=H, layers=layers)
     p = nkv.nkv_default_params()
     ws = nkv.alloc_workspace(K, p)
     before = nkv.nkv_launch_count()
-    nkv.nkv_set_first_pass("tensor")
+    nkv.nkv_set_key_passes(mode)
     try:
         res = nkv.nkv_compress(K, V, r, p, ws=ws, want_a_star=True)
     finally:
-        nkv.nkv_set_first_pass("auto")
+        nkv.nkv_set_key_passes("auto")
     assert nkv.nkv_last_device_status(ws) == nkv.NKV_OK
     assert nkv.nkv_launch_count() > before
     rep = pr.SwapReport()
