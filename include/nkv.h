@@ -265,7 +265,8 @@ NKV_API int nkv_set_scan_options(nkv_handle* h, int lag, int l2_hints);
  * keys' Gram matrix, in the second pass the dots of the keys with the anchors, the fp32 anchors split
  * three ways into bf16.  A pass whose inputs do not allow the tensor form runs the FMA kernel.
  * NKV_KEY_PASS_AUTO (default) takes the tensor form of the second pass whenever it is allowed, and of
- * the first pass when in addition the call has at least half as many heads as the GPU has SMs.
+ * the first pass when in addition the call's heads, dealt one per SM, keep at least 85 % of the SMs
+ * busy over the rounds that takes.
  * The forms agree to fp32 rounding. */
 enum { NKV_KEY_PASS_AUTO = 0, NKV_KEY_PASS_FMA = 1, NKV_KEY_PASS_TENSOR = 2 };
 NKV_API int nkv_set_key_passes(nkv_handle* h, int mode);

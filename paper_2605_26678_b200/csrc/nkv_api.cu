@@ -408,12 +408,14 @@ int nkv_compress(nkv_handle* h, const nkv_tensor* K, const nkv_tensor* V, double
         CU(mark());
     } else if (stream_path_supported(sp)) {
         // pass A: norms, block sums and the current-memory anomaly; pass B: the two anchor anomalies
-        // the tensor-core form walks whole heads, one CTA each: by default it runs when there are enough
-        // heads to fill the GPU
+        // the tensor-core form walks whole heads, one CTA each: by default it runs when the heads fill
+        // the SMs to at least 85 % over its waves (below that the FMA form, which splits heads, is faster)
         const bool tensor_ok = gram_pass_supported(kv, K->dtype, sp);
+        const int waves = (units + h->sm_count - 1) / h->sm_count;
+        const bool fills = (double)units >= 0.85 * (double)waves * (double)h->sm_count;
         const bool use_tensor = h->key_pass == NKV_KEY_PASS_TENSOR
                                     ? tensor_ok
-                                    : h->key_pass == NKV_KEY_PASS_AUTO && tensor_ok && 2 * units >= h->sm_count;
+                                    : h->key_pass == NKV_KEY_PASS_AUTO && tensor_ok && fills;
         if (use_tensor)
             CU(launch_gram_pass(kv, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm), at<float>(ws, L.a_raw),
                                 at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));
