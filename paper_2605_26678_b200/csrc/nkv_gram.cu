@@ -572,8 +572,9 @@ bool gram_pass_supported(const TensorView& K, int dtype, const ScoreParams& sp) 
     if (dtype != NKV_BF16 || K.d != kD || sp.window != 64 || sp.block % kSeg != 0) return false;
     if (reinterpret_cast<uintptr_t>(K.ptr) % 16 != 0) return false;
     if (K.stride_h % 8 != 0 || K.stride_g % 8 != 0) return false;
-    if (K.stride_h < (int64_t)K.N * kD || K.stride_g < K.stride_h) return false;
-    return true;
+    if (K.stride_h < (int64_t)K.N * kD || K.stride_g < (int64_t)K.N * kD) return false;
+    CUtensorMap probe;   // the driver has the last word on what a tensor map can describe
+    return encode_key_map(K, 1, kSlabRows, &probe) == cudaSuccess;
 }
 
 cudaError_t launch_gram_pass(const TensorView& K, int G, const ScoreParams& sp, float* block_sums, float* inv_norm,
