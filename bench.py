@@ -39,7 +39,7 @@ DEFAULT_RATIO = 0.75
 # DRAM bytes per key (dram__bytes_read.sum + dram__bytes_write.sum of one launch / keys of the launch)
 # from the ncu capture summarised in profiles/ (cfg2, bf16, d = 128; traffic grows with the number of
 # keys).  Only kernels unchanged since their capture are listed.
-NCU_DRAM_BYTES_PER_KEY = {("anchors", "bf16", 128): (604.030976e6 + 23.657728e6) / 2359296}
+NCU_DRAM_BYTES_PER_KEY = {("anchors", "bf16", 128): (604.278784e6 + 23.610624e6) / 2359296}
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
@@ -57,6 +57,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--scan-lag", type=int, default=None, help="heads between the two key passes (library default if unset)")
     ap.add_argument("--scan-hints", type=int, default=1, help="L2 eviction hints on the key loads (0/1)")
+    ap.add_argument("--key-passes", default="auto", choices=["auto", "fma", "tensor"],
+                    help="kernels of the two key passes (library default: auto)")
     return ap.parse_args()
 
 
@@ -250,6 +252,7 @@ def run_nkv(args, cfg, r):
     h = nkv.handle(local)
     if args.scan_lag is not None:
         nkv.nkv_set_scan_options(args.scan_lag, bool(args.scan_hints), h)
+    nkv.nkv_set_key_passes(args.key_passes, h)
 
     def step():
         nkv.nkv_compress(K, V, r, params, out=out, ws=ws, h=h)
@@ -340,6 +343,7 @@ def run_nkv(args, cfg, r):
                        "keys_per_step_per_gpu": cfg.keys, "kv_bytes_per_gpu": cfg.kv_bytes(),
                        "l2": "inputs (%.1f GB) are far larger than the 126 MB L2; no flush needed" % (
                            cfg.kv_bytes() / 1e9) if cfg.kv_bytes() > 1e9 else "inputs fit L2: warm-cache number",
+                       "key_passes": args.key_passes,
                        "parallelism": "independent sequences per GPU (replicas), no collective"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "pipeline": pipeline,
             "cpu_baseline": cpu,
