@@ -163,7 +163,6 @@ struct Geo {
     static constexpr int kSegs = kRows / kSeg;
     static constexpr int kThreads = kSegs * kL;                // compute threads: one lane group per staged segment
     static constexpr size_t kTileBytes = (size_t)kRows * kRowBytes;
-    static constexpr size_t kSmem = 2 * kTileBytes + (size_t)kSegs * D * 4 + (size_t)kRows * 4 + 128;
     static_assert(kChunks >= 1 && kThreads % 32 == 0 && kThreads + 32 <= 1024, "bad geometry");
 
     __device__ __forceinline__ static int col0(int l, int j) { return (l + kL * j) * kPerChunk; }

@@ -46,7 +46,7 @@ constexpr int kHalfBytes = (kRing + 1) * kSlabHalfBytes;    // all slabs of one 
                                                             // that starts at position 7 is contiguous too
 constexpr int kRingBytes = 2 * kHalfBytes;
 constexpr int kBandThreads = 256, kNormThreads = 256, kScanThreads = 128;
-constexpr int kBandWarp0 = 0, kNormWarp0 = 8, kScanWarp0 = 16, kProducerWarp = 20, kMmaWarp = 21;
+constexpr int kNormWarp0 = 8, kScanWarp0 = 16, kProducerWarp = 20, kMmaWarp = 21;
 constexpr int kThreads = 22 * 32;
 constexpr int kWRing = 2048;                  // per-row scalars kept in rings of 2048 rows
 constexpr int kCfRing = 4;                    // band -> scan hand-over buffers

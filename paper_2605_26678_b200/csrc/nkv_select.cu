@@ -489,7 +489,17 @@ __device__ bool two_tail_sums(SelectShared& S, BracketShared<CAP>& X, const floa
     const int positions = min(max(n / 8, kSampleMin), kSampleMax);
     for (int b = tid; b < kBins; b += nt) S.hist[b] = 0;
     __syncthreads();
-    for (int i = tid; i < positions; i += nt) atomicAdd(&S.hist[bin_of(a[(int)(((long long)i * n) / positions)], lo0, sc0)], 1);
+    for (int i0 = 0; i0 < positions; i0 += 4 * nt) {   // four loads in flight per thread
+        float sv[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int i = i0 + k * nt + tid;
+            sv[k] = i < positions ? a[(int)(((long long)i * n) / positions)] : 0.f;
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (i0 + k * nt + tid < positions) atomicAdd(&S.hist[bin_of(sv[k], lo0, sc0)], 1);
+    }
     __syncthreads();
     const int sn = positions;
     // 2. four pivots: ranks (counted from the top) around m and around n - m + 1
@@ -519,10 +529,15 @@ __device__ bool two_tail_sums(SelectShared& S, BracketShared<CAP>& X, const floa
     __syncthreads();
     int cnt_t = 0, cnt_b = 0;
     float sum_t = 0.f, sum_b = 0.f;
-    for (int j0 = 0; j0 < n; j0 += nt) {
-        const int j = j0 + tid;
+    for (int jb = 0; jb < n; jb += 4 * nt) {   // four loads in flight per thread
+      float vv[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) vv[k] = jb + k * nt + tid < n ? a[jb + k * nt + tid] : 0.f;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int j = jb + k * nt + tid;
         const bool in = j < n;
-        const float v = in ? a[j] : 0.f;
+        const float v = vv[k];
         const bool above = in && v > pt_hi, below = in && v < pb_lo;
         const bool in_t = in && !above && v >= pt_lo, in_b = in && !below && v <= pb_hi;
         cnt_t += above;
@@ -541,6 +556,7 @@ __device__ bool two_tail_sums(SelectShared& S, BracketShared<CAP>& X, const floa
                 if (mine && pos < kHalf) X.cand[side * kHalf + pos] = v;
             }
         }
+      }
     }
     cnt_t = block_sum_int(S, cnt_t);
     __syncthreads();

@@ -569,207 +569,6 @@ stream_b_kernel(TensorView K, ScoreParams sp, int units, const float* __restrict
     }
 }
 
-// ============================================================================================
-// stream_b on tensor cores (bf16 keys, episodic block a multiple of 16, at most four blocks per tile)
-// ============================================================================================
-// The two dots of every key against mu_s and mu_e are a skinny matrix product [16 keys x d] x [d x 8].
-// The fp32 anchors are split three ways into bf16 (hi + mid + lo keeps all 24 mantissa bits); products
-// of bf16 numbers are exact in fp32 and the accumulation is fp32, so each result is an fp32 dot product
-// up to summation order.  Right-hand-side columns: 0..2 = mu_s hi/mid/lo, 3..5 = mu_e hi/mid/lo, 6..7 = 0.
-// The contraction index may be visited in any order, so lane (g, t) of a warp takes the 16-byte chunks
-// t, t+4, ... of rows g and g+8 straight from the staged tile and the right-hand side uses that order.
-template <int D, int TILE>
-struct BMmaCfg {
-    static constexpr int kRowBytes = D * 2;
-    static constexpr int kThreads = 512;
-    static constexpr int kWarps = kThreads / 32;
-    static constexpr int kIters = (TILE / 16 + kWarps - 1) / kWarps;
-    static constexpr size_t kTileBytes = (size_t)TILE * kRowBytes;
-    static constexpr size_t kRhsBytes = (size_t)4 * 8 * D * 2;           // [4 blocks][8 columns][D] bf16
-    static constexpr int kBufs = 3;   // two tiles in flight while one is consumed: the pass is a pure stream
-    static constexpr size_t kSmem = kBufs * kTileBytes + kRhsBytes + 8 * 4 + 64 * 4 + 64;
-};
-
-template <int D, int TILE>
-__global__ void __launch_bounds__(BMmaCfg<D, TILE>::kThreads, 1)
-stream_b_mma_kernel(TensorView K, ScoreParams sp, int units, const float* __restrict__ mu_s,
-                    const float* __restrict__ mu_e, const float* __restrict__ inv_norm,
-                    const float* __restrict__ inv_s, const float* __restrict__ inv_e, float* __restrict__ a_raw,
-                    uint32_t* __restrict__ mm, int* status) {
-    using C = BMmaCfg<D, TILE>;
-    constexpr int kCh = D / 32;   // 16-byte chunks per lane and row
-    extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char* tiles = smem;
-    __nv_bfloat16* rhs = reinterpret_cast<__nv_bfloat16*>(smem + C::kBufs * C::kTileBytes);
-    float* scal = reinterpret_cast<float*>(smem + C::kBufs * C::kTileBytes + C::kRhsBytes);   // [0] 1/|mu_s|, [1..4] 1/|mu_e|
-    float* red = scal + 8;
-    uint64_t* full = reinterpret_cast<uint64_t*>(red + 64);
-
-    const int N = K.N, b = sp.block, nb = sp.nblocks;
-    const int tiles_per_unit = (N + TILE - 1) / TILE;
-    const long long total = (long long)units * tiles_per_unit;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-
-    if (tid == 0) {
-        for (int i = 0; i < C::kBufs; ++i) mbar_init(&full[i], 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-
-    auto issue = [&](long long tt, int buf) {
-        const int u = (int)(tt / tiles_per_unit);
-        const int i0 = (int)(tt - (long long)u * tiles_per_unit) * TILE;
-        const int gg = u / K.H, h = u % K.H;
-        const unsigned char* src = reinterpret_cast<const unsigned char*>(K.ptr) +
-                                   ((int64_t)gg * K.stride_g + (int64_t)h * K.stride_h) * 2 + (int64_t)i0 * C::kRowBytes;
-        const uint32_t bytes = (uint32_t)(min(N, i0 + TILE) - i0) * C::kRowBytes;
-        unsigned char* dst = tiles + (size_t)buf * C::kTileBytes;
-        fence_async_smem();
-        mbar_expect_tx(&full[buf], bytes);
-        for (uint32_t off = 0; off < bytes; off += 16384u)
-            bulk_load(dst + off, src + off, min(16384u, bytes - off), &full[buf]);
-    };
-
-    // anchors of a tile, one column per thread (threads < D), fetched one iteration ahead
-    struct Anchors {
-        float ms, me[4], sc;
-    };
-    auto load_anchors = [&](long long t2, Anchors& an) {
-        const int u2 = (int)(t2 / tiles_per_unit);
-        const int blk2 = ((int)(t2 - (long long)u2 * tiles_per_unit) * TILE) / b;
-        const int n2 = min(nb - blk2, TILE / b);
-        an.ms = mu_s[(int64_t)u2 * D + tid];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) an.me[q] = q < n2 ? mu_e[((int64_t)u2 * nb + blk2 + q) * D + tid] : 0.f;
-        an.sc = tid == 0 ? inv_s[u2] : (tid <= n2 ? inv_e[(int64_t)u2 * nb + blk2 + tid - 1] : 0.f);
-    };
-    uint32_t* keys = reinterpret_cast<uint32_t*>(red);   // [2][4] ordered min/max keys of the tile in flight
-    if (tid < 8) keys[tid] = (tid & 1) ? 0u : 0xffffffffu;
-
-    long long tt = blockIdx.x;
-    if (tid == 0) {
-        if (tt < total) issue(tt, 0);
-        if (tt + gridDim.x < total) issue(tt + gridDim.x, 1);
-    }
-    Anchors cur_an;
-    if (tt < total && tid < D) load_anchors(tt, cur_an);
-    int it = 0;
-    for (; tt < total; tt += gridDim.x, ++it) {
-        const int buf = it % C::kBufs;
-        const long long tn = tt + gridDim.x;
-        // the buffer of the tile before this one was released by the barrier that ended it
-        if (tt + 2LL * gridDim.x < total && tid == 0) issue(tt + 2LL * gridDim.x, (it + 2) % C::kBufs);
-        const int u = (int)(tt / tiles_per_unit);
-        const int i0 = (int)(tt - (long long)u * tiles_per_unit) * TILE;
-        const unsigned char* tile = tiles + (size_t)buf * C::kTileBytes;
-        const int blk0 = i0 / b;
-        const int nblk = min(nb - blk0, TILE / b);
-        const int rows = min(N, i0 + TILE) - i0;
-
-        // split right-hand sides of this tile's blocks from the prefetched anchors, then start the next fetch
-        if (tid < D) {
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                if (q < nblk) {
-                    __nv_bfloat16* r = rhs + (size_t)q * 8 * D + tid;
-                    split3_bf16(cur_an.ms, r, D);
-                    split3_bf16(cur_an.me[q], r + 3 * D, D);
-                    r[6 * D] = __float2bfloat16_rn(0.f);
-                    r[7 * D] = __float2bfloat16_rn(0.f);
-                }
-            }
-            if (tid <= nblk) scal[tid] = cur_an.sc;
-            if (tn < total) load_anchors(tn, cur_an);
-        }
-        // each lane finishes one of the four results of its quad: t=0: a_s(row g), t=1: a_e(row g),
-        // t=2: a_s(row g+8), t=3: a_e(row g+8); its key's reciprocal norm is fetched before the copy is awaited
-        const int row_in_block = g + ((t & 2) ? 8 : 0);
-        float inv_pre[C::kIters];
-#pragma unroll
-        for (int k = 0; k < C::kIters; ++k) {
-            const int r0 = (warp + k * C::kWarps) * 16;
-            inv_pre[k] = r0 < rows && i0 + r0 + row_in_block < N ? inv_norm[(int64_t)u * N + i0 + r0 + row_in_block] : 0.f;
-        }
-        __syncthreads();
-        const float rs = scal[0];
-        if (!mbar_wait(&full[buf], (uint32_t)((it / C::kBufs) & 1), status, 403)) return;
-
-        float lo_s = INFINITY, hi_s = -INFINITY, lo_e = INFINITY, hi_e = -INFINITY;
-#pragma unroll
-        for (int k = 0; k < C::kIters; ++k) {
-            const int r0 = (warp + k * C::kWarps) * 16;
-            if (r0 >= rows) break;
-            const int q = min((i0 + r0) / b, nb - 1) - blk0;
-            const float re = scal[1 + q];
-            float c[4] = {0.f, 0.f, 0.f, 0.f};
-            const unsigned char* row_lo = tile + (size_t)(r0 + g) * C::kRowBytes;
-            const unsigned char* row_hi = row_lo + 8 * C::kRowBytes;
-            const __nv_bfloat16* rq = rhs + ((size_t)q * 8 + g) * D;
-#pragma unroll
-            for (int j = 0; j < kCh; ++j) {
-                const uint4 x = *reinterpret_cast<const uint4*>(row_lo + (t + 4 * j) * 16);
-                const uint4 y = *reinterpret_cast<const uint4*>(row_hi + (t + 4 * j) * 16);
-                const uint4 w = *reinterpret_cast<const uint4*>(rq + (t + 4 * j) * 8);
-                const uint32_t a_first[4] = {x.x, y.x, x.y, y.y};
-                const uint32_t a_second[4] = {x.z, y.z, x.w, y.w};
-                mma_bf16_16816(c, a_first, w.x, w.y);
-                mma_bf16_16816(c, a_second, w.z, w.w);
-            }
-            // columns 0,1 (t=0) and 2 (t=1, c[0]) belong to mu_s; 3 (t=1, c[1]) and 4,5 (t=2) to mu_e
-            float xs_lo = t == 0 ? c[0] + c[1] : (t == 1 ? c[0] : 0.f);
-            float xe_lo = t == 1 ? c[1] : (t == 2 ? c[0] + c[1] : 0.f);
-            float xs_hi = t == 0 ? c[2] + c[3] : (t == 1 ? c[2] : 0.f);
-            float xe_hi = t == 1 ? c[3] : (t == 2 ? c[2] + c[3] : 0.f);
-#pragma unroll
-            for (int o = 1; o <= 2; o <<= 1) {
-                xs_lo += __shfl_xor_sync(0xffffffffu, xs_lo, o);
-                xe_lo += __shfl_xor_sync(0xffffffffu, xe_lo, o);
-                xs_hi += __shfl_xor_sync(0xffffffffu, xs_hi, o);
-                xe_hi += __shfl_xor_sync(0xffffffffu, xe_hi, o);
-            }
-            const float dot = t == 0 ? xs_lo : (t == 1 ? xe_lo : (t == 2 ? xs_hi : xe_hi));
-            const float a = -(dot * inv_pre[k]) * ((t & 1) ? re : rs) + 0.f;
-            const int gi = i0 + r0 + row_in_block;
-            if (gi < N) {
-                a_raw[((int64_t)u * 3 + (t & 1)) * N + gi] = a;
-                if (t & 1) {
-                    lo_e = fminf(lo_e, a);
-                    hi_e = fmaxf(hi_e, a);
-                } else {
-                    lo_s = fminf(lo_s, a);
-                    hi_s = fmaxf(hi_s, a);
-                }
-            }
-        }
-        lo_s = warp_min(lo_s);
-        hi_s = warp_max(hi_s);
-        lo_e = warp_min(lo_e);
-        hi_e = warp_max(hi_e);
-        uint32_t* kk = keys + (it & 1) * 4;
-        if (lane == 0) {
-            if (lo_s <= hi_s) {
-                atomicMin(&kk[0], ord_key(lo_s));
-                atomicMax(&kk[1], ord_key(hi_s));
-            }
-            if (lo_e <= hi_e) {
-                atomicMin(&kk[2], ord_key(lo_e));
-                atomicMax(&kk[3], ord_key(hi_e));
-            }
-        }
-        __syncthreads();   // the tile, rhs and scal may be overwritten from here on; the tile's keys are final
-        if (tid < 4) {
-            const uint32_t v = kk[tid];
-            if (tid & 1) {
-                if (v != 0u) atomicMax(&mm[(int64_t)u * 6 + tid], v);
-                kk[tid] = 0u;
-            } else {
-                if (v != 0xffffffffu) atomicMin(&mm[(int64_t)u * 6 + tid], v);
-                kk[tid] = 0xffffffffu;
-            }
-        }
-    }
-}
-
 // reset of the per-head min/max keys (and, when blocks straddle tiles, of the block sums)
 __global__ void stream_init_kernel(int units, uint32_t* mm, float* block_sums, long long n_sums) {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -793,13 +592,6 @@ cudaError_t set_attrs() {
     return cudaFuncSetAttribute(stream_b_kernel<T, D, Tiles<T, D>::B>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)BCfg<T, D, Tiles<T, D>::B>::kSmem);
 }
-template <int D>
-cudaError_t set_mma_attr() {
-    constexpr int TILE = Tiles<__nv_bfloat16, D>::B;
-    return cudaFuncSetAttribute(stream_b_mma_kernel<D, TILE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)BMmaCfg<D, TILE>::kSmem);
-}
-
 }  // namespace
 
 cudaError_t configure_stream_kernels() {
@@ -808,8 +600,6 @@ cudaError_t configure_stream_kernels() {
     if ((e = set_attrs<__nv_bfloat16, 128>()) != cudaSuccess) return e;
     if ((e = set_attrs<float, 64>()) != cudaSuccess) return e;
     if ((e = set_attrs<float, 128>()) != cudaSuccess) return e;
-    if ((e = set_mma_attr<64>()) != cudaSuccess) return e;
-    if ((e = set_mma_attr<128>()) != cudaSuccess) return e;
     return cudaSuccess;
 }
 
@@ -861,24 +651,6 @@ cudaError_t launch_stream_b(const TensorView& K, int dtype, int G, const ScorePa
 #undef CALL
     const long long total = (long long)units * ((K.N + tile - 1) / tile);
     const unsigned grid = (unsigned)(total < sm_count ? total : sm_count);
-    // The tensor-core variant gives the same results but measures slower on B200 (3.8 ms against 2.3 ms at
-    // 36 x 4 x 8 heads of 32768 bf16 keys, d = 128): it waits on barriers with next to nothing to overlap.
-    constexpr bool kTensorCoreSecondPass = false;
-    if (kTensorCoreSecondPass && dtype == NKV_BF16 && sp.block % 16 == 0 && tile / sp.block <= 4) {
-        // bf16 keys: the two dots per key run on the tensor cores
-        if (K.d == 128)
-            stream_b_mma_kernel<128, Tiles<__nv_bfloat16, 128>::B>
-                <<<grid, BMmaCfg<128, Tiles<__nv_bfloat16, 128>::B>::kThreads,
-                   BMmaCfg<128, Tiles<__nv_bfloat16, 128>::B>::kSmem, stream>>>(K, sp, units, mu_s, mu_e, inv_norm,
-                                                                                  inv_s, inv_e, a_raw, mm, status);
-        else
-            stream_b_mma_kernel<64, Tiles<__nv_bfloat16, 64>::B>
-                <<<grid, BMmaCfg<64, Tiles<__nv_bfloat16, 64>::B>::kThreads,
-                   BMmaCfg<64, Tiles<__nv_bfloat16, 64>::B>::kSmem, stream>>>(K, sp, units, mu_s, mu_e, inv_norm, inv_s,
-                                                                                inv_e, a_raw, mm, status);
-        ++*launches;
-        return cudaGetLastError();
-    }
 #define CALL(T, D)                                                                                         \
     stream_b_kernel<T, D, Tiles<T, D>::B><<<grid, BCfg<T, D, Tiles<T, D>::B>::kThreads,                       \
                                             BCfg<T, D, Tiles<T, D>::B>::kSmem, stream>>>(                    \
