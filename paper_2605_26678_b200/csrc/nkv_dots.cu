@@ -157,22 +157,36 @@ __device__ void dots_epilogue(Smem* s, uint32_t tmem_base, ScoreParams sp, TileR
         lo_s = lo_e = INFINITY;
         hi_s = hi_e = -INFINITY;
     };
+    // per-tile inputs of this thread's row, fetched one tile ahead of their use
+    struct RowIn {
+        int u, i;
+        bool second;
+        float inv_i, re;
+    };
+    auto fetch = [&](long long t) {
+        RowIn x;
+        x.u = (int)(t / tr.tiles_per_unit);
+        const int i0 = (int)(t - (long long)x.u * tr.tiles_per_unit) * kTile;
+        const int blk0 = i0 / sp.block;
+        x.i = i0 + r;
+        x.second = x.i >= (blk0 + 1) * sp.block;   // the key lies in the block after the tile's first
+        const int blk = min(blk0 + (x.second ? 1 : 0), sp.nblocks - 1);
+        x.inv_i = x.i < N ? inv_norm[(int64_t)x.u * N + x.i] : 0.f;
+        x.re = inv_e[(int64_t)x.u * sp.nblocks + blk];
+        return x;
+    };
     long long n = 0;
+    RowIn nxt = {};
+    if (tr.first < tr.last) nxt = fetch(tr.first);
     for (long long t = tr.first; t < tr.last; ++t, ++n) {
         const int stage = (int)(n % kStages);
-        const int u = (int)(t / tr.tiles_per_unit);
-        const int i0 = (int)(t - (long long)u * tr.tiles_per_unit) * kTile;
-        if (u != cur_u) {
+        const RowIn cur = nxt;
+        if (t + 1 < tr.last) nxt = fetch(t + 1);
+        if (cur.u != cur_u) {
             flush();
-            cur_u = u;
-            rs = inv_s[u];
+            cur_u = cur.u;
+            rs = inv_s[cur.u];
         }
-        const int blk0 = i0 / sp.block;
-        const int i = i0 + r;
-        const bool second = i >= (blk0 + 1) * sp.block;   // the key lies in the block after the tile's first
-        const int blk = min(blk0 + (second ? 1 : 0), sp.nblocks - 1);
-        const float inv_i = i < N ? inv_norm[(int64_t)u * N + i] : 0.f;
-        const float re = inv_e[(int64_t)u * sp.nblocks + blk];
         if (!mbar_wait(&s->tfull[stage], (uint32_t)((n / kStages) & 1), status, 716)) return;
         tc_fence_after();
         float d[16];
@@ -182,12 +196,12 @@ __device__ void dots_epilogue(Smem* s, uint32_t tmem_base, ScoreParams sp, TileR
         __syncwarp();
         if (lane == 0) mbar_arrive(&s->tempty[stage]);
         const float ds = d[0] + d[1] + d[2];
-        const float de = second ? d[6] + d[7] + d[8] : d[3] + d[4] + d[5];
-        const float a_s = -(ds * inv_i) * rs + 0.f;
-        const float a_e = -(de * inv_i) * re + 0.f;
-        if (i < N) {
-            a_raw[((int64_t)u * 3 + 0) * N + i] = a_s;
-            a_raw[((int64_t)u * 3 + 1) * N + i] = a_e;
+        const float de = cur.second ? d[6] + d[7] + d[8] : d[3] + d[4] + d[5];
+        const float a_s = -(ds * cur.inv_i) * rs + 0.f;
+        const float a_e = -(de * cur.inv_i) * cur.re + 0.f;
+        if (cur.i < N) {
+            a_raw[((int64_t)cur.u * 3 + 0) * N + cur.i] = a_s;
+            a_raw[((int64_t)cur.u * 3 + 1) * N + cur.i] = a_e;
             lo_s = fminf(lo_s, a_s);
             hi_s = fmaxf(hi_s, a_s);
             lo_e = fminf(lo_e, a_e);

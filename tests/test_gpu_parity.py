@@ -178,7 +178,8 @@ def test_fused_compress_end_to_end(N, d, dtype, H, layers, r, scan_lag):
 
 
 @pytest.mark.parametrize("N,H,layers,r", [
-    (100, 2, 1, 0.5), (777, 1, 3, 0.9), (2500, 8, 2, 0.95), (4096, 4, 1, 0.75), (8200, 3, 1, 0.75)])
+    (100, 2, 1, 0.5), (777, 1, 3, 0.9), (2500, 8, 2, 0.95), (4096, 4, 1, 0.75), (8200, 3, 1, 0.75),
+    (4352, 2, 1, 0.75), (6144, 2, 1, 0.5)])   # the last two: blocks of 136 and 192 keys straddle the 128-key tiles
 @pytest.mark.parametrize("mode", ["tensor", "fma"])
 def test_key_pass_kernels_end_to_end(N, H, layers, r, mode):
     """Both key passes on the tensor cores (tcgen05: band sums of the keys' Gram matrix, dots with the
