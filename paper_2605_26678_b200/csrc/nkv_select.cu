@@ -330,12 +330,21 @@ __device__ void block_select_bracket(SelectShared& S, BracketShared<CAP>& X, con
         for (int b = tid; b < kBins; b += nt) S.hist[b] = 0;
         __syncthreads();
         int mine = 0;
-        for (int i = tid; i < positions; i += nt) {
-            float v;
-            if (src.get((int)(((long long)i * n) / positions), v)) {
-                atomicAdd(&S.hist[bin_of(v, lo0, sc0)], 1);
-                ++mine;
+        for (int i0 = 0; i0 < positions; i0 += 4 * nt) {   // four loads in flight per thread
+            float sv[4];
+            bool sk[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int i = i0 + k * nt + tid;
+                sv[k] = 0.f;
+                sk[k] = i < positions && src.get((int)(((long long)i * n) / positions), sv[k]);
             }
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (sk[k]) {
+                    atomicAdd(&S.hist[bin_of(sv[k], lo0, sc0)], 1);
+                    ++mine;
+                }
         }
         const int sn = block_sum_int(S, mine);
         // 2. pivots: sample ranks around rank * sn / n_eff, four standard deviations of the rank error apart
@@ -380,21 +389,31 @@ __device__ void block_select_bracket(SelectShared& S, BracketShared<CAP>& X, con
         int cnt = 0;
         float sum = 0.f;
         const int lane = tid & 31;
-        for (int j0 = 0; j0 < n; j0 += nt) {
-            const int j = j0 + tid;
-            float v = 0.f;
-            const bool in = j < n && src.get(j, v);
-            const bool above = in && v > p_hi;
-            const bool inside = in && !above && v >= p_lo;
-            cnt += above;
-            if (above) sum += v;
-            const unsigned ballot = __ballot_sync(0xffffffffu, inside);
-            if (ballot) {
-                int base = 0;
-                if (lane == 0) base = atomicAdd(&X.cand_n, __popc(ballot));
-                base = __shfl_sync(0xffffffffu, base, 0);
-                const int pos = base + __popc(ballot & ((1u << lane) - 1u));
-                if (inside && pos < kCandCap) X.cand[pos] = v;
+        for (int jb = 0; jb < n; jb += 4 * nt) {   // four loads in flight per thread
+            float vv[4];
+            bool vk[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int j = jb + k * nt + tid;
+                vv[k] = 0.f;
+                vk[k] = j < n && src.get(j, vv[k]);
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float v = vv[k];
+                const bool in = vk[k];
+                const bool above = in && v > p_hi;
+                const bool inside = in && !above && v >= p_lo;
+                cnt += above;
+                if (above) sum += v;
+                const unsigned ballot = __ballot_sync(0xffffffffu, inside);
+                if (ballot) {
+                    int base = 0;
+                    if (lane == 0) base = atomicAdd(&X.cand_n, __popc(ballot));
+                    base = __shfl_sync(0xffffffffu, base, 0);
+                    const int pos = base + __popc(ballot & ((1u << lane) - 1u));
+                    if (inside && pos < kCandCap) X.cand[pos] = v;
+                }
             }
         }
         cnt = block_sum_int(S, cnt);
