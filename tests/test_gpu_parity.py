@@ -201,6 +201,26 @@ def test_key_pass_kernels_end_to_end(N, H, layers, r, mode):
     assert rep.swapped_tokens <= max(2, rep.heads)
 
 
+@pytest.mark.parametrize("N,d,dtype,H,layers,r", [(600, 128, "bf16", 2, 9, 0.75), (333, 64, "fp32", 3, 10, 0.5)])
+def test_many_groups_and_repeated_calls(N, d, dtype, H, layers, r):
+    """Nine and ten layer groups in one call: every group matches the oracle, and two calls in a row on
+    the same buffers and workspace give identical outputs (nothing is left over from the first)."""
+    K, V = _cache(N, d, dtype, H=H, layers=layers)
+    p = nkv.nkv_default_params()
+    ws = nkv.alloc_workspace(K, p)
+    res = nkv.nkv_compress(K, V, r, p, ws=ws, want_a_star=True)
+    torch.cuda.synchronize()
+    assert nkv.nkv_last_device_status(ws) == nkv.NKV_OK
+    first = (res.idx.clone(), res.k_out.clone(), res.v_out.clone(), res.budgets.clone())
+    rep = pr.SwapReport()
+    for g in range(K.shape[0]):
+        pr.check_group_against_oracle(K, V, res, g, r, p, rep)
+    assert rep.swapped_tokens <= max(2, rep.heads)
+    res = nkv.nkv_compress(K, V, r, p, out=res, ws=ws)
+    torch.cuda.synchronize()
+    assert all(torch.equal(a, b) for a, b in zip(first, (res.idx, res.k_out, res.v_out, res.budgets)))
+
+
 def test_identical_keys_take_the_tie_path():
     """All keys equal: every score is 0 and every selection is decided by position alone."""
     K = torch.ones((1, 2, 3000, 64), dtype=torch.bfloat16, device=DEV)
