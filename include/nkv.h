@@ -260,11 +260,12 @@ NKV_API int nkv_set_scan_options(nkv_handle* h, int lag, int l2_hints);
  * pass yields 1/||k||, the block sums of normalised keys and the current-memory anomaly a_c; the
  * second the anomalies a_s and a_e against the global and block anchors.
  * NKV_KEY_PASS_FMA does both with fp32 FMAs on staged key tiles (any supported dtype and d).
- * NKV_KEY_PASS_TENSOR (bf16 keys, d = 128) forms on the tensor cores what is a contraction: in the
- * first pass (W = 64 only, one CTA per head) k_hat_i . S_i and ||S_i||^2 as sums over a band of the
- * keys' Gram matrix, in the second pass the dots of the keys with the anchors, the fp32 anchors split
- * three ways into bf16.  A pass whose inputs do not allow the tensor form runs the FMA kernel.
- * NKV_KEY_PASS_AUTO (default) takes the tensor form of the second pass whenever it is allowed, and of
+ * NKV_KEY_PASS_TENSOR (bf16 keys) forms on the tensor cores what is a contraction: in the first pass
+ * (d = 128, W = 64 only, one CTA per head) k_hat_i . S_i and ||S_i||^2 as sums over a band of the
+ * keys' Gram matrix, in the second pass (d = 64 or 128) the dots of the keys with the anchors, the
+ * fp32 anchors split three ways into bf16.  A pass whose inputs do not allow the tensor form runs the
+ * FMA kernel.
+ * NKV_KEY_PASS_AUTO (default) takes the tensor form of the second pass when d = 128, and of
  * the first pass when in addition the call's heads, dealt one per SM, keep at least 85 % of the SMs
  * busy over the rounds that takes.
  * The forms agree to fp32 rounding. */

@@ -427,7 +427,9 @@ int nkv_compress(nkv_handle* h, const nkv_tensor* K, const nkv_tensor* V, double
         CU(launch_anchor_norms(units, d, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_s),
                                at<float>(ws, L.inv_e), nullptr, st, &h->launches));
         CU(mark());
-        if (h->key_pass != NKV_KEY_PASS_FMA && anchor_dots_supported(kv, K->dtype, sp))
+        // d = 64 tiles are too small to pay for the per-tile hand-overs: the FMA form is faster there
+        const bool dots_wanted = h->key_pass == NKV_KEY_PASS_TENSOR || (h->key_pass == NKV_KEY_PASS_AUTO && d == 128);
+        if (dots_wanted && anchor_dots_supported(kv, K->dtype, sp))
             CU(launch_anchor_dots(kv, G, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm),
                                   at<float>(ws, L.inv_s), at<float>(ws, L.inv_e), at<float>(ws, L.a_raw),
                                   at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));

@@ -1,4 +1,4 @@
-// Second key pass on the tensor cores (bf16 keys, d = 128): a_s(i) = -cos(k_hat_i, mu_s) and
+// Second key pass on the tensor cores (bf16 keys, d = 64 or 128): a_s(i) = -cos(k_hat_i, mu_s) and
 // a_e(i) = -cos(k_hat_i, mu_e(block of i)) with their per-head min/max (Section 2.3).
 //
 // The dots of 128 keys with the anchors are one skinny product [128 x d] x [d x 16] per tile.  The fp32
@@ -18,27 +18,38 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kD = 128;
 constexpr int kTile = 128;                        // keys per tile
-constexpr int kSlots = 5;                         // key tiles staged at once
 constexpr int kTileHalfBytes = kTile * 128;       // one 64-column half of a tile
-constexpr int kTileBytes = 2 * kTileHalfBytes;
 constexpr int kRhsHalfBytes = 16 * 128;           // 16 right-hand-side rows of 64 columns
-constexpr int kRhsBytes = 2 * kRhsHalfBytes;
 constexpr int kStages = 4;                        // accumulators of 32 columns (16 used)
 constexpr uint32_t kTmemCols = 128;
 constexpr int kPrepWarp0 = 0, kEpiWarp0 = 4, kProducerWarp = 8, kMmaWarp = 9;
 constexpr int kThreads = 10 * 32;
+constexpr int kMaxSlots = 10;
+
+// Sizes for head dimension D (64 or 128): a key row is D / 64 swizzled halves of 128 bytes.
+template <int D>
+struct Cfg {
+    static constexpr int kHalves = D / 64;
+    static constexpr int kSlots = 640 / D;                       // key tiles staged at once (160 KB)
+    static constexpr int kTileBytes = kHalves * kTileHalfBytes;
+    static constexpr int kRhsBytes = kHalves * kRhsHalfBytes;
+    static constexpr int kPrepWarps = D / 32;                    // one thread per column
+    static_assert(kSlots <= kMaxSlots, "barrier arrays too small");
+};
 
 struct Smem {
-    uint64_t full[kSlots];      // key tile landed
-    uint64_t rready[kSlots];    // right-hand side written (one arrival per building warp)
-    uint64_t kfree[kSlots];     // tile and right-hand side consumed by the MMAs
+    uint64_t full[kMaxSlots];   // key tile landed
+    uint64_t rready[kMaxSlots]; // right-hand side written (one arrival per building warp)
+    uint64_t kfree[kMaxSlots];  // tile and right-hand side consumed by the MMAs
     uint64_t tfull[kStages];    // accumulator written
     uint64_t tempty[kStages];   // accumulator read (one arrival per reading warp)
     uint32_t tmem_base;
 };
-constexpr size_t kSmemBytes = 1024 + (size_t)kSlots * (kTileBytes + kRhsBytes) + sizeof(Smem);
+template <int D>
+constexpr size_t smem_bytes() {
+    return 1024 + (size_t)Cfg<D>::kSlots * (Cfg<D>::kTileBytes + Cfg<D>::kRhsBytes) + sizeof(Smem);
+}
 
 struct TileRange {
     long long first, last;      // this CTA's tiles [first, last)
@@ -54,39 +65,44 @@ __device__ __forceinline__ TileRange my_tiles(int units, int N) {
 }
 
 // ---------------------------------------------------------------------------- roles
+template <int D>
 __device__ void dots_producer(const CUtensorMap* tmap, unsigned char* tiles, Smem* s, TileRange tr, int H, int* status) {
+    using C = Cfg<D>;
     long long n = 0;
     for (long long t = tr.first; t < tr.last; ++t, ++n) {
-        const int slot = (int)(n % kSlots);
-        const long long fill = n / kSlots;
+        const int slot = (int)(n % C::kSlots);
+        const long long fill = n / C::kSlots;
         if (fill > 0 && !mbar_wait(&s->kfree[slot], (uint32_t)((fill - 1) & 1), status, 711)) return;
         const int u = (int)(t / tr.tiles_per_unit);
         const int i0 = (int)(t - (long long)u * tr.tiles_per_unit) * kTile;
         const int g = u / H, h = u - g * H;
-        unsigned char* dst = tiles + (size_t)slot * kTileBytes;
-        mbar_expect_tx(&s->full[slot], kTileBytes);
-        tma_load_4d(dst, tmap, 0, i0, h, g, &s->full[slot]);
-        tma_load_4d(dst + kTileHalfBytes, tmap, 64, i0, h, g, &s->full[slot]);
+        unsigned char* dst = tiles + (size_t)slot * C::kTileBytes;
+        mbar_expect_tx(&s->full[slot], C::kTileBytes);
+#pragma unroll
+        for (int half = 0; half < C::kHalves; ++half)
+            tma_load_4d(dst + half * kTileHalfBytes, tmap, 64 * half, i0, h, g, &s->full[slot]);
     }
 }
 
+template <int D>
 __device__ void dots_mma(unsigned char* tiles, unsigned char* rhs, Smem* s, uint32_t tmem_base, TileRange tr,
                          int* status) {
+    using C = Cfg<D>;
     constexpr uint32_t idesc = umma_idesc_bf16(kTile, 16);
     const uint32_t tiles_addr = smem_addr(tiles), rhs_addr = smem_addr(rhs);
     long long n = 0;
     for (long long t = tr.first; t < tr.last; ++t, ++n) {
-        const int slot = (int)(n % kSlots), stage = (int)(n % kStages);
-        const uint32_t fpar = (uint32_t)((n / kSlots) & 1), upar = (uint32_t)((n / kStages) & 1);
+        const int slot = (int)(n % C::kSlots), stage = (int)(n % kStages);
+        const uint32_t fpar = (uint32_t)((n / C::kSlots) & 1), upar = (uint32_t)((n / kStages) & 1);
         if (!mbar_wait(&s->full[slot], fpar, status, 712)) return;
         if (!mbar_wait(&s->rready[slot], fpar, status, 713)) return;
         if (!mbar_wait(&s->tempty[stage], upar ^ 1u, status, 714)) return;
         tc_fence_after();
 #pragma unroll
-        for (int kk = 0; kk < kD / 16; ++kk) {
-            const uint32_t a = tiles_addr + (uint32_t)slot * kTileBytes + (uint32_t)(kk >> 2) * kTileHalfBytes +
+        for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t a = tiles_addr + (uint32_t)slot * C::kTileBytes + (uint32_t)(kk >> 2) * kTileHalfBytes +
                                (uint32_t)(kk & 3) * 32u;
-            const uint32_t b = rhs_addr + (uint32_t)slot * kRhsBytes + (uint32_t)(kk >> 2) * kRhsHalfBytes +
+            const uint32_t b = rhs_addr + (uint32_t)slot * C::kRhsBytes + (uint32_t)(kk >> 2) * kRhsHalfBytes +
                                (uint32_t)(kk & 3) * 32u;
             umma_bf16(tmem_base + (uint32_t)stage * 32u, umma_desc_sw128(a), umma_desc_sw128(b), idesc, kk > 0);
         }
@@ -96,23 +112,31 @@ __device__ void dots_mma(unsigned char* tiles, unsigned char* rhs, Smem* s, uint
 }
 
 // Thread k writes column k of the nine right-hand-side rows of every tile (rows 9..15 stay zero).
+template <int D>
 __device__ void dots_prep(unsigned char* rhs, Smem* s, ScoreParams sp, TileRange tr, const float* __restrict__ mu_s,
                           const float* __restrict__ mu_e, int* status) {
+    using C = Cfg<D>;
     const int k = threadIdx.x - kPrepWarp0 * 32, lane = k & 31;
+    if (k >= D) return;   // d = 64 needs two of the four warps
     const int half = k >> 6, kk = k & 63;
+    float v[3] = {0.f, 0.f, 0.f};
+    int cur_u = -1, cur_blk = -1;
     long long n = 0;
     for (long long t = tr.first; t < tr.last; ++t, ++n) {
-        const int slot = (int)(n % kSlots);
-        const long long fill = n / kSlots;
+        const int slot = (int)(n % C::kSlots);
+        const long long fill = n / C::kSlots;
         if (fill > 0 && !mbar_wait(&s->kfree[slot], (uint32_t)((fill - 1) & 1), status, 715)) return;
         const int u = (int)(t / tr.tiles_per_unit);
         const int i0 = (int)(t - (long long)u * tr.tiles_per_unit) * kTile;
         const int blk0 = i0 / sp.block;
-        float v[3];
-        v[0] = mu_s[(int64_t)u * kD + k];
-        v[1] = mu_e[((int64_t)u * sp.nblocks + blk0) * kD + k];
-        v[2] = blk0 + 1 < sp.nblocks ? mu_e[((int64_t)u * sp.nblocks + blk0 + 1) * kD + k] : 0.f;
-        unsigned char* base = rhs + (size_t)slot * kRhsBytes + (size_t)half * kRhsHalfBytes + (kk & 7) * 2;
+        if (u != cur_u || blk0 != cur_blk) {   // the anchors change every few tiles only
+            if (u != cur_u) v[0] = mu_s[(int64_t)u * D + k];
+            v[1] = mu_e[((int64_t)u * sp.nblocks + blk0) * D + k];
+            v[2] = blk0 + 1 < sp.nblocks ? mu_e[((int64_t)u * sp.nblocks + blk0 + 1) * D + k] : 0.f;
+            cur_u = u;
+            cur_blk = blk0;
+        }
+        unsigned char* base = rhs + (size_t)slot * C::kRhsBytes + (size_t)half * kRhsHalfBytes + (kk & 7) * 2;
 #pragma unroll
         for (int a = 0; a < 3; ++a) {
             const __nv_bfloat16 hi = __float2bfloat16_rn(v[a]);
@@ -211,22 +235,24 @@ __device__ void dots_epilogue(Smem* s, uint32_t tmem_base, ScoreParams sp, TileR
     flush();
 }
 
+template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 anchor_dots_kernel(const __grid_constant__ CUtensorMap tmap, ScoreParams sp, int units, int H, int N,
                    const float* __restrict__ mu_s, const float* __restrict__ mu_e, const float* __restrict__ inv_norm,
                    const float* __restrict__ inv_s, const float* __restrict__ inv_e, float* __restrict__ a_raw,
                    uint32_t* __restrict__ mm, int* status) {
+    using C = Cfg<D>;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* tiles = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
-    unsigned char* rhs = tiles + (size_t)kSlots * kTileBytes;
-    Smem* s = reinterpret_cast<Smem*>(rhs + (size_t)kSlots * kRhsBytes);
+    unsigned char* rhs = tiles + (size_t)C::kSlots * C::kTileBytes;
+    Smem* s = reinterpret_cast<Smem*>(rhs + (size_t)C::kSlots * C::kRhsBytes);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const TileRange tr = my_tiles(units, N);
 
     if (tid == 0) {
-        for (int i = 0; i < kSlots; ++i) {
+        for (int i = 0; i < C::kSlots; ++i) {
             mbar_init(&s->full[i], 1);
-            mbar_init(&s->rready[i], 4);
+            mbar_init(&s->rready[i], C::kPrepWarps);
             mbar_init(&s->kfree[i], 1);
         }
         for (int i = 0; i < kStages; ++i) {
@@ -235,7 +261,7 @@ anchor_dots_kernel(const __grid_constant__ CUtensorMap tmap, ScoreParams sp, int
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int i = tid; i < kSlots * kRhsBytes / 16; i += kThreads) reinterpret_cast<uint4*>(rhs)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < C::kSlots * C::kRhsBytes / 16; i += kThreads) reinterpret_cast<uint4*>(rhs)[i] = make_uint4(0, 0, 0, 0);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     if (warp == kMmaWarp) tmem_alloc(&s->tmem_base, kTmemCols);
     tc_fence_before();
@@ -244,15 +270,15 @@ anchor_dots_kernel(const __grid_constant__ CUtensorMap tmap, ScoreParams sp, int
     const uint32_t tmem_base = s->tmem_base;
 
     if (warp == kProducerWarp) {
-        if (lane == 0) dots_producer(&tmap, tiles, s, tr, H, status);
+        if (lane == 0) dots_producer<D>(&tmap, tiles, s, tr, H, status);
         __syncwarp();
     } else if (warp == kMmaWarp) {
-        if (lane == 0) dots_mma(tiles, rhs, s, tmem_base, tr, status);
+        if (lane == 0) dots_mma<D>(tiles, rhs, s, tmem_base, tr, status);
         __syncwarp();
     } else if (warp >= kEpiWarp0) {
         dots_epilogue(s, tmem_base, sp, tr, N, inv_norm, inv_s, inv_e, a_raw, mm, status);
     } else {
-        dots_prep(rhs, s, sp, tr, mu_s, mu_e, status);
+        dots_prep<D>(rhs, s, sp, tr, mu_s, mu_e, status);
     }
 
     tc_fence_before();
@@ -263,16 +289,20 @@ anchor_dots_kernel(const __grid_constant__ CUtensorMap tmap, ScoreParams sp, int
 }  // namespace
 
 cudaError_t configure_dots_kernels() {
-    return cudaFuncSetAttribute(anchor_dots_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(anchor_dots_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem_bytes<64>());
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(anchor_dots_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)smem_bytes<128>());
 }
 
-// Same input conditions as the tensor-core first pass, and blocks of at least 128 keys (a tile of 128
-// keys then touches at most two blocks).
+// bf16 keys of 64 or 128 columns, strides a tensor map accepts, and blocks of at least 128 keys (a tile
+// of 128 keys then touches at most two blocks).
 bool anchor_dots_supported(const TensorView& K, int dtype, const ScoreParams& sp) {
-    if (dtype != NKV_BF16 || K.d != kD || sp.block < kTile) return false;
+    if (dtype != NKV_BF16 || (K.d != 64 && K.d != 128) || sp.block < kTile) return false;
     if (reinterpret_cast<uintptr_t>(K.ptr) % 16 != 0) return false;
     if (K.stride_h % 8 != 0 || K.stride_g % 8 != 0) return false;
-    if (K.stride_h < (int64_t)K.N * kD || K.stride_g < (int64_t)K.N * kD) return false;
+    if (K.stride_h < (int64_t)K.N * K.d || K.stride_g < (int64_t)K.N * K.d) return false;
     CUtensorMap probe;   // the driver has the last word on what a tensor map can describe
     return encode_key_map(K, 1, kTile, &probe) == cudaSuccess;
 }
@@ -286,8 +316,12 @@ cudaError_t launch_anchor_dots(const TensorView& K, int G, const ScoreParams& sp
     const int units = G * K.H;
     const long long total = (long long)units * ((K.N + kTile - 1) / kTile);
     const unsigned grid = (unsigned)(total < sm_count ? total : sm_count);
-    anchor_dots_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tmap, sp, units, K.H, K.N, mu_s, mu_e, inv_norm, inv_s,
-                                                               inv_e, a_raw, mm, status);
+    if (K.d == 128)
+        anchor_dots_kernel<128><<<grid, kThreads, smem_bytes<128>(), stream>>>(tmap, sp, units, K.H, K.N, mu_s, mu_e,
+                                                                               inv_norm, inv_s, inv_e, a_raw, mm, status);
+    else
+        anchor_dots_kernel<64><<<grid, kThreads, smem_bytes<64>(), stream>>>(tmap, sp, units, K.H, K.N, mu_s, mu_e,
+                                                                             inv_norm, inv_s, inv_e, a_raw, mm, status);
     ++*launches;
     return cudaGetLastError();
 }

@@ -180,11 +180,12 @@ def test_fused_compress_end_to_end(N, d, dtype, H, layers, r, scan_lag):
 @pytest.mark.parametrize("N,H,layers,r", [
     (100, 2, 1, 0.5), (777, 1, 3, 0.9), (2500, 8, 2, 0.95), (4096, 4, 1, 0.75), (8200, 3, 1, 0.75),
     (4352, 2, 1, 0.75), (6144, 2, 1, 0.5)])   # the last two: blocks of 136 and 192 keys straddle the 128-key tiles
-@pytest.mark.parametrize("mode", ["tensor", "fma"])
-def test_key_pass_kernels_end_to_end(N, H, layers, r, mode):
+@pytest.mark.parametrize("mode,d", [("tensor", 128), ("fma", 128), ("tensor", 64)])
+def test_key_pass_kernels_end_to_end(N, H, layers, r, mode, d):
     """Both key passes on the tensor cores (tcgen05: band sums of the keys' Gram matrix, dots with the
-    split anchors) and both as FMA kernels, each against the oracle."""
-    K, V = _cache(N, 128, "bf16", H=H, layers=layers)
+    split anchors) and both as FMA kernels, each against the oracle.  With d = 64 only the second pass
+    has a tensor-core form."""
+    K, V = _cache(N, d, "bf16", H=H, layers=layers)
     p = nkv.nkv_default_params()
     ws = nkv.alloc_workspace(K, p)
     before = nkv.nkv_launch_count()
