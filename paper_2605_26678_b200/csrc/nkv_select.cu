@@ -35,6 +35,7 @@ struct SelectShared {
     int found;
     float red_f[32];
     int red_i[32];
+    int scan_w[32];   // per-warp totals of find_bin_desc
     // elements to remove from the multiset (value, multiplicity)
     float corr_v[kMaxCorr];
     int corr_m[kMaxCorr];
@@ -57,33 +58,39 @@ __device__ __forceinline__ bool matches(const Levels& L, float v) {
     return true;
 }
 
-// warp 0: the bin holding the `need`-th element counted from the top, and the count above it.
+// The bin holding the `need`-th element counted from the top, and the count above it (S.bin, S.above,
+// S.nbin).  Whole CTA: thread t sums the kBins / blockDim.x bins below bin kBins - 1 - t * per, a scan over
+// the threads finds the owner, which walks its own bins.  The caller synchronises before reading S.*.
 __device__ __forceinline__ void find_bin_desc(SelectShared& S, int need) {
-    if (threadIdx.x < 32) {
-        const int lane = threadIdx.x;
-        constexpr int per = kBins / 32;
-        const int top = kBins - 1 - lane * per;  // lane 0 owns the highest bins
-        int sum = 0;
-        for (int j = 0; j < per; ++j) sum += S.hist[top - j];
-        int incl = sum;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int per = kBins / (int)blockDim.x;   // 8 or 2 (CTAs of 256 or 1024 threads)
+    const int top = kBins - 1 - tid * per;      // thread 0 owns the highest bins
+    int c[8], sum = 0;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            int t = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += t;
-        }
-        const int excl = incl - sum;
-        if (need > excl && need <= incl) {
-            int run = excl;
-            for (int j = 0; j < per; ++j) {
-                const int c = S.hist[top - j];
-                if (need <= run + c) {
-                    S.bin = top - j;
-                    S.above = run;
-                    S.nbin = c;
-                    break;
-                }
-                run += c;
+    for (int j = 0; j < 8; ++j) {
+        c[j] = j < per ? S.hist[top - j] : 0;
+        sum += c[j];
+    }
+    int incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) S.scan_w[warp] = incl;
+    __syncthreads();
+    int excl = incl - sum;
+    for (int w = 0; w < warp; ++w) excl += S.scan_w[w];
+    if (need > excl && need <= excl + sum) {
+        int run = excl;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (j < per && need > run && need <= run + c[j]) {
+                S.bin = top - j;
+                S.above = run;
+                S.nbin = c[j];
             }
+            run += c[j];
         }
     }
 }
