@@ -742,26 +742,48 @@ __global__ void __launch_bounds__(kMixThreads) mix_kernel(int N, ScoreParams sp,
     const float s_mean = s_range > 0.f ? (hs[5] / (float)N - s_lo) / s_range : 0.f;
 
     const int base = blockIdx.x * (kMixThreads * kMixPerThread);
+    // one token: min-max normalise, blend, gate, pin the sinks
+    auto route = [&](float r0, float r1, float r2, int j) {
+        const float x0 = norm01(r0, lo[0], range[0]);
+        const float x1 = norm01(r1, lo[1], range[1]);
+        const float x2 = norm01(r2, lo[2], range[2]);
+        const float blend = w[0] * x0 + w[1] * x1 + w[2] * x2;
+        const float win = fmaxf(x0, fmaxf(x1, x2));
+        float alpha;
+        if (sp.gate_mode == NKV_GATE_AVERAGE) alpha = 0.f;
+        else if (sp.gate_mode == NKV_GATE_MAX) alpha = 1.f;
+        else {
+            const float sn = norm01(surprise3(x0, x1, x2), s_lo, s_range);
+            const float sprime = fmaxf(0.f, sn - s_mean);
+            alpha = 1.0f / (1.0f + expf(-sp.kappa * (sprime - sp.tau)));
+        }
+        const float v = (1.0f - alpha) * blend + alpha * win + 0.f;
+        return j < sp.n_sink ? INFINITY : v;
+    };
+    if ((N & 3) == 0 && ((reinterpret_cast<uintptr_t>(a_raw) | reinterpret_cast<uintptr_t>(a_star)) & 15) == 0) {
+        // rows are 16-byte aligned: four tokens per load
+        const float4* q0 = reinterpret_cast<const float4*>(a0);
+        const float4* q1 = reinterpret_cast<const float4*>(a1);
+        const float4* q2 = reinterpret_cast<const float4*>(a2);
+        float4* out4 = reinterpret_cast<float4*>(a_star + (int64_t)u * N);
 #pragma unroll
-    for (int e = 0; e < kMixPerThread; ++e) {
-        const int j = base + e * kMixThreads + threadIdx.x;
-        if (j < N) {
-            const float x0 = norm01(a0[j], lo[0], range[0]);
-            const float x1 = norm01(a1[j], lo[1], range[1]);
-            const float x2 = norm01(a2[j], lo[2], range[2]);
-            const float blend = w[0] * x0 + w[1] * x1 + w[2] * x2;
-            const float win = fmaxf(x0, fmaxf(x1, x2));
-            float alpha;
-            if (sp.gate_mode == NKV_GATE_AVERAGE) alpha = 0.f;
-            else if (sp.gate_mode == NKV_GATE_MAX) alpha = 1.f;
-            else {
-                const float sn = norm01(surprise3(x0, x1, x2), s_lo, s_range);
-                const float sprime = fmaxf(0.f, sn - s_mean);
-                alpha = 1.0f / (1.0f + expf(-sp.kappa * (sprime - sp.tau)));
+        for (int e = 0; e < kMixPerThread / 4; ++e) {
+            const int j4 = base / 4 + e * kMixThreads + threadIdx.x;
+            if (4 * j4 < N) {
+                const float4 r0 = q0[j4], r1 = q1[j4], r2 = q2[j4];
+                float4 o;
+                o.x = route(r0.x, r1.x, r2.x, 4 * j4);
+                o.y = route(r0.y, r1.y, r2.y, 4 * j4 + 1);
+                o.z = route(r0.z, r1.z, r2.z, 4 * j4 + 2);
+                o.w = route(r0.w, r1.w, r2.w, 4 * j4 + 3);
+                out4[j4] = o;
             }
-            float v = (1.0f - alpha) * blend + alpha * win + 0.f;
-            if (j < sp.n_sink) v = INFINITY;
-            a_star[(int64_t)u * N + j] = v;
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < kMixPerThread; ++e) {
+            const int j = base + e * kMixThreads + threadIdx.x;
+            if (j < N) a_star[(int64_t)u * N + j] = route(a0[j], a1[j], a2[j], j);
         }
     }
     if (stats_out && blockIdx.x == 0 && threadIdx.x == 0) {
