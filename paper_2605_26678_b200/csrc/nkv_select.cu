@@ -688,12 +688,42 @@ __global__ void __launch_bounds__(kStatThreads, 4) scale_stats_kernel(int N, Sco
         if (threadIdx.x == 0) out[k] = gap;
     } else {
         float smin = INFINITY, smax = -INFINITY, ssum = 0.f;
-        for (int j = threadIdx.x; j < N; j += blockDim.x) {
-            const float s = surprise3(norm01(a[0][j], lo[0], range[0]), norm01(a[1][j], lo[1], range[1]),
-                                      norm01(a[2][j], lo[2], range[2]));
+        auto take = [&](float r0, float r1, float r2) {
+            const float s = surprise3(norm01(r0, lo[0], range[0]), norm01(r1, lo[1], range[1]), norm01(r2, lo[2], range[2]));
             smin = fminf(smin, s);
             smax = fmaxf(smax, s);
             ssum += s;
+        };
+        if ((N & 3) == 0 && (reinterpret_cast<uintptr_t>(a_raw) & 15) == 0) {
+            // rows are 16-byte aligned: four tokens per load, two sets of loads in flight
+            const float4* q0 = reinterpret_cast<const float4*>(a[0]);
+            const float4* q1 = reinterpret_cast<const float4*>(a[1]);
+            const float4* q2 = reinterpret_cast<const float4*>(a[2]);
+            const int n4 = N >> 2, nt = blockDim.x;
+            for (int jb = 0; jb < n4; jb += 2 * nt) {
+                float4 r[2][3];
+                bool in[2];
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
+                    const int j = jb + k * nt + threadIdx.x;
+                    in[k] = j < n4;
+                    if (in[k]) {
+                        r[k][0] = q0[j];
+                        r[k][1] = q1[j];
+                        r[k][2] = q2[j];
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < 2; ++k)
+                    if (in[k]) {
+                        take(r[k][0].x, r[k][1].x, r[k][2].x);
+                        take(r[k][0].y, r[k][1].y, r[k][2].y);
+                        take(r[k][0].z, r[k][1].z, r[k][2].z);
+                        take(r[k][0].w, r[k][1].w, r[k][2].w);
+                    }
+            }
+        } else {
+            for (int j = threadIdx.x; j < N; j += blockDim.x) take(a[0][j], a[1][j], a[2][j]);
         }
         smin = block_reduce_f(S, smin, 1);
         smax = block_reduce_f(S, smax, 2);
