@@ -912,10 +912,36 @@ __global__ void __launch_bounds__(kThreads) budget_kernel(int H, int N, int keep
     for (int h = 0; h < H; ++h) {
         int mid = 0, eq = 0;
         const uint32_t Th = T[h];
-        for (int j = threadIdx.x; j < N; j += blockDim.x) {
-            const uint32_t key = ord_key(v[(int64_t)h * N + j]);
+        const float* vh = v + (int64_t)h * N;
+        auto tally = [&](float x) {
+            const uint32_t key = ord_key(x);
             mid += (key > tau && key <= Th);
             eq += (key == tau && key <= Th);
+        };
+        if ((N & 3) == 0 && (reinterpret_cast<uintptr_t>(a_star) & 15) == 0) {
+            // rows are 16-byte aligned: four tokens per load, four loads in flight
+            const float4* q = reinterpret_cast<const float4*>(vh);
+            const int n4 = N >> 2, nt = blockDim.x;
+            for (int jb = 0; jb < n4; jb += 4 * nt) {
+                float4 r[4];
+                bool in[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int j = jb + k * nt + threadIdx.x;
+                    in[k] = j < n4;
+                    if (in[k]) r[k] = q[j];
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    if (in[k]) {
+                        tally(r[k].x);
+                        tally(r[k].y);
+                        tally(r[k].z);
+                        tally(r[k].w);
+                    }
+            }
+        } else {
+            for (int j = threadIdx.x; j < N; j += blockDim.x) tally(vh[j]);
         }
         mid = block_sum_int(S, mid);
         __syncthreads();
