@@ -252,7 +252,11 @@ __device__ __noinline__ void block_select_desc(SelectShared& S, const Src& src, 
 // ------------------------------------------------------------------------------------------
 // head_scores: one CTA per head.
 // ------------------------------------------------------------------------------------------
+// A source yields element j of a multiset (get returns false for an element it leaves out).  A source
+// with kVec also yields four consecutive elements at once when vec_ok() says its rows are 16-byte aligned
+// (get4: values in x, bit e of the result set when element 4 j4 + e belongs to the multiset).
 struct ScaleSrc {      // values of one scale of one head; `flip` turns bottom-m into top-m of the negated values
+    static constexpr bool kVec = false;
     const float* a;
     float sign;
     __device__ __forceinline__ bool get(int j, float& v) const {
@@ -315,6 +319,7 @@ struct BracketShared {
 };
 
 struct SmemSrc {
+    static constexpr bool kVec = false;
     const float* p;
     __device__ __forceinline__ bool get(int j, float& v) const {
         v = p[j];
@@ -396,31 +401,57 @@ __device__ void block_select_bracket(SelectShared& S, BracketShared<CAP>& X, con
         int cnt = 0;
         float sum = 0.f;
         const int lane = tid & 31;
-        for (int jb = 0; jb < n; jb += 4 * nt) {   // four loads in flight per thread
-            float vv[4];
-            bool vk[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int j = jb + k * nt + tid;
-                vv[k] = 0.f;
-                vk[k] = j < n && src.get(j, vv[k]);
+        // one element: counted (and summed) above the bracket, appended to the list inside it
+        auto consume = [&](float v, bool in) {
+            const bool above = in && v > p_hi;
+            const bool inside = in && !above && v >= p_lo;
+            cnt += above;
+            if (above) sum += v;
+            const unsigned ballot = __ballot_sync(0xffffffffu, inside);
+            if (ballot) {
+                int base = 0;
+                if (lane == 0) base = atomicAdd(&X.cand_n, __popc(ballot));
+                base = __shfl_sync(0xffffffffu, base, 0);
+                const int pos = base + __popc(ballot & ((1u << lane) - 1u));
+                if (inside && pos < kCandCap) X.cand[pos] = v;
             }
+        };
+        bool vec = false;
+        if constexpr (Src::kVec) vec = src.vec_ok() && (n & 3) == 0;
+        if (vec) {
+            if constexpr (Src::kVec) {
+                const int n4 = n >> 2;
+                for (int jb = 0; jb < n4; jb += 4 * nt) {   // sixteen elements in flight per thread
+                    float4 q[4];
+                    unsigned keep[4];
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const float v = vv[k];
-                const bool in = vk[k];
-                const bool above = in && v > p_hi;
-                const bool inside = in && !above && v >= p_lo;
-                cnt += above;
-                if (above) sum += v;
-                const unsigned ballot = __ballot_sync(0xffffffffu, inside);
-                if (ballot) {
-                    int base = 0;
-                    if (lane == 0) base = atomicAdd(&X.cand_n, __popc(ballot));
-                    base = __shfl_sync(0xffffffffu, base, 0);
-                    const int pos = base + __popc(ballot & ((1u << lane) - 1u));
-                    if (inside && pos < kCandCap) X.cand[pos] = v;
+                    for (int k = 0; k < 4; ++k) {
+                        const int j = jb + k * nt + tid;
+                        keep[k] = 0u;
+                        q[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (j < n4) keep[k] = src.get4(j, q[k]);
+                    }
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        consume(q[k].x, (keep[k] & 1u) != 0);
+                        consume(q[k].y, (keep[k] & 2u) != 0);
+                        consume(q[k].z, (keep[k] & 4u) != 0);
+                        consume(q[k].w, (keep[k] & 8u) != 0);
+                    }
                 }
+            }
+        } else {
+            for (int jb = 0; jb < n; jb += 4 * nt) {   // four loads in flight per thread
+                float vv[4];
+                bool vk[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int j = jb + k * nt + tid;
+                    vv[k] = 0.f;
+                    vk[k] = j < n && src.get(j, vv[k]);
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) consume(vv[k], vk[k]);
             }
         }
         cnt = block_sum_int(S, cnt);
@@ -835,19 +866,34 @@ __global__ void __launch_bounds__(kMixThreads) mix_kernel(int N, ScoreParams sp,
 // budget: one CTA per layer group.
 // ------------------------------------------------------------------------------------------
 struct HeadSrc {
+    static constexpr bool kVec = true;
     const float* v;
+    int n;
     __device__ __forceinline__ bool get(int j, float& x) const {
         x = v[j];
         return true;
+    }
+    __device__ __forceinline__ bool vec_ok() const { return (n & 3) == 0 && (reinterpret_cast<uintptr_t>(v) & 15) == 0; }
+    __device__ __forceinline__ unsigned get4(int j4, float4& x) const {
+        x = reinterpret_cast<const float4*>(v)[j4];
+        return 15u;
     }
 };
 struct PoolSrc {       // all (head, token) pairs of a group whose key does not exceed the head's safeguard threshold
     const float* v;    // [H, N]
     const uint32_t* T; // per-head safeguard threshold keys (shared memory)
     int N;
+    static constexpr bool kVec = true;
     __device__ __forceinline__ bool get(int j, float& x) const {
         x = v[j];
         return ord_key(x) <= T[j / N];
+    }
+    __device__ __forceinline__ bool vec_ok() const { return (N & 3) == 0 && (reinterpret_cast<uintptr_t>(v) & 15) == 0; }
+    __device__ __forceinline__ unsigned get4(int j4, float4& x) const {
+        x = reinterpret_cast<const float4*>(v)[j4];
+        const uint32_t t = T[(4 * j4) / N];   // N is a multiple of 4: the four share a head
+        return (ord_key(x.x) <= t ? 1u : 0u) | (ord_key(x.y) <= t ? 2u : 0u) | (ord_key(x.z) <= t ? 4u : 0u) |
+               (ord_key(x.w) <= t ? 8u : 0u);
     }
 };
 
@@ -862,7 +908,7 @@ __global__ void __launch_bounds__(kStatThreads, 4) safeguard_kernel(int N, int n
     if (threadIdx.x == 0) S.ncorr = 0;
     __syncthreads();
     if (n_safe > 0) {
-        HeadSrc src{a_star + (int64_t)u * N};
+        HeadSrc src{a_star + (int64_t)u * N, N};
         block_select_bracket(S, X, src, N, (long long)N, n_safe, 0.f, (float)kBins, status, nullptr);
         if (threadIdx.x == 0) {
             thr[(int64_t)u * 2] = S.theta;
@@ -1037,7 +1083,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(int H, int N, int64_t 
         theta = thr[(int64_t)u * 2];
         q = (int)thr[(int64_t)u * 2 + 1];
     } else {
-        HeadSrc src{v};
+        HeadSrc src{v, N};
         block_select_desc(S, src, N, B, 0.f, (float)kBins, status);
         theta = S.theta;
         q = B - S.gt;
