@@ -1090,14 +1090,23 @@ __global__ void __launch_bounds__(kThreads) select_kernel(int H, int N, int64_t 
         __syncthreads();
     }
     int run_eq = 0, run_sel = 0;
+    // the four scores of the next round are fetched before the scans of this one
+    float nxt[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) nxt[e] = (threadIdx.x * 4 + e < N) ? v[threadIdx.x * 4 + e] : 0.f;
     for (int base = 0; base < N; base += kThreads * 4) {
         const int j0 = base + threadIdx.x * 4;
         uint32_t key[4];
         int eq_cnt = 0;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            key[e] = (j0 + e < N) ? ord_key(v[j0 + e]) : 0u;
+            key[e] = (j0 + e < N) ? ord_key(nxt[e]) : 0u;
             eq_cnt += (j0 + e < N && key[e] == theta);
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int jn = j0 + kThreads * 4 + e;
+            nxt[e] = jn < N ? v[jn] : 0.f;
         }
         int t_eq;
         int tie_rank = run_eq + block_exclusive_scan(eq_cnt, warp_tot, &tot);
