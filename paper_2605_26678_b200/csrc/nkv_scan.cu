@@ -125,15 +125,23 @@ __global__ void anchor_means_kernel(int N, int d, ScoreParams sp, float* __restr
     const int u = blockIdx.x, c = threadIdx.x;
     if (c >= d) return;
     float sum = 0.f, comp = 0.f;
-    for (int t = 0; t < sp.nblocks; ++t) {
-        float* p = mu_e + ((int64_t)u * sp.nblocks + t) * d + c;
-        const float s = *p;
-        const float y = s - comp;
-        const float z = sum + y;
-        comp = (z - sum) - y;
-        sum = z;
-        const int cnt = min(N, (t + 1) * sp.block) - t * sp.block;
-        *p = s / (float)cnt;
+    float* col = mu_e + (int64_t)u * sp.nblocks * d + c;
+    for (int t0 = 0; t0 < sp.nblocks; t0 += 8) {   // eight block sums in flight, then added in block order
+        float s[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) s[k] = t0 + k < sp.nblocks ? col[(int64_t)(t0 + k) * d] : 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int t = t0 + k;
+            if (t < sp.nblocks) {
+                const float y = s[k] - comp;
+                const float z = sum + y;
+                comp = (z - sum) - y;
+                sum = z;
+                const int cnt = min(N, (t + 1) * sp.block) - t * sp.block;
+                col[(int64_t)t * d] = s[k] / (float)cnt;
+            }
+        }
     }
     mu_s[(int64_t)u * d + c] = sum / (float)N;
 }
