@@ -151,6 +151,7 @@ __global__ void __launch_bounds__(128) anchor_norms_kernel(int d, ScoreParams sp
                                                            const float* __restrict__ mu_e, float* __restrict__ inv_s,
                                                            float* __restrict__ inv_e, uint32_t* __restrict__ mm) {
     const int u = blockIdx.x, w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#pragma unroll 4
     for (int t = w - 1; t < sp.nblocks; t += 4) {
         const float* v = (t < 0) ? mu_s + (int64_t)u * d : mu_e + ((int64_t)u * sp.nblocks + t) * d;
         float ss = 0.f;
