@@ -247,30 +247,58 @@ NKV_API int nkv_get_stage_ms(nkv_handle* h, float* ms_out);
 /* Number of kernels this handle has launched since creation. */
 NKV_API int64_t nkv_launch_count(const nkv_handle* h);
 
-/* Choice of the key scan inside nkv_compress.  Sections 2.1-2.3 need two passes over the keys of a
- * head.  lag = 0 (default) runs them as two kernels over the whole cache.  lag in 1..64 runs one
- * kernel that interleaves the passes head by head, the second pass trailing the first by `lag`
- * heads so that it reads the keys from L2 (larger hides the anchor reduction better, smaller keeps
- * fewer keys live in L2).  `l2_hints` non-zero = first-pass loads ask L2 to keep the lines and
- * second-pass loads mark them disposable (interleaved kernel only).  Results do not depend on
- * either setting. */
-NKV_API int nkv_set_scan_options(nkv_handle* h, int lag, int l2_hints);
-
-/* Choice of the kernels that make the two key passes of nkv_compress (Sections 2.1-2.3).  The first
- * pass yields 1/||k||, the block sums of normalised keys and the current-memory anomaly a_c; the
- * second the anomalies a_s and a_e against the global and block anchors.
- * NKV_KEY_PASS_FMA does both with fp32 FMAs on staged key tiles (any supported dtype and d).
- * NKV_KEY_PASS_TENSOR (bf16 keys) forms on the tensor cores what is a contraction: in the first pass
- * (d = 128, W = 64 only, one CTA per head) k_hat_i . S_i and ||S_i||^2 as sums over a band of the
- * keys' Gram matrix, in the second pass (d = 64 or 128) the dots of the keys with the anchors, the
- * fp32 anchors split three ways into bf16.  A pass whose inputs do not allow the tensor form runs the
- * FMA kernel.
- * NKV_KEY_PASS_AUTO (default) takes the tensor form of the second pass when d = 128, and of
- * the first pass when in addition the call's heads, dealt one per SM, keep at least 85 % of the SMs
- * busy over the rounds that takes.
- * The forms agree to fp32 rounding. */
+/*
+ * Choice of the kernels that scan the keys inside nkv_compress (Sections 2.1-2.3).  A head's keys are
+ * touched twice: the first touch yields 1/||k||, the sums of normalised keys per episodic block and the
+ * current-memory anomaly a_c; the second, which needs the anchors of the whole head, yields a_s and a_e.
+ *   NKV_KEY_PASS_AUTO (default), NKV_KEY_PASS_TENSOR: bf16 keys with d = 128, W = 64 and episodic blocks
+ *       of 128 or 256 keys (the paper's schedule gives those for N <= 4127 and N >= 8192) run one
+ *       persistent tcgen05 kernel: k_hat_i . S_i and ||S_i||^2 are sums over a band of the keys' Gram
+ *       matrix, ||k_i||^2 is its diagonal, block sums and anchor dots are skinny products with fp32
+ *       factors split three ways into bf16.  Heads are cut into pieces that all SMs work on, and the
+ *       second touch trails the first closely enough to find the keys in L2.  Other inputs run the FMA
+ *       kernels.
+ *   NKV_KEY_PASS_FMA: fp32 FMAs on staged key tiles, two kernels (any supported dtype and d).
+ * The forms agree to fp32 rounding.
+ */
 enum { NKV_KEY_PASS_AUTO = 0, NKV_KEY_PASS_FMA = 1, NKV_KEY_PASS_TENSOR = 2 };
 NKV_API int nkv_set_key_passes(nkv_handle* h, int mode);
+
+/*
+ * Sections 2.1-2.3 exactly as nkv_compress runs them (same kernels, same choice), with the intermediates
+ * copied out for inspection and tests:
+ *   inv_norm out f32 [G,H,N]     mu_s out f32 [G,H,d]     mu_e out f32 [G,H,nb,d]
+ *   a_raw    out f32 [G,H,3,N]   a_s, a_e, a_c before normalisation
+ *   minmax   out f32 [G,H,6]     lo_s, hi_s, lo_e, hi_e, lo_c, hi_c of the head
+ * `ws` as for nkv_compress.  Enqueues on `stream` and returns.
+ */
+NKV_API int nkv_key_scan(nkv_handle* h, const nkv_tensor* K, const nkv_params* params, float* inv_norm, float* mu_s,
+                         float* mu_e, float* a_raw, float* minmax, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Test and tuning hooks (no counterpart in the paper; results never depend on the tuning values).
+ *   NKV_DEBUG_TILES_PER_PIECE   128-key tiles per piece of a head in the persistent key scan (0: automatic)
+ *   NKV_DEBUG_LAG_ITEMS         first-touch pieces issued ahead of the first second-touch piece (0: automatic)
+ *   NKV_DEBUG_L2_HINTS          bit 0: first-touch loads ask L2 to keep the lines; bit 1: second-touch
+ *                               loads mark them as the first to leave
+ *   NKV_DEBUG_HOLD_HEAD_FLAGS   non-zero: the key scan never raises its "anchors of this head are final"
+ *                               flags, so every bounded wait on one runs out: the call completes with
+ *                               meaningless scores and the device status NKV_ERR_TIMEOUT
+ *   NKV_DEBUG_FLAG_SPIN_LIMIT   polls after which such a wait gives up (0: default)
+ *   NKV_DEBUG_INJECT_HOST_STATUS  value = chunk * 16 + code: nkv_compress_host plants device status `code`
+ *                               in that chunk's status words before reading them back (0 clears)
+ *   NKV_DEBUG_SEPARATE_PASSES   non-zero: NKV_KEY_PASS_TENSOR runs the two-kernel tensor-core form instead
+ */
+enum {
+    NKV_DEBUG_TILES_PER_PIECE = 0,
+    NKV_DEBUG_LAG_ITEMS = 1,
+    NKV_DEBUG_L2_HINTS = 2,
+    NKV_DEBUG_HOLD_HEAD_FLAGS = 3,
+    NKV_DEBUG_FLAG_SPIN_LIMIT = 4,
+    NKV_DEBUG_INJECT_HOST_STATUS = 5,
+    NKV_DEBUG_SEPARATE_PASSES = 6
+};
+NKV_API int nkv_debug_set(nkv_handle* h, int what, int64_t value);
 
 /*
  * nkv_budget for callers that cannot allocate device memory (the paper has no

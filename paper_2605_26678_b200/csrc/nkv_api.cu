@@ -16,12 +16,16 @@ struct nkv_handle {
     int timing;
     int timing_valid;
     int key_pass;     // NKV_KEY_PASS_*: which kernels make the two key passes
-    int scan_lag;     // heads between the two passes of the fused scan (0: use the separate passes)
-    int scan_hints;   // L2 eviction hints on the key loads of the fused scan
+    KeyPassOptions kp;   // scheduling of the single-kernel key scan (zeros: chosen per call)
     cudaEvent_t ev[NKV_NUM_STAGES + 1];
     cudaStream_t copy_streams[2];
     cudaEvent_t slot_done[2];
+    int* chunk_status;   // pinned host copy of every chunk's status words (nkv_compress_host)
+    int inject_status;   // tests: status code planted in chunk `inject_chunk` of nkv_compress_host
+    int inject_chunk;
 };
+
+constexpr int kMaxHostChunks = 4096;
 
 namespace {
 
@@ -72,7 +76,7 @@ Layout make_layout(int64_t units, int64_t N, int64_t d, int64_t nb) {
     L.a_raw = take((size_t)units * 3 * N * 4);
     L.a_star = take((size_t)units * N * 4);
     L.thr = take((size_t)units * 2 * 4);
-    L.ctrl = take(fused_ctrl_bytes(units));
+    L.ctrl = take(keypass_ctrl_bytes(units));
     L.hstat = take(head_stat_bytes(units));
     L.total = o;
     return L;
@@ -94,6 +98,9 @@ int check_tensor(const nkv_tensor* t) {
         return NKV_ERR_INVALID_ARG;
     return NKV_OK;
 }
+
+// Some score-side kernels put the heads on gridDim.y.
+int check_units(int64_t units) { return units > 65535 ? NKV_ERR_UNSUPPORTED : NKV_OK; }
 
 TensorView view_of(const nkv_tensor* t) {
     TensorView v;
@@ -136,6 +143,64 @@ T* at(void* ws, size_t off) { return reinterpret_cast<T*>(reinterpret_cast<unsig
         cudaError_t e__ = (expr);                 \
         if (e__ != cudaSuccess) return NKV_ERR_CUDA; \
     } while (0)
+
+// The two passes over the keys (Sections 2.1-2.3): afterwards the workspace holds 1/||k||, the anchors, the
+// three raw anomalies and their per-head min/max keys.  `mark` is called once between the passes (stage
+// timing).  *sums_only: the anchor arrays hold block sums and the head sum, not means.
+template <typename Mark>
+int key_scan(nkv_handle* h, const TensorView& kv, int dtype, int G, const ScoreParams& sp, void* ws, const Layout& L,
+             cudaStream_t st, Mark&& mark, bool* sums_only) {
+    const int units = G * kv.H, N = kv.N, d = kv.d;
+    int* status = at<int>(ws, L.status);
+    *sums_only = false;
+    if (h->key_pass != NKV_KEY_PASS_FMA && !(h->kp.debug & 2) && keypass_supported(kv, dtype, sp)) {
+        // one persistent kernel makes both passes; the stage mark between them stays empty
+        CU(launch_keypass(kv, G, sp, h->kp, at<float>(ws, L.mu_e), at<float>(ws, L.mu_s), at<float>(ws, L.inv_s),
+                          at<float>(ws, L.inv_e), at<float>(ws, L.inv_norm), at<float>(ws, L.a_raw),
+                          at<uint32_t>(ws, L.mm), at<int>(ws, L.ctrl), status, h->sm_count, st, &h->launches));
+        CU(mark());
+        *sums_only = true;
+    } else if (stream_path_supported(sp)) {
+        // pass A: norms, block sums and the current-memory anomaly; pass B: the two anchor anomalies
+        const bool tensor_ok = h->key_pass == NKV_KEY_PASS_TENSOR && gram_pass_supported(kv, dtype, sp);
+        if (tensor_ok)
+            CU(launch_gram_pass(kv, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm), at<float>(ws, L.a_raw),
+                                at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));
+        else
+            CU(launch_stream_a(kv, dtype, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm),
+                               at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), status, h->sm_count, st,
+                               &h->launches));
+        CU(launch_anchor_means(units, N, d, sp, at<float>(ws, L.mu_e), at<float>(ws, L.mu_s), st, &h->launches));
+        CU(launch_anchor_norms(units, d, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_s),
+                               at<float>(ws, L.inv_e), nullptr, st, &h->launches));
+        CU(mark());
+        if (h->key_pass == NKV_KEY_PASS_TENSOR && anchor_dots_supported(kv, dtype, sp))
+            CU(launch_anchor_dots(kv, G, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm),
+                                  at<float>(ws, L.inv_s), at<float>(ws, L.inv_e), at<float>(ws, L.a_raw),
+                                  at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));
+        else
+            CU(launch_stream_b(kv, dtype, G, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e),
+                               at<float>(ws, L.inv_norm), at<float>(ws, L.inv_s), at<float>(ws, L.inv_e),
+                               at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), status, h->sm_count, st,
+                               &h->launches));
+    } else {
+        CU(launch_anchor_sums(kv, dtype, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm), st, &h->launches));
+        CU(launch_anchor_means(units, N, d, sp, at<float>(ws, L.mu_e), at<float>(ws, L.mu_s), st, &h->launches));
+        CU(launch_anchor_norms(units, d, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_s),
+                               at<float>(ws, L.inv_e), at<uint32_t>(ws, L.mm), st, &h->launches));
+        CU(mark());
+        CU(launch_scan_scores(kv, dtype, G, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e),
+                              at<float>(ws, L.inv_norm), at<float>(ws, L.inv_s), at<float>(ws, L.inv_e),
+                              at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), st, &h->launches));
+    }
+    return NKV_OK;
+}
+
+// ordered min/max keys -> floats (lo_s, hi_s, lo_e, hi_e, lo_c, hi_c per head)
+__global__ void minmax_floats_kernel(int n, const uint32_t* keys, float* out) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = ord_float(keys[i]);
+}
 
 }  // namespace
 
@@ -203,9 +268,14 @@ int64_t nkv_top_count(int64_t N, const nkv_params* p) {
 int nkv_create(nkv_handle** out, int device) {
     if (!out) return NKV_ERR_INVALID_ARG;
     *out = nullptr;
-    int count = 0;
+    int count = 0, previous = 0;
     if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return NKV_ERR_CUDA;
+    CU(cudaGetDevice(&previous));
     CU(cudaSetDevice(device));
+    struct Restore {   // the caller's current device is left as it was
+        int dev;
+        ~Restore() { cudaSetDevice(dev); }
+    } restore{previous};
     nkv_handle* h = new (std::nothrow) nkv_handle();
     if (!h) return NKV_ERR_INVALID_ARG;
     memset(h, 0, sizeof(*h));
@@ -217,11 +287,10 @@ int nkv_create(nkv_handle** out, int device) {
     }
     h->sm_count = prop.multiProcessorCount;
     h->l2_bytes = prop.l2CacheSize;
-    h->scan_lag = 0;   // the separate passes are faster today; see nkv_set_scan_options
-    h->scan_hints = 1;
     h->key_pass = NKV_KEY_PASS_AUTO;
     if (configure_scan_kernels() != cudaSuccess || configure_stream_kernels() != cudaSuccess ||
-        configure_fused_kernels() != cudaSuccess || configure_gram_kernels() != cudaSuccess || configure_dots_kernels() != cudaSuccess || configure_select_kernels() != cudaSuccess) {
+        configure_keypass_kernels() != cudaSuccess || configure_gram_kernels() != cudaSuccess ||
+        configure_dots_kernels() != cudaSuccess || configure_select_kernels() != cudaSuccess) {
         delete h;
         return NKV_ERR_CUDA;
     }
@@ -230,6 +299,10 @@ int nkv_create(nkv_handle** out, int device) {
             delete h;
             return NKV_ERR_CUDA;
         }
+    if (cudaMallocHost(reinterpret_cast<void**>(&h->chunk_status), kMaxHostChunks * 4 * sizeof(int)) != cudaSuccess) {
+        delete h;
+        return NKV_ERR_CUDA;
+    }
     for (int i = 0; i < 2; ++i) {
         if (cudaStreamCreateWithFlags(&h->copy_streams[i], cudaStreamNonBlocking) != cudaSuccess ||
             cudaEventCreateWithFlags(&h->slot_done[i], cudaEventDisableTiming) != cudaSuccess) {
@@ -248,6 +321,7 @@ int nkv_destroy(nkv_handle* h) {
         cudaStreamDestroy(h->copy_streams[i]);
         cudaEventDestroy(h->slot_done[i]);
     }
+    cudaFreeHost(h->chunk_status);
     delete h;
     return NKV_OK;
 }
@@ -284,6 +358,7 @@ int nkv_score(nkv_handle* h, const nkv_tensor* K, const float* mu_s, const float
     if (!h || !mu_s || !mu_e || !inv_norm || !a_star) return NKV_ERR_INVALID_ARG;
     int rc = check_tensor(K);
     if (rc) return rc;
+    if ((rc = check_units(K->G * K->H))) return rc;
     ScoreParams sp;
     if ((rc = resolve_params(params, K->N, &sp))) return rc;
     const int units = (int)(K->G * K->H);
@@ -375,6 +450,7 @@ int nkv_compress(nkv_handle* h, const nkv_tensor* K, const nkv_tensor* V, double
     if (V->G != K->G || V->H != K->H || V->N != K->N) return NKV_ERR_INVALID_ARG;
     if (!(r >= 0.0 && r < 1.0)) return NKV_ERR_INVALID_ARG;
     if (K->H > 64 || K->H * K->N > (int64_t)1 << 30) return NKV_ERR_UNSUPPORTED;
+    if ((rc = check_units(K->G * K->H))) return rc;
     if (((uintptr_t)K_out) % 16 || ((uintptr_t)V_out) % 16) return NKV_ERR_INVALID_ARG;
     ScoreParams sp;
     if ((rc = resolve_params(params, K->N, &sp))) return rc;
@@ -399,56 +475,8 @@ int nkv_compress(nkv_handle* h, const nkv_tensor* K, const nkv_tensor* V, double
 
     CU(cudaMemsetAsync(status, 0, kStatusWords * sizeof(int), st));
     CU(mark());
-    if (h->scan_lag > 0 && fused_scan_supported(sp, K->dtype, d)) {
-        // both key passes in one persistent kernel; the stage mark between them stays empty
-        CU(launch_fused_scan(kv, K->dtype, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.mu_s), at<float>(ws, L.inv_s),
-                             at<float>(ws, L.inv_e), at<float>(ws, L.inv_norm), at<float>(ws, L.a_raw),
-                             at<uint32_t>(ws, L.mm), at<int>(ws, L.ctrl), status, h->sm_count, h->scan_lag,
-                             h->scan_hints, st, &h->launches));
-        CU(mark());
-    } else if (stream_path_supported(sp)) {
-        // pass A: norms, block sums and the current-memory anomaly; pass B: the two anchor anomalies
-        // the tensor-core form walks whole heads, one CTA each: by default it runs when the heads fill
-        // the SMs to at least 85 % over its waves (below that the FMA form, which splits heads, is faster)
-        const bool tensor_ok = gram_pass_supported(kv, K->dtype, sp);
-        const int waves = (units + h->sm_count - 1) / h->sm_count;
-        const bool fills = (double)units >= 0.85 * (double)waves * (double)h->sm_count;
-        const bool use_tensor = h->key_pass == NKV_KEY_PASS_TENSOR
-                                    ? tensor_ok
-                                    : h->key_pass == NKV_KEY_PASS_AUTO && tensor_ok && fills;
-        if (use_tensor)
-            CU(launch_gram_pass(kv, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm), at<float>(ws, L.a_raw),
-                                at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));
-        else
-            CU(launch_stream_a(kv, K->dtype, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm),
-                               at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), status, h->sm_count, st,
-                               &h->launches));
-        CU(launch_anchor_means(units, N, d, sp, at<float>(ws, L.mu_e), at<float>(ws, L.mu_s), st, &h->launches));
-        CU(launch_anchor_norms(units, d, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_s),
-                               at<float>(ws, L.inv_e), nullptr, st, &h->launches));
-        CU(mark());
-        // d = 64 tiles are too small to pay for the per-tile hand-overs: the FMA form is faster there
-        const bool dots_wanted = h->key_pass == NKV_KEY_PASS_TENSOR || (h->key_pass == NKV_KEY_PASS_AUTO && d == 128);
-        if (dots_wanted && anchor_dots_supported(kv, K->dtype, sp))
-            CU(launch_anchor_dots(kv, G, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm),
-                                  at<float>(ws, L.inv_s), at<float>(ws, L.inv_e), at<float>(ws, L.a_raw),
-                                  at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));
-        else
-            CU(launch_stream_b(kv, K->dtype, G, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e),
-                               at<float>(ws, L.inv_norm), at<float>(ws, L.inv_s), at<float>(ws, L.inv_e),
-                               at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), status, h->sm_count, st,
-                               &h->launches));
-    } else {
-        CU(launch_anchor_sums(kv, K->dtype, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm), st,
-                              &h->launches));
-        CU(launch_anchor_means(units, N, d, sp, at<float>(ws, L.mu_e), at<float>(ws, L.mu_s), st, &h->launches));
-        CU(launch_anchor_norms(units, d, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_s),
-                               at<float>(ws, L.inv_e), at<uint32_t>(ws, L.mm), st, &h->launches));
-        CU(mark());
-        CU(launch_scan_scores(kv, K->dtype, G, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e),
-                              at<float>(ws, L.inv_norm), at<float>(ws, L.inv_s), at<float>(ws, L.inv_e),
-                              at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), st, &h->launches));
-    }
+    bool sums_only = false;
+    if ((rc = key_scan(h, kv, K->dtype, G, sp, ws, L, st, mark, &sums_only))) return rc;
     CU(mark());
     CU(launch_head_scores(units, N, sp, at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), a_star, nullptr,
                           at<float>(ws, L.hstat), status, st, &h->launches));
@@ -547,6 +575,11 @@ int nkv_compress_host(nkv_handle* h, const nkv_tensor* Kh, const nkv_tensor* Vh,
             result = rc;
             break;
         }
+        if (h->inject_status && chunk_index == h->inject_chunk &&
+            cudaMemcpyAsync(dWs, &h->inject_status, sizeof(int), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+            result = NKV_ERR_CUDA;
+            break;
+        }
         if (cudaMemcpyAsync((unsigned char*)K_out_host + g0 * grp_out, dKo, gc * grp_out, cudaMemcpyDeviceToHost, st) !=
                 cudaSuccess ||
             cudaMemcpyAsync((unsigned char*)V_out_host + g0 * grp_out, dVo, gc * grp_out, cudaMemcpyDeviceToHost, st) !=
@@ -555,13 +588,19 @@ int nkv_compress_host(nkv_handle* h, const nkv_tensor* Kh, const nkv_tensor* Vh,
                 cudaSuccess ||
             cudaMemcpyAsync(head_offsets_host + g0 * (H + 1), dOff, gc * (H + 1) * 4, cudaMemcpyDeviceToHost, st) !=
                 cudaSuccess ||
-            cudaMemcpyAsync(budgets_host + g0 * H, dBud, gc * H * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
+            cudaMemcpyAsync(budgets_host + g0 * H, dBud, gc * H * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+            (chunk_index < kMaxHostChunks &&
+             cudaMemcpyAsync(h->chunk_status + chunk_index * 4, dWs, 16, cudaMemcpyDeviceToHost, st) != cudaSuccess)) {
             result = NKV_ERR_CUDA;
             break;
         }
     }
     for (int i = 0; i < 2; ++i)
         if (cudaStreamSynchronize(h->copy_streams[i]) != cudaSuccess) result = result ? result : NKV_ERR_CUDA;
+    // every chunk's device status words were copied out before its slot was reused: report the first failure
+    for (int c2 = 0; c2 < chunk_index && c2 < kMaxHostChunks && result == NKV_OK; ++c2)
+        if (h->chunk_status[c2 * 4 + kStatusCode] != 0)
+            result = h->chunk_status[c2 * 4 + kStatusCode] == NKV_ERR_TIMEOUT ? NKV_ERR_TIMEOUT : NKV_ERR_DEVICE_CHECK;
     return result;
 }
 
@@ -592,11 +631,70 @@ int nkv_get_stage_ms(nkv_handle* h, float* ms_out) {
 
 int64_t nkv_launch_count(const nkv_handle* h) { return h ? h->launches : -1; }
 
-int nkv_set_scan_options(nkv_handle* h, int lag, int l2_hints) {
-    if (!h || lag < 0 || lag > 64) return NKV_ERR_INVALID_ARG;
-    h->scan_lag = lag;
-    h->scan_hints = l2_hints ? 1 : 0;
+int nkv_key_scan(nkv_handle* h, const nkv_tensor* K, const nkv_params* params, float* inv_norm, float* mu_s,
+                 float* mu_e, float* a_raw, float* minmax, void* ws, size_t ws_bytes, void* stream) {
+    if (!h || !inv_norm || !mu_s || !mu_e || !a_raw || !minmax) return NKV_ERR_INVALID_ARG;
+    int rc = check_tensor(K);
+    if (rc) return rc;
+    if ((rc = check_units(K->G * K->H))) return rc;
+    ScoreParams sp;
+    if ((rc = resolve_params(params, K->N, &sp))) return rc;
+    const int G = (int)K->G, N = (int)K->N, d = (int)K->d, units = (int)(K->G * K->H);
+    const Layout L = make_layout(units, N, d, sp.nblocks);
+    if ((rc = check_ws(ws, ws_bytes, L.total))) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    CU(cudaMemsetAsync(at<int>(ws, L.status), 0, kStatusWords * sizeof(int), st));
+    bool sums_only = false;
+    auto no_mark = []() -> cudaError_t { return cudaSuccess; };
+    if ((rc = key_scan(h, view_of(K), K->dtype, G, sp, ws, L, st, no_mark, &sums_only))) return rc;
+    if (sums_only) {
+        CU(launch_keypass_means(units, N, sp, at<float>(ws, L.mu_e), at<float>(ws, L.mu_s), mu_e, mu_s, st,
+                                &h->launches));
+    } else {
+        CU(cudaMemcpyAsync(mu_s, at<float>(ws, L.mu_s), (size_t)units * d * 4, cudaMemcpyDeviceToDevice, st));
+        CU(cudaMemcpyAsync(mu_e, at<float>(ws, L.mu_e), (size_t)units * sp.nblocks * d * 4, cudaMemcpyDeviceToDevice,
+                           st));
+    }
+    CU(cudaMemcpyAsync(inv_norm, at<float>(ws, L.inv_norm), (size_t)units * N * 4, cudaMemcpyDeviceToDevice, st));
+    CU(cudaMemcpyAsync(a_raw, at<float>(ws, L.a_raw), (size_t)units * 3 * N * 4, cudaMemcpyDeviceToDevice, st));
+    minmax_floats_kernel<<<(units * 6 + 255) / 256, 256, 0, st>>>(units * 6, at<uint32_t>(ws, L.mm), minmax);
+    ++h->launches;
+    CU(cudaGetLastError());
     return NKV_OK;
+}
+
+int nkv_debug_set(nkv_handle* h, int what, int64_t value) {
+    if (!h) return NKV_ERR_INVALID_ARG;
+    switch (what) {
+        case NKV_DEBUG_TILES_PER_PIECE:
+            if (value < 0 || value > 64) return NKV_ERR_INVALID_ARG;
+            h->kp.tiles_per_piece = (int)value;
+            return NKV_OK;
+        case NKV_DEBUG_LAG_ITEMS:
+            if (value < 0) return NKV_ERR_INVALID_ARG;
+            h->kp.lag_items = value;
+            return NKV_OK;
+        case NKV_DEBUG_L2_HINTS:
+            if (value < 0 || value > 3) return NKV_ERR_INVALID_ARG;
+            h->kp.hints = (int)value;
+            return NKV_OK;
+        case NKV_DEBUG_HOLD_HEAD_FLAGS:
+            h->kp.debug = (h->kp.debug & ~1) | (value ? 1 : 0);
+            return NKV_OK;
+        case NKV_DEBUG_FLAG_SPIN_LIMIT:
+            if (value < 0 || value > (1 << 24)) return NKV_ERR_INVALID_ARG;
+            h->kp.flag_spin_limit = (int)value;
+            return NKV_OK;
+        case NKV_DEBUG_INJECT_HOST_STATUS:   // value = chunk * 16 + status code (0 clears)
+            h->inject_status = (int)(value & 15);
+            h->inject_chunk = (int)(value >> 4);
+            return NKV_OK;
+        case NKV_DEBUG_SEPARATE_PASSES:
+            h->kp.debug = (h->kp.debug & ~2) | (value ? 2 : 0);
+            return NKV_OK;
+        default:
+            return NKV_ERR_INVALID_ARG;
+    }
 }
 
 int nkv_set_key_passes(nkv_handle* h, int mode) {

@@ -145,14 +145,26 @@ cudaError_t configure_dots_kernels();
 cudaError_t launch_anchor_dots(const TensorView& K, int G, const ScoreParams& sp, const float* mu_s, const float* mu_e,
                                const float* inv_norm, const float* inv_s, const float* inv_e, float* a_raw,
                                uint32_t* mm, int* status, int sm_count, cudaStream_t stream, int64_t* launches);
-// fused two-pass scan (one persistent kernel; the second pass reads the keys from L2)
-bool fused_scan_supported(const ScoreParams& sp, int dtype, int d);
-size_t fused_ctrl_bytes(int64_t units);
-cudaError_t configure_fused_kernels();
-cudaError_t launch_fused_scan(const TensorView& K, int dtype, int G, const ScoreParams& sp, float* block_sums,
-                              float* mu_s, float* inv_s, float* inv_e, float* inv_norm, float* a_raw, uint32_t* mm,
-                              int* ctrl, int* status, int sm_count, int lag, int hints, cudaStream_t stream,
-                              int64_t* launches);
+// both key passes in one persistent tensor-core kernel (bf16 keys, d = 128, blocks of whole 128-key tiles);
+// the second touch of a key finds it in L2.  Anchors come out as sums (block_sums, head_sum) with the
+// reciprocals of their norms; launch_keypass_means turns them into the means mu_e, mu_s.
+struct KeyPassOptions {
+    int tiles_per_piece;   // 0: chosen from the call's size
+    long long lag_items;   // 0: chosen from the grid
+    int hints;             // bit 0 / bit 1: L2 eviction hints on first- / second-touch loads
+    int debug;             // bit 0: never raise the head flags (makes the bounded flag wait run out)
+    int flag_spin_limit;   // 0: default
+};
+bool keypass_supported(const TensorView& K, int dtype, const ScoreParams& sp);
+size_t keypass_ctrl_bytes(int64_t units);
+cudaError_t configure_keypass_kernels();
+cudaError_t launch_keypass(const TensorView& K, int G, const ScoreParams& sp, const KeyPassOptions& opt,
+                           float* block_sums, float* head_sum, float* inv_s, float* inv_e, float* inv_norm,
+                           float* a_raw, uint32_t* mm, int* ctrl, int* status, int sm_count, cudaStream_t stream,
+                           int64_t* launches);
+cudaError_t launch_keypass_means(int units, int N, const ScoreParams& sp, const float* block_sums,
+                                 const float* head_sum, float* mu_e, float* mu_s, cudaStream_t stream,
+                                 int64_t* launches);
 cudaError_t configure_select_kernels();
 cudaError_t configure_scan_kernels();
 cudaError_t configure_stream_kernels();

@@ -36,7 +36,8 @@ EXPORTS = (
     "nkv_keep_per_head", "nkv_safeguard_count", "nkv_top_count", "nkv_create", "nkv_destroy",
     "nkv_workspace_bytes", "nkv_anchors", "nkv_score", "nkv_budget", "nkv_select", "nkv_compact",
     "nkv_compress", "nkv_host_staging_bytes", "nkv_compress_host", "nkv_last_device_status",
-    "nkv_set_timing", "nkv_get_stage_ms", "nkv_launch_count", "nkv_budget_static", "nkv_set_scan_options", "nkv_set_key_passes",
+    "nkv_set_timing", "nkv_get_stage_ms", "nkv_launch_count", "nkv_budget_static", "nkv_set_key_passes",
+    "nkv_key_scan", "nkv_debug_set",
 )
 
 
@@ -111,7 +112,8 @@ def load_library():
     L.nkv_get_stage_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     L.nkv_launch_count.argtypes = [vp]
     L.nkv_launch_count.restype = i64
-    L.nkv_set_scan_options.argtypes = [vp, ctypes.c_int, ctypes.c_int]
+    L.nkv_key_scan.argtypes = [vp, tp, pp, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.nkv_debug_set.argtypes = [vp, ctypes.c_int, i64]
     L.nkv_set_key_passes.argtypes = [vp, ctypes.c_int]
     L.nkv_budget_static.argtypes = [vp, i64, i64, i64, dbl, pp, vp, vp]
     _lib = L
@@ -429,7 +431,32 @@ def nkv_set_key_passes(mode: str = "auto", h: Optional[Handle] = None) -> None:
     _check(h.lib.nkv_set_key_passes(h.h, KEY_PASS[mode]), "nkv_set_key_passes")
 
 
-def nkv_set_scan_options(lag: int = 0, l2_hints: bool = True, h: Optional[Handle] = None) -> None:
-    """lag = heads between the two key passes of the fused scan (0: separate kernels); see nkv.h."""
+DEBUG = {"tiles_per_piece": 0, "lag_items": 1, "l2_hints": 2, "hold_head_flags": 3, "flag_spin_limit": 4,
+         "inject_host_status": 5, "separate_passes": 6}
+
+
+def nkv_debug_set(what: str, value: int, h: Optional[Handle] = None) -> None:
+    """Test and tuning hooks of the library (see nkv.h); results never depend on the tuning values."""
     h = h or handle()
-    _check(h.lib.nkv_set_scan_options(h.h, int(lag), 1 if l2_hints else 0), "nkv_set_scan_options")
+    _check(h.lib.nkv_debug_set(h.h, DEBUG[what], int(value)), "nkv_debug_set")
+
+
+def nkv_key_scan(K: torch.Tensor, params: Optional[Params] = None, ws: Optional[torch.Tensor] = None,
+                 h: Optional[Handle] = None):
+    """The key scan of nkv_compress with its intermediates copied out:
+    -> (inv_norm [G,H,N], mu_s [G,H,d], mu_e [G,H,nb,d], a_raw [G,H,3,N], minmax [G,H,6])"""
+    h = h or handle()
+    params = params or nkv_default_params()
+    G, H, N, d = K.shape
+    nb = nkv_num_blocks(N, params)
+    f32 = dict(dtype=torch.float32, device=K.device)
+    inv_norm = torch.empty((G, H, N), **f32)
+    mu_s = torch.empty((G, H, d), **f32)
+    mu_e = torch.empty((G, H, nb, d), **f32)
+    a_raw = torch.empty((G, H, 3, N), **f32)
+    minmax = torch.empty((G, H, 6), **f32)
+    ws = ws if ws is not None else alloc_workspace(K, params, h)
+    kt = _tensor(K)
+    _check(h.lib.nkv_key_scan(h.h, ctypes.byref(kt), ctypes.byref(params), _p(inv_norm), _p(mu_s), _p(mu_e),
+                              _p(a_raw), _p(minmax), _p(ws), ws.numel(), _stream()), "nkv_key_scan")
+    return inv_norm, mu_s, mu_e, a_raw, minmax
