@@ -55,8 +55,6 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--scan-lag", type=int, default=None, help="heads between the two key passes (library default if unset)")
-    ap.add_argument("--scan-hints", type=int, default=1, help="L2 eviction hints on the key loads (0/1)")
     ap.add_argument("--key-passes", default="auto", choices=["auto", "fma", "tensor"],
                     help="kernels of the two key passes (library default: auto)")
     return ap.parse_args()
@@ -250,8 +248,6 @@ def run_nkv(args, cfg, r):
     ws = nkv.alloc_workspace(K, params)
     out = nkv.alloc_outputs(K, V, r)
     h = nkv.handle(local)
-    if args.scan_lag is not None:
-        nkv.nkv_set_scan_options(args.scan_lag, bool(args.scan_hints), h)
     nkv.nkv_set_key_passes(args.key_passes, h)
 
     def step():

@@ -278,7 +278,6 @@ NKV_API int nkv_key_scan(nkv_handle* h, const nkv_tensor* K, const nkv_params* p
 /*
  * Test and tuning hooks (no counterpart in the paper; results never depend on the tuning values).
  *   NKV_DEBUG_TILES_PER_PIECE   128-key tiles per piece of a head in the persistent key scan (0: automatic)
- *   NKV_DEBUG_LAG_ITEMS         first-touch pieces issued ahead of the first second-touch piece (0: automatic)
  *   NKV_DEBUG_L2_HINTS          bit 0: first-touch loads ask L2 to keep the lines; bit 1: second-touch
  *                               loads mark them as the first to leave
  *   NKV_DEBUG_HOLD_HEAD_FLAGS   non-zero: the key scan never raises its "anchors of this head are final"
@@ -291,7 +290,6 @@ NKV_API int nkv_key_scan(nkv_handle* h, const nkv_tensor* K, const nkv_params* p
  */
 enum {
     NKV_DEBUG_TILES_PER_PIECE = 0,
-    NKV_DEBUG_LAG_ITEMS = 1,
     NKV_DEBUG_L2_HINTS = 2,
     NKV_DEBUG_HOLD_HEAD_FLAGS = 3,
     NKV_DEBUG_FLAG_SPIN_LIMIT = 4,

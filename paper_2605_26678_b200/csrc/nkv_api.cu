@@ -2,6 +2,7 @@
 #include <math.h>
 #include <new>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "nkv_common.cuh"
@@ -55,7 +56,7 @@ int64_t keep_count(int64_t N, double r) { return (int64_t)floor((1.0 - r) * (dou
 
 // Workspace carving shared by every entry point.
 struct Layout {
-    size_t status, inv_norm, mu_s, mu_e, inv_s, inv_e, mm, a_raw, a_star, thr, ctrl, hstat, total;
+    size_t status, inv_norm, mu_s, mu_e, inv_s, inv_e, mm, a_raw, a_star, thr, ctrl, tsum, hstat, total;
 };
 
 Layout make_layout(int64_t units, int64_t N, int64_t d, int64_t nb) {
@@ -77,6 +78,7 @@ Layout make_layout(int64_t units, int64_t N, int64_t d, int64_t nb) {
     L.a_star = take((size_t)units * N * 4);
     L.thr = take((size_t)units * 2 * 4);
     L.ctrl = take(keypass_ctrl_bytes(units));
+    L.tsum = d == 128 ? take(keypass_tile_sum_bytes(units, N)) : o;
     L.hstat = take(head_stat_bytes(units));
     L.total = o;
     return L;
@@ -138,10 +140,17 @@ int check_ws(const void* ws, size_t ws_bytes, size_t need) {
 template <typename T>
 T* at(void* ws, size_t off) { return reinterpret_cast<T*>(reinterpret_cast<unsigned char*>(ws) + off); }
 
-#define CU(expr)                                  \
-    do {                                          \
-        cudaError_t e__ = (expr);                 \
-        if (e__ != cudaSuccess) return NKV_ERR_CUDA; \
+// With NKV_TRACE set in the environment a failing CUDA call is named on stderr.
+int cuda_failed(cudaError_t e, const char* what, int line) {
+    static const bool trace = getenv("NKV_TRACE") != nullptr;
+    if (trace) fprintf(stderr, "nkv: %s (nkv_api.cu:%d): %s\n", what, line, cudaGetErrorString(e));
+    return NKV_ERR_CUDA;
+}
+
+#define CU(expr)                                                     \
+    do {                                                             \
+        cudaError_t e__ = (expr);                                    \
+        if (e__ != cudaSuccess) return cuda_failed(e__, #expr, __LINE__); \
     } while (0)
 
 // The two passes over the keys (Sections 2.1-2.3): afterwards the workspace holds 1/||k||, the anchors, the
@@ -155,7 +164,7 @@ int key_scan(nkv_handle* h, const TensorView& kv, int dtype, int G, const ScoreP
     *sums_only = false;
     if (h->key_pass != NKV_KEY_PASS_FMA && !(h->kp.debug & 2) && keypass_supported(kv, dtype, sp)) {
         // one persistent kernel makes both passes; the stage mark between them stays empty
-        CU(launch_keypass(kv, G, sp, h->kp, at<float>(ws, L.mu_e), at<float>(ws, L.mu_s), at<float>(ws, L.inv_s),
+        CU(launch_keypass(kv, G, sp, h->kp, at<float>(ws, L.tsum), at<float>(ws, L.mu_e), at<float>(ws, L.mu_s), at<float>(ws, L.inv_s),
                           at<float>(ws, L.inv_e), at<float>(ws, L.inv_norm), at<float>(ws, L.a_raw),
                           at<uint32_t>(ws, L.mm), at<int>(ws, L.ctrl), status, h->sm_count, st, &h->launches));
         CU(mark());
@@ -669,10 +678,6 @@ int nkv_debug_set(nkv_handle* h, int what, int64_t value) {
         case NKV_DEBUG_TILES_PER_PIECE:
             if (value < 0 || value > 64) return NKV_ERR_INVALID_ARG;
             h->kp.tiles_per_piece = (int)value;
-            return NKV_OK;
-        case NKV_DEBUG_LAG_ITEMS:
-            if (value < 0) return NKV_ERR_INVALID_ARG;
-            h->kp.lag_items = value;
             return NKV_OK;
         case NKV_DEBUG_L2_HINTS:
             if (value < 0 || value > 3) return NKV_ERR_INVALID_ARG;

@@ -150,18 +150,18 @@ cudaError_t launch_anchor_dots(const TensorView& K, int G, const ScoreParams& sp
 // reciprocals of their norms; launch_keypass_means turns them into the means mu_e, mu_s.
 struct KeyPassOptions {
     int tiles_per_piece;   // 0: chosen from the call's size
-    long long lag_items;   // 0: chosen from the grid
     int hints;             // bit 0 / bit 1: L2 eviction hints on first- / second-touch loads
     int debug;             // bit 0: never raise the head flags (makes the bounded flag wait run out)
     int flag_spin_limit;   // 0: default
 };
 bool keypass_supported(const TensorView& K, int dtype, const ScoreParams& sp);
 size_t keypass_ctrl_bytes(int64_t units);
+size_t keypass_tile_sum_bytes(int64_t units, int64_t N);
 cudaError_t configure_keypass_kernels();
 cudaError_t launch_keypass(const TensorView& K, int G, const ScoreParams& sp, const KeyPassOptions& opt,
-                           float* block_sums, float* head_sum, float* inv_s, float* inv_e, float* inv_norm,
-                           float* a_raw, uint32_t* mm, int* ctrl, int* status, int sm_count, cudaStream_t stream,
-                           int64_t* launches);
+                           float* tile_sums, float* block_sums, float* head_sum, float* inv_s, float* inv_e,
+                           float* inv_norm, float* a_raw, uint32_t* mm, int* ctrl, int* status, int sm_count,
+                           cudaStream_t stream, int64_t* launches);
 cudaError_t launch_keypass_means(int units, int N, const ScoreParams& sp, const float* block_sums,
                                  const float* head_sum, float* mu_e, float* mu_s, cudaStream_t stream,
                                  int64_t* launches);

@@ -1,8 +1,8 @@
-// Both key passes in one persistent kernel on the tensor cores (bf16 keys, d = 128, window W = 64, episodic
-// blocks of 128 or 256 keys).
+// The key scan (Sections 2.1-2.3) as one persistent kernel on the tensor cores: bf16 keys, d = 128, window
+// W = 64, episodic blocks of 128 or 256 keys.
 //
-// What is computed (Sections 2.1-2.3): w_i = 1/||k_i||, the sum of the normalised keys of every episodic
-// block and of the whole head, and the three anomalies
+// What is computed: w_i = 1/||k_i||, the sum of the normalised keys of every episodic block and of the whole
+// head, and the three anomalies
 //     a_c(i) = -cos(k_hat_i, mu_c(i))     mu_c(i) = mean of the last W normalised keys
 //     a_e(i) = -cos(k_hat_i, mu_e(block of i))
 //     a_s(i) = -cos(k_hat_i, mu_s)
@@ -14,7 +14,7 @@
 // g_jl: sums over a band of the keys' Gram matrix.  Per tile the tensor core forms
 //     D      = K[tile rows] x K[64 rows before .. tile rows]^T     128 x 192, fp32 in tensor memory
 //     corner = K[previous tile rows] x K[first 64 tile rows]^T     128 x 64 (its last 64 rows are used)
-//     bsum   = K[tile rows]^T x [w hi | w mid | w lo]              128 (channels) x 16: sum_i w_i k_i
+//     tsum   = K[tile rows]^T x [w hi | w mid | w lo]              128 (channels) x 16: sum_i w_i k_i
 // bf16 products are exact in fp32 and the accumulation is fp32, so D holds fp32 dot products; w enters the
 // last product as three bf16 numbers that add up to its 24 mantissa bits.  ||k_i||^2 is the diagonal of D.
 // Row r of D gives the backward band sum c_r (k_hat . S) and, with the corner that arrives one tile later,
@@ -24,23 +24,24 @@
 // block of the previous tile's last rows).  No quantity looks ahead of the keys already loaded.
 //
 // Second touch ("B tiles"): the dots of 128 keys with the head sum and with the block sum are one product
-// [128 x d] x [d x 16] (both anchors split three ways into bf16).  It needs the sums over the whole head, so
-// it trails the first touch; the work is ordered so that it finds the keys in L2.
+// [128 x d] x [d x 16] (both anchors split three ways into bf16).  It needs the sums over the whole head,
+// so it trails the first touch, closely enough to find the keys in L2.
 //
-// Work is cut into items: a piece of a head (a few tiles, whole blocks) for the first touch or for the
-// second.  One global sequence interleaves them, second-touch items trailing first-touch items by a fixed
-// number of items; CTAs (one per SM) draw from it with an atomic counter.  A first-touch item starts with a
-// "halo" tile of the 128 rows before the piece, which yields the restart value, the norms and the forward
-// sums the first real tile needs.  The CTA that completes the last piece of a head sums its block sums,
-// takes the norms of the anchors and raises the head's flag; a second-touch item waits (bounded) for that
-// flag.  Every item depends only on items earlier in the sequence, which running CTAs hold, so the waits
-// end.  A flag wait that runs out records NKV_ERR_TIMEOUT and goes on with whatever the buffers hold.
+// A head is cut into pieces of a few tiles (whole blocks).  Every CTA (one per SM) runs two independent
+// pipelines, each drawing pieces from its own global counter: the first-touch pipeline never waits for the
+// other one; a second-touch piece waits (bounded) for the flag of its head.  A first-touch piece starts
+// with a "halo" tile of the 128 rows before it, which yields the restart value, the norms and the forward
+// sums its first real tile needs.  Per-tile sums of normalised keys go to global memory; the CTA that
+// completes the last piece of a head adds them up per block and per head, takes the norms of those anchors
+// and raises the head's flag.  A flag wait that runs out records NKV_ERR_TIMEOUT and the call goes on with
+// whatever the buffers hold.
 //
-// Warp roles in a CTA: 4 warps backward sums, norms and block sums; 4 warps forward sums, prefix scan and
-// a_c; 4 warps that turn second-touch accumulators into a_s, a_e; 4 warps that build the split anchors;
-// one TMA producer thread (also draws the items); one MMA issuer thread.  Keys are staged by TMA in a ring
-// of 128-row slots (64-row slabs, 128-byte swizzle); hand-overs are mbarriers and two named barriers per
-// tile; every wait is bounded.
+// Warps of a CTA: two teams of 8 warps take the first-touch tiles in turn (4 warps: norms, backward sums,
+// tile sums; 4 warps: forward sums, prefix scan, a_c), so two tiles are in flight and a team's chain of
+// tensor-memory round trips overlaps the other team's; 4 warps build the split anchors of the second touch
+// and turn its accumulators into a_s, a_e; one TMA producer thread and one MMA issuer thread per pipeline.
+// Keys are staged by TMA in two rings of 128-row slots (64-row slabs, 128-byte swizzle); hand-overs are
+// mbarriers and named barriers inside a team; every wait is bounded.
 #include "nkv_sm100.cuh"
 
 namespace nkv {
@@ -52,76 +53,88 @@ using namespace sm100;
 constexpr int kD = 128;                       // head dimension
 constexpr int kTile = 128;                    // keys per tile
 constexpr int kSlabRows = 64;                 // rows per staged slab
-constexpr int kSlots = 5;                     // tiles staged at once
-constexpr int kSlabs = 2 * kSlots + 1;        // slab 0 is a copy of the slab before slot 0's tile
+constexpr int kSlotsA = 3;                    // first-touch tiles staged at once
+constexpr int kSlotsB = 2;                    // second-touch tiles staged at once
+constexpr int kSlabsA = 2 * kSlotsA + 1;      // slab 0 is a copy of the slab before slot 0's tile
+constexpr int kSlabs = kSlabsA + 2 * kSlotsB;
 constexpr int kSlabHalfBytes = kSlabRows * 128;            // one 64-column half of a slab
 constexpr int kHalfBytes = kSlabs * kSlabHalfBytes;        // all slabs of one half are contiguous
 constexpr int kRingBytes = 2 * kHalfBytes;
 constexpr int kOperandBytes = 2 * 16 * 128;   // a 16-row operand of 128 columns: two swizzled halves
-constexpr int kQueue = 4;                     // item descriptors in flight inside a CTA
-constexpr int kWRing = 512, kWMask = kWRing - 1;   // per-row scalars of the last four first-touch tiles
+constexpr int kQueue = 4;                     // piece descriptors in flight per pipeline
+constexpr int kHist = 8;                      // first-touch tiles whose hand-over state is kept
+constexpr int kWRing = kHist * kTile, kWMask = kWRing - 1;   // per-row scalars of those tiles
+constexpr int kPrefetchTiles = 3;             // first-touch tiles requested from DRAM into L2 ahead of their slot
 
 // tensor-memory columns
-constexpr uint32_t kColMain0 = 0, kColCorner = 192, kColMain1 = 256, kColBsum = 448, kColDots = 480;
+constexpr uint32_t kColMain0 = 0, kColCorner = 192, kColMain1 = 256, kColTsum = 448, kColDots = 480;
 constexpr uint32_t kTmemCols = 512;
 
-constexpr int kBandThreads = 256;             // warps 0-3 backward, 4-7 forward
-constexpr int kEpiWarp0 = 8, kPrepWarp0 = 12, kProducerWarp = 16, kMmaWarp = 17;
-constexpr int kThreads = 18 * 32;
-constexpr int kConsumerWarps = 17;            // every warp but the producer reads the item queue
-constexpr int kBarBand = 1, kBarFwd = 2;      // named barriers
-
-enum { kItemA = 0, kItemB = 1, kItemEnd = 2 };
+// warps: team 0 = 0..7, team 1 = 8..15 (first four backward, last four forward), second touch 16..19,
+// then one thread each of warps 20..23
+constexpr int kTeamThreads = 256;
+constexpr int kBWarp0 = 16, kProdAWarp = 20, kProdBWarp = 21, kMmaAWarp = 22, kMmaBWarp = 23;
+constexpr int kThreads = 24 * 32;
+constexpr int kConsumersA = 17, kConsumersB = 5;   // warps (or single threads) that read a pipeline's queue
 
 struct Item {
-    int kind, u, g, h, row0, ntiles;
+    int end, u, g, h, row0, ntiles;
 };
 
 struct KeyPassArgs {
     ScoreParams sp;
     int units, H, N;
     int tiles_per_piece, pieces;       // pieces per head
-    long long lag_items;               // first-touch items ahead of the first second-touch item
     int hints;                         // bit 0: keep first-touch lines in L2, bit 1: second-touch lines leave first
     int debug;                         // bit 0 (tests): the head flags are never raised
     uint32_t flag_spin_limit;
-    float* block_sums;                 // [units][nblocks][d] sums of normalised keys
+    float* tile_sums;                  // [units][tiles][d] sums of normalised keys per 128-key tile
+    float* block_sums;                 // [units][nblocks][d]
     float* head_sum;                   // [units][d]
     float* inv_s;                      // [units]          1 / ||head sum||
     float* inv_e;                      // [units][nblocks] 1 / ||block sum||
     float* inv_norm;                   // [units][N]
     float* a_raw;                      // [units][3][N]
     uint32_t* mm;                      // [units][6] ordered min/max keys
-    unsigned long long* next_item;
+    unsigned long long* next_a;        // pieces handed out, first touch
+    unsigned long long* next_b;        // pieces handed out, second touch
     int* head_count;                   // [units] first-touch pieces completed
     int* head_ready;                   // [units] anchors final
     int* status;
 };
 
+struct alignas(16) TeamSmem {
+    float c[kTile];              // backward band sums of the team's tile
+    float fcur[64];              // forward band sums of the tile's rows 0..63
+    float fprev[64];             // forward band sums of the previous tile's rows 64..127
+    float wtot[4];               // per-warp totals of the tile's prefix sum
+    float red[8];                // min/max reduction at the end of a piece
+    float fin[2][kD];            // column sums of the finaliser
+    int fin_flag;
+};
+
 struct Smem {
     float w[kWRing];             // 1/||k|| by row (0 outside the head)
     float g[kWRing];             // g_ii by row
-    float c[2][kTile];           // backward band sums of a tile
-    float fcur[2][64];           // forward band sums of the tile's rows 0..63
-    float fprev[2][64];          // forward band sums of the previous tile's rows 64..127
-    float apart[2][2];           // per-warp parts of the next tile's restart value
-    float wtot[2][4];            // per-warp totals of a tile's prefix sum
-    float red[8];                // min/max reduction at the end of an item
-    float fin[2][kD];            // column sums of the finaliser
-    Item items[kQueue];
-    uint64_t qfull[kQueue], qfree[kQueue];
-    uint64_t full[kSlots];       // slot landed
-    uint64_t sfree[kSlots];      // slot no longer read
-    uint64_t tfull[2], tempty[2];       // Gram accumulators
+    float carry[kHist][64];          // rows 64..127 of a tile: forward sums over the tile's own columns (unscaled)
+    float apart[kHist][2];           // per-warp parts of the next tile's restart value
+    TeamSmem team[2];
+    Item qa[kQueue], qb[kQueue];
+    uint64_t qa_full[kQueue], qa_free[kQueue], qb_full[kQueue], qb_free[kQueue];
+    uint64_t full_a[kSlotsA], free_a[kSlotsA];   // first-touch slot landed / no longer read
+    uint64_t full_b[kSlotsB], free_b[kSlotsB];
+    uint64_t tfull[2], tempty[2];       // Gram accumulators (one per team)
     uint64_t cempty;                    // corner accumulator read
+    uint64_t wpub[kHist];                   // norms of a tile are in the ring
+    uint64_t spub[kHist];                   // carry and restart parts of a tile are written
+    uint64_t done[kHist];                   // every global write of a tile has been issued and fenced
     uint64_t wsready[2];                // split norms written
-    uint64_t bsfull[2], bsempty[2];     // block-sum accumulators
+    uint64_t tsfull[2], tsempty[2];     // tile-sum accumulators
     uint64_t rready[2], rfree[2];       // split anchors
     uint64_t dfull[2], dempty[2];       // second-touch accumulators
-    uint64_t drain;
+    uint64_t drain_a, drain_b;
     uint32_t tmem_base;
     int abort;
-    int fin_flag;
 };
 constexpr size_t kSmemBytes = 1024 + kRingBytes + 4 * kOperandBytes + sizeof(Smem);
 
@@ -133,56 +146,38 @@ struct Waiter {
 // Bounded wait that also leaves when another role of the CTA has given up.
 __device__ __forceinline__ bool bwait(uint64_t* bar, uint32_t parity, const Waiter& wt, int where) {
     if (mbar_try_wait(bar, parity)) return true;
-    uint32_t ns = 32;
     for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*wt.abort) return false;
-        __nanosleep(ns);
-        if (ns < 256) ns <<= 1;
+        if (spin >= 8) __nanosleep(spin < 64 ? 32 : 128);
     }
     set_status(wt.status, NKV_ERR_TIMEOUT, where);
     *wt.abort = 1;
     return false;
 }
 
-// Item `cnt` of the CTA's queue.  kWarp: the whole warp calls (one release per warp); else one thread.
+// Descriptor `cnt` of a pipeline's queue.  kWarp: the whole warp calls (one release per warp); else one thread.
 template <bool kWarp>
-__device__ __forceinline__ bool get_item(Smem* s, long long cnt, Item& it, const Waiter& wt, int where) {
-    const int q = (int)(cnt & (kQueue - 1));
-    if (!bwait(&s->qfull[q], (uint32_t)((cnt / kQueue) & 1), wt, where)) return false;
-    it = s->items[q];
+__device__ __forceinline__ bool get_item(const Item* q, uint64_t* qfull, uint64_t* qfree, long long cnt, Item& it,
+                                         const Waiter& wt, int where) {
+    const int k = (int)(cnt & (kQueue - 1));
+    if (!bwait(&qfull[k], (uint32_t)((cnt / kQueue) & 1), wt, where)) return false;
+    it = q[k];
     if (kWarp) {
         __syncwarp();
-        if ((threadIdx.x & 31) == 0) mbar_arrive(&s->qfree[q]);
+        if ((threadIdx.x & 31) == 0) mbar_arrive(&qfree[k]);
     } else {
-        mbar_arrive(&s->qfree[q]);
+        mbar_arrive(&qfree[k]);
     }
     return true;
 }
 
-// Place `pos` of the global sequence: the first `lag` places are first-touch items, then second- and
-// first-touch items alternate until the first-touch items are used up, then the rest.
-__device__ __forceinline__ Item decode_item(long long pos, const KeyPassArgs& p) {
+// Piece `idx` of the call: heads in order, pieces of a head in order.
+__device__ __forceinline__ Item decode_item(long long idx, const KeyPassArgs& p) {
     Item it;
-    it.kind = kItemEnd;
+    it.end = idx >= (long long)p.units * p.pieces;
     it.u = it.g = it.h = it.row0 = it.ntiles = 0;
-    const long long UP = (long long)p.units * p.pieces;
-    if (pos >= 2 * UP) return it;
-    const long long L = p.lag_items < UP ? p.lag_items : UP;
-    long long idx;
-    if (pos < L) {
-        it.kind = kItemA;
-        idx = pos;
-    } else {
-        const long long t = pos - L, RA = UP - L;
-        if (t < 2 * RA) {
-            it.kind = (t & 1) ? kItemA : kItemB;
-            idx = (t & 1) ? L + (t >> 1) : (t >> 1);
-        } else {
-            it.kind = kItemB;
-            idx = t - RA;
-        }
-    }
+    if (it.end) return it;
     it.u = (int)(idx / p.pieces);
     const int piece = (int)(idx - (long long)it.u * p.pieces);
     it.g = it.u / p.H;
@@ -193,74 +188,125 @@ __device__ __forceinline__ Item decode_item(long long pos, const KeyPassArgs& p)
     return it;
 }
 
-// ---------------------------------------------------------------------------- producer
-__device__ void producer_role(const CUtensorMap* tmap, unsigned char* ring, Smem* s, const KeyPassArgs& p,
-                              const Waiter& wt) {
-    const uint64_t pol_a = l2_policy_evict_last(), pol_b = l2_policy_evict_first();
-    long long n = 0, ic = 0;
-    bool ok = true;
-    while (ok) {
-        const long long pos = (long long)atomicAdd(p.next_item, 1ULL);
-        const Item it = decode_item(pos, p);
-        const int q = (int)(ic & (kQueue - 1));
-        if (!bwait(&s->qfree[q], (uint32_t)(((ic / kQueue) & 1) ^ 1), wt, 731)) break;
-        s->items[q] = it;
-        mbar_arrive(&s->qfull[q]);
-        ++ic;
-        if (it.kind == kItemEnd) break;
-        const bool first_touch = it.kind == kItemA;
-        const int ntl = first_touch ? it.ntiles + 1 : it.ntiles;
-        const bool hint = first_touch ? (p.hints & 1) != 0 : (p.hints & 2) != 0;
-        const uint64_t pol = first_touch ? pol_a : pol_b;
-        for (int tl = 0; tl < ntl; ++tl, ++n) {
-            const int slot = (int)(n % kSlots);
-            if (!bwait(&s->sfree[slot], (uint32_t)(((n / kSlots) & 1) ^ 1), wt, 732)) {
-                ok = false;
-                break;
-            }
-            const int R = first_touch ? it.row0 + (tl - 1) * kTile : it.row0 + tl * kTile;
-            const bool before = first_touch && tl > 0 && slot == 0;
-            mbar_expect_tx(&s->full[slot], (before ? 3 : 2) * 2 * kSlabHalfBytes);
-            for (int j = before ? -1 : 0; j < 2; ++j) {
-                unsigned char* dst = ring + (size_t)(j < 0 ? 0 : 1 + 2 * slot + j) * kSlabHalfBytes;
-                const int row = R + j * kSlabRows;
-                if (hint) {
-                    tma_load_4d_hint(dst, tmap, 0, row, it.h, it.g, &s->full[slot], pol);
-                    tma_load_4d_hint(dst + kHalfBytes, tmap, 64, row, it.h, it.g, &s->full[slot], pol);
-                } else {
-                    tma_load_4d(dst, tmap, 0, row, it.h, it.g, &s->full[slot]);
-                    tma_load_4d(dst + kHalfBytes, tmap, 64, row, it.h, it.g, &s->full[slot]);
-                }
-            }
-        }
-    }
-    if (*wt.abort) {
-        // copies already armed still land in this CTA's shared memory: stay until they have
-        for (long long m = n > kSlots ? n - kSlots : 0; m < n; ++m) {
-            uint64_t* bar = &s->full[m % kSlots];
-            const uint32_t par = (uint32_t)((m / kSlots) & 1);
-            for (uint32_t spin = 0; spin < (1u << 16) && !mbar_try_wait(bar, par); ++spin) __nanosleep(256);
-        }
+// 1/sqrt(x) to fp32 rounding for x well inside the normal range (one Newton step on the hardware estimate)
+__device__ __forceinline__ float fast_rsqrt(float x) {
+    const float y = rsqrtf(x);
+    return y * fmaf(-0.5f * x * y, y, 1.5f);
+}
+
+// ---------------------------------------------------------------------------- producers
+__device__ __forceinline__ void load_slab(unsigned char* dst, const CUtensorMap* tmap, int row, int h, int g, uint64_t* bar,
+                                          bool hint, uint64_t pol) {
+    if (hint) {
+        tma_load_4d_hint(dst, tmap, 0, row, h, g, bar, pol);
+        tma_load_4d_hint(dst + kHalfBytes, tmap, 64, row, h, g, bar, pol);
+    } else {
+        tma_load_4d(dst, tmap, 0, row, h, g, bar);
+        tma_load_4d(dst + kHalfBytes, tmap, 64, row, h, g, bar);
     }
 }
 
-// ---------------------------------------------------------------------------- MMA issuer
-__device__ void mma_role(unsigned char* ring, unsigned char* wsplit, unsigned char* rhs, Smem* s, uint32_t tmem,
-                         const Waiter& wt) {
+// Copies already armed still land in this CTA's shared memory: after a give-up, stay until they have.
+__device__ __forceinline__ void settle_loads(uint64_t* full, int slots, long long n) {
+    for (long long m = n > slots ? n - slots : 0; m < n; ++m) {
+        uint64_t* bar = &full[m % slots];
+        const uint32_t par = (uint32_t)((m / slots) & 1);
+        for (uint32_t spin = 0; spin < (1u << 16) && !mbar_try_wait(bar, par); ++spin) __nanosleep(256);
+    }
+}
+
+// First-touch producer (one thread): draws pieces, publishes them, stages halo + tiles.
+__device__ void producer_a(const CUtensorMap* tmap, unsigned char* ring, Smem* s, const KeyPassArgs& p, const Waiter& wt) {
+    const uint64_t pol = l2_policy_evict_last();
+    const bool hint = (p.hints & 1) != 0;
+    long long n = 0, ic = 0;
+    bool ok = true;
+    while (ok) {
+        const Item it = decode_item((long long)atomicAdd(p.next_a, 1ULL), p);
+        const int k = (int)(ic & (kQueue - 1));
+        if (!bwait(&s->qa_free[k], (uint32_t)(((ic / kQueue) & 1) ^ 1), wt, 731)) break;
+        s->qa[k] = it;
+        mbar_arrive(&s->qa_full[k]);
+        ++ic;
+        if (it.end) break;
+        // the first rows are asked of DRAM now; further on every tile asks for the one kPrefetchTiles ahead
+        for (int tl = 1; tl <= min(kPrefetchTiles, it.ntiles); ++tl) {
+            tma_prefetch_4d(tmap, 0, it.row0 + (tl - 1) * kTile, it.h, it.g);
+            tma_prefetch_4d(tmap, 0, it.row0 + (tl - 1) * kTile + kSlabRows, it.h, it.g);
+            tma_prefetch_4d(tmap, 64, it.row0 + (tl - 1) * kTile, it.h, it.g);
+            tma_prefetch_4d(tmap, 64, it.row0 + (tl - 1) * kTile + kSlabRows, it.h, it.g);
+        }
+        for (int tl = 0; tl <= it.ntiles; ++tl, ++n) {
+            if (tl + kPrefetchTiles <= it.ntiles && tl > 0) {
+                const int row = it.row0 + (tl + kPrefetchTiles - 1) * kTile;
+                tma_prefetch_4d(tmap, 0, row, it.h, it.g);
+                tma_prefetch_4d(tmap, 0, row + kSlabRows, it.h, it.g);
+                tma_prefetch_4d(tmap, 64, row, it.h, it.g);
+                tma_prefetch_4d(tmap, 64, row + kSlabRows, it.h, it.g);
+            }
+            const int slot = (int)(n % kSlotsA);
+            if (!bwait(&s->free_a[slot], (uint32_t)(((n / kSlotsA) & 1) ^ 1), wt, 732)) {
+                ok = false;
+                break;
+            }
+            const int R = it.row0 + (tl - 1) * kTile;
+            const bool before = tl > 0 && slot == 0;   // slot 0's tile keeps its own copy of the slab before it
+            mbar_expect_tx(&s->full_a[slot], (before ? 3 : 2) * 2 * kSlabHalfBytes);
+            for (int j = before ? -1 : 0; j < 2; ++j)
+                load_slab(ring + (size_t)(j < 0 ? 0 : 1 + 2 * slot + j) * kSlabHalfBytes, tmap, R + j * kSlabRows, it.h,
+                          it.g, &s->full_a[slot], hint, pol);
+        }
+    }
+    if (*wt.abort) settle_loads(s->full_a, kSlotsA, n);
+}
+
+// Second-touch producer (one thread).
+__device__ void producer_b(const CUtensorMap* tmap, unsigned char* ring, Smem* s, const KeyPassArgs& p, const Waiter& wt) {
+    const uint64_t pol = l2_policy_evict_first();
+    const bool hint = (p.hints & 2) != 0;
+    long long n = 0, ic = 0;
+    bool ok = true;
+    while (ok) {
+        const Item it = decode_item((long long)atomicAdd(p.next_b, 1ULL), p);
+        const int k = (int)(ic & (kQueue - 1));
+        if (!bwait(&s->qb_free[k], (uint32_t)(((ic / kQueue) & 1) ^ 1), wt, 733)) break;
+        s->qb[k] = it;
+        mbar_arrive(&s->qb_full[k]);
+        ++ic;
+        if (it.end) break;
+        for (int tl = 0; tl < it.ntiles; ++tl, ++n) {
+            const int slot = (int)(n % kSlotsB);
+            if (!bwait(&s->free_b[slot], (uint32_t)(((n / kSlotsB) & 1) ^ 1), wt, 734)) {
+                ok = false;
+                break;
+            }
+            const int R = it.row0 + tl * kTile;
+            mbar_expect_tx(&s->full_b[slot], 2 * 2 * kSlabHalfBytes);
+            for (int j = 0; j < 2; ++j)
+                load_slab(ring + (size_t)(kSlabsA + 2 * slot + j) * kSlabHalfBytes, tmap, R + j * kSlabRows, it.h, it.g,
+                          &s->full_b[slot], hint, pol);
+        }
+    }
+    if (*wt.abort) settle_loads(s->full_b, kSlotsB, n);
+}
+
+// ---------------------------------------------------------------------------- MMA issuers
+// First touch (one thread).  Tile n of the CTA goes to the accumulator of team n & 1.
+__device__ void mma_a(unsigned char* ring, unsigned char* wsplit, Smem* s, uint32_t tmem, const Waiter& wt) {
     constexpr uint32_t idesc192 = umma_idesc_bf16(kTile, 192), idesc128 = umma_idesc_bf16(kTile, 128);
-    constexpr uint32_t idesc64 = umma_idesc_bf16(kTile, 64), idesc16 = umma_idesc_bf16(kTile, 16);
-    constexpr uint32_t idesc_bs = umma_idesc_bf16(kD, 16) | kUmmaAMajorMN;
-    const uint32_t ring_a = smem_addr(ring), ws_a = smem_addr(wsplit), rhs_a = smem_addr(rhs);
-    long long n = 0, nA = 0, nC = 0, nS = 0, nB = 0, ic = 0;
+    constexpr uint32_t idesc64 = umma_idesc_bf16(kTile, 64);
+    constexpr uint32_t idesc_ts = umma_idesc_bf16(kD, 16) | kUmmaAMajorMN;
+    const uint32_t ring_a = smem_addr(ring), ws_a = smem_addr(wsplit);
+    long long n = 0, nC = 0, nS = 0, ic = 0;
     int pend_slot = -1;
     bool pend_real = false;
-    // The tile whose slot is still read: issue its block-sum product (real tiles) and release the slot.
+    // The tile whose slot is still read: issue its tile-sum product (real tiles) and release the slot.
     auto flush = [&]() -> bool {
         if (pend_slot < 0) return true;
         if (pend_real) {
             const int b = (int)(nS & 1);
             if (!bwait(&s->wsready[b], (uint32_t)((nS >> 1) & 1), wt, 741)) return false;
-            if (!bwait(&s->bsempty[b], (uint32_t)(((nS >> 1) & 1) ^ 1), wt, 742)) return false;
+            if (!bwait(&s->tsempty[b], (uint32_t)(((nS >> 1) & 1) ^ 1), wt, 742)) return false;
             tc_fence_after();
             const uint32_t a0 = ring_a + (uint32_t)(1 + 2 * pend_slot) * kSlabHalfBytes;
 #pragma unroll
@@ -268,88 +314,98 @@ __device__ void mma_role(unsigned char* ring, unsigned char* wsplit, unsigned ch
                 const uint64_t adesc = umma_desc_sw128_mn(a0 + (uint32_t)kk * 2048u, kHalfBytes);
                 const uint64_t bdesc = umma_desc_sw128(ws_a + (uint32_t)b * kOperandBytes + (uint32_t)(kk >> 2) * 2048u +
                                                        (uint32_t)(kk & 3) * 32u);
-                umma_bf16(tmem + kColBsum + 16u * (uint32_t)b, adesc, bdesc, idesc_bs, kk > 0);
+                umma_bf16(tmem + kColTsum + 16u * (uint32_t)b, adesc, bdesc, idesc_ts, kk > 0);
             }
-            umma_commit(&s->bsfull[b]);
+            umma_commit(&s->tsfull[b]);
             ++nS;
         }
-        umma_commit(&s->sfree[pend_slot]);
+        umma_commit(&s->free_a[pend_slot]);
         pend_slot = -1;
         return true;
     };
     for (;;) {
         Item it;
-        if (!get_item<false>(s, ic++, it, wt, 743)) return;
-        if (it.kind == kItemEnd) {
-            if (!flush()) return;
-            break;
-        }
-        if (it.kind == kItemA) {
-            for (int tl = 0; tl <= it.ntiles; ++tl, ++n, ++nA) {
-                const int slot = (int)(n % kSlots), par = (int)(nA & 1);
-                if (!bwait(&s->full[slot], (uint32_t)((n / kSlots) & 1), wt, 744)) return;
-                if (!bwait(&s->tempty[par], (uint32_t)(((nA >> 1) & 1) ^ 1), wt, 745)) return;
-                if (tl > 0 && !bwait(&s->cempty, (uint32_t)((nC & 1) ^ 1), wt, 746)) return;
-                tc_fence_after();
-                const uint32_t dmain = tmem + (par ? kColMain1 : kColMain0);
-                const uint32_t a0 = ring_a + (uint32_t)(1 + 2 * slot) * kSlabHalfBytes;
-                if (tl == 0) {
-                    // halo: Gram of the 128 rows with themselves, columns 64..191 of the accumulator
-#pragma unroll
-                    for (int kk = 0; kk < kD / 16; ++kk) {
-                        const uint32_t koff = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
-                        umma_bf16(dmain + 64u, umma_desc_sw128(a0 + koff), umma_desc_sw128(a0 + koff), idesc128, kk > 0);
-                    }
-                } else {
-                    const uint32_t b0 = ring_a + (uint32_t)(2 * slot) * kSlabHalfBytes;   // the slab before the tile
-#pragma unroll
-                    for (int kk = 0; kk < kD / 16; ++kk) {
-                        const uint32_t koff = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
-                        umma_bf16(dmain, umma_desc_sw128(a0 + koff), umma_desc_sw128(b0 + koff), idesc192, kk > 0);
-                    }
-                    const uint32_t pa = ring_a + (uint32_t)(1 + 2 * (int)((n - 1) % kSlots)) * kSlabHalfBytes;
-#pragma unroll
-                    for (int kk = 0; kk < kD / 16; ++kk) {
-                        const uint32_t koff = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
-                        umma_bf16(tmem + kColCorner, umma_desc_sw128(pa + koff), umma_desc_sw128(a0 + koff), idesc64,
-                                  kk > 0);
-                    }
-                    ++nC;
-                }
-                umma_commit(&s->tfull[par]);
-                if (!flush()) return;
-                pend_slot = slot;
-                pend_real = tl > 0;
-            }
-        } else {
-            // nothing of a first-touch item may wait behind a second-touch tile
-            if (!flush()) return;
-            for (int tl = 0; tl < it.ntiles; ++tl, ++n, ++nB) {
-                const int slot = (int)(n % kSlots), b = (int)(nB & 1);
-                if (!bwait(&s->full[slot], (uint32_t)((n / kSlots) & 1), wt, 747)) return;
-                if (!bwait(&s->rready[b], (uint32_t)((nB >> 1) & 1), wt, 748)) return;
-                if (!bwait(&s->dempty[b], (uint32_t)(((nB >> 1) & 1) ^ 1), wt, 749)) return;
-                tc_fence_after();
-                const uint32_t a0 = ring_a + (uint32_t)(1 + 2 * slot) * kSlabHalfBytes;
+        if (!get_item<false>(s->qa, s->qa_full, s->qa_free, ic++, it, wt, 743)) return;
+        if (it.end) break;
+        for (int tl = 0; tl <= it.ntiles; ++tl, ++n) {
+            const int slot = (int)(n % kSlotsA), par = (int)(n & 1);
+            if (!bwait(&s->full_a[slot], (uint32_t)((n / kSlotsA) & 1), wt, 744)) return;
+            if (!bwait(&s->tempty[par], (uint32_t)(((n >> 1) & 1) ^ 1), wt, 745)) return;
+            if (tl > 0 && !bwait(&s->cempty, (uint32_t)((nC & 1) ^ 1), wt, 746)) return;
+            tc_fence_after();
+            const uint32_t dmain = tmem + (par ? kColMain1 : kColMain0);
+            const uint32_t a0 = ring_a + (uint32_t)(1 + 2 * slot) * kSlabHalfBytes;
+            if (tl == 0) {
+                // halo: Gram of the 128 rows with themselves, columns 64..191 of the accumulator
 #pragma unroll
                 for (int kk = 0; kk < kD / 16; ++kk) {
                     const uint32_t koff = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
-                    const uint64_t bdesc = umma_desc_sw128(rhs_a + (uint32_t)b * kOperandBytes +
-                                                           (uint32_t)(kk >> 2) * 2048u + (uint32_t)(kk & 3) * 32u);
-                    umma_bf16(tmem + kColDots + 16u * (uint32_t)b, umma_desc_sw128(a0 + koff), bdesc, idesc16, kk > 0);
+                    umma_bf16(dmain + 64u, umma_desc_sw128(a0 + koff), umma_desc_sw128(a0 + koff), idesc128, kk > 0);
                 }
-                umma_commit(&s->dfull[b]);
-                umma_commit(&s->rfree[b]);
-                umma_commit(&s->sfree[slot]);
+            } else {
+                const uint32_t b0 = ring_a + (uint32_t)(2 * slot) * kSlabHalfBytes;   // the slab before the tile
+#pragma unroll
+                for (int kk = 0; kk < kD / 16; ++kk) {
+                    const uint32_t koff = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
+                    umma_bf16(dmain, umma_desc_sw128(a0 + koff), umma_desc_sw128(b0 + koff), idesc192, kk > 0);
+                }
+                const uint32_t pa = ring_a + (uint32_t)(1 + 2 * (int)((n - 1) % kSlotsA)) * kSlabHalfBytes;
+#pragma unroll
+                for (int kk = 0; kk < kD / 16; ++kk) {
+                    const uint32_t koff = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
+                    umma_bf16(tmem + kColCorner, umma_desc_sw128(pa + koff), umma_desc_sw128(a0 + koff), idesc64, kk > 0);
+                }
+                ++nC;
+            }
+            umma_commit(&s->tfull[par]);
+            if (!flush()) return;
+            pend_slot = slot;
+            pend_real = tl > 0;
+        }
+    }
+    if (!flush()) return;
+    // every product issued has completed before the accumulators are given back
+    umma_commit(&s->drain_a);
+    bwait(&s->drain_a, 0, wt, 747);
+}
+
+// Second touch (one thread): the tiles of a block share one pair of split anchors.
+__device__ void mma_b(unsigned char* ring, unsigned char* rhs, Smem* s, uint32_t tmem, int tiles_per_block,
+                      const Waiter& wt) {
+    constexpr uint32_t idesc16 = umma_idesc_bf16(kTile, 16);
+    const uint32_t ring_a = smem_addr(ring), rhs_a = smem_addr(rhs);
+    long long n = 0, nR = 0, ic = 0;
+    for (;;) {
+        Item it;
+        if (!get_item<false>(s->qb, s->qb_full, s->qb_free, ic++, it, wt, 748)) return;
+        if (it.end) break;
+        for (int tl = 0; tl < it.ntiles; ++tl, ++n) {
+            const int slot = (int)(n % kSlotsB), b = (int)(n & 1), rb = (int)(nR & 1);
+            if (tl % tiles_per_block == 0 && !bwait(&s->rready[rb], (uint32_t)((nR >> 1) & 1), wt, 749)) return;
+            if (!bwait(&s->full_b[slot], (uint32_t)((n / kSlotsB) & 1), wt, 750)) return;
+            if (!bwait(&s->dempty[b], (uint32_t)(((n >> 1) & 1) ^ 1), wt, 751)) return;
+            tc_fence_after();
+            const uint32_t a0 = ring_a + (uint32_t)(kSlabsA + 2 * slot) * kSlabHalfBytes;
+#pragma unroll
+            for (int kk = 0; kk < kD / 16; ++kk) {
+                const uint32_t koff = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
+                const uint64_t bdesc = umma_desc_sw128(rhs_a + (uint32_t)rb * kOperandBytes + (uint32_t)(kk >> 2) * 2048u +
+                                                       (uint32_t)(kk & 3) * 32u);
+                umma_bf16(tmem + kColDots + 16u * (uint32_t)b, umma_desc_sw128(a0 + koff), bdesc, idesc16, kk > 0);
+            }
+            umma_commit(&s->dfull[b]);
+            umma_commit(&s->free_b[slot]);
+            if ((tl + 1) % tiles_per_block == 0 || tl + 1 == it.ntiles) {
+                umma_commit(&s->rfree[rb]);
+                ++nR;
             }
         }
     }
-    // every product issued has completed before the accumulators are given back
-    umma_commit(&s->drain);
-    bwait(&s->drain, 0, wt, 750);
+    umma_commit(&s->drain_b);
+    bwait(&s->drain_b, 0, wt, 752);
 }
 
-// ---------------------------------------------------------------------------- band group
+// ---------------------------------------------------------------------------- first-touch teams
 // Band sums of one row of D over three 32-column chunks: column o of chunk A counts when o >= thr, chunk B
 // counts whole, column o of chunk C counts when o < thr.  Every column is weighted by its key's 1/||k||;
 // iA, iB, iC are the ring indices (multiples of 32) of the chunks' first keys.
@@ -420,81 +476,71 @@ __device__ __forceinline__ float select_lane(const float* v, int lane) {
     return (lane & 1) ? d[1] : d[0];
 }
 
-// The CTA that completed a head's last piece: head sum, 1/||head sum||, 1/||block sum|| (256 threads).
-__device__ void finalise_head(Smem* s, const KeyPassArgs& p, int u, int tid) {
-    const int nb = p.sp.nblocks;
-    const float* bs = p.block_sums + (size_t)u * nb * kD;
+// The team that completed a head's last piece: block sums, head sum and the reciprocals of their norms
+// (256 threads, `tid` inside the team, `bar` the team's named barrier).
+__device__ void finalise_head(TeamSmem* ts, const KeyPassArgs& p, int u, int tid, int bar) {
+    const int nb = p.sp.nblocks, T = (p.N + kTile - 1) / kTile, tpb = p.sp.block / kTile;
+    const float* tsum = p.tile_sums + (size_t)u * T * kD;
+    float* bs = p.block_sums + (size_t)u * nb * kD;
     const int c = tid & (kD - 1), half = tid >> 7, warp = tid >> 5, lane = tid & 31;
     float sum = 0.f, comp = 0.f;   // compensated: the head sum is the anchor of every key of the head
     for (int b = half; b < nb; b += 2) {
-        const float y = __ldcg(bs + (size_t)b * kD + c) - comp;
-        const float t = sum + y;
-        comp = (t - sum) - y;
-        sum = t;
+        float v = 0.f;
+        for (int t = b * tpb; t < min((b + 1) * tpb, T); ++t) v += __ldcg(tsum + (size_t)t * kD + c);
+        bs[(size_t)b * kD + c] = v;
+        const float y = v - comp;
+        const float t2 = sum + y;
+        comp = (t2 - sum) - y;
+        sum = t2;
     }
-    s->fin[half][c] = sum;
-    bar_sync(kBarBand, kBandThreads);
+    ts->fin[half][c] = sum;
+    bar_sync(bar, kTeamThreads);   // also orders this team's block-sum writes before its reads below
     if (tid < kD) {
-        const float tot = s->fin[0][c] + s->fin[1][c];
+        const float tot = ts->fin[0][c] + ts->fin[1][c];
         p.head_sum[(size_t)u * kD + c] = tot;
-        s->fin[0][c] = tot;
+        ts->fin[0][c] = tot;
     }
-    bar_sync(kBarBand, kBandThreads);
+    bar_sync(bar, kTeamThreads);
     if (warp == 0) {
-        const float4 v = *reinterpret_cast<const float4*>(&s->fin[0][4 * lane]);
+        const float4 v = *reinterpret_cast<const float4*>(&ts->fin[0][4 * lane]);
         const float ss = warp_sum(v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w);
         if (lane == 0) p.inv_s[u] = 1.0f / fmaxf(sqrtf(ss), kEps);
     }
-    for (int b = warp; b < nb; b += kBandThreads / 32) {
+    for (int b = warp; b < nb; b += kTeamThreads / 32) {
         const float4 v = __ldcg(reinterpret_cast<const float4*>(bs + (size_t)b * kD) + lane);
         const float ss = warp_sum(v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w);
         if (lane == 0) p.inv_e[(size_t)u * nb + b] = 1.0f / fmaxf(sqrtf(ss), kEps);
     }
 }
 
-__device__ void band_role(unsigned char* wsplit, Smem* s, uint32_t tmem, const KeyPassArgs& p, const Waiter& wt) {
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+// One team (8 warps) takes every second first-touch tile of the CTA.
+__device__ void team_role(int team, unsigned char* wsplit, Smem* s, uint32_t tmem, const KeyPassArgs& p,
+                          const Waiter& wt) {
+    const int tid = threadIdx.x - team * kTeamThreads, warp = tid >> 5, lane = tid & 31;
     const int q = warp & 3, side = warp >> 2;   // quarter of the tile's rows; 0 backward band, 1 forward band
     const int r = q * 32 + lane;                // row of the tile
-    const int N = p.N, nb = p.sp.nblocks, blk_len = p.sp.block;
+    const int N = p.N, T = (N + kTile - 1) / kTile;
+    const int bar_team = 1 + team, bar_fwd = 3 + team;
     const uint32_t lane_base = (uint32_t)(32 * q) << 16;
-    long long ic = 0, nA = 0, nW = 0, nS = 0;   // items, first-touch tiles, split norms written, block sums read
-    float carry = 0.f;   // forward sums of this thread's row of the previous tile over that tile's own columns
+    const uint32_t dmain = tmem + lane_base + (team ? kColMain1 : kColMain0);
+    TeamSmem* ts = &s->team[team];
+    long long ic = 0, n0 = 0, real0 = 0;   // pieces read, first-touch tiles and real tiles before the piece
     for (;;) {
         Item it;
-        const bool got = get_item<true>(s, ic++, it, wt, 751);
-        if (bar_or(kBarBand, kBandThreads, !got)) return;   // the group leaves together or not at all
-        if (it.kind == kItemEnd) return;
-        if (it.kind == kItemB) continue;
+        const bool got = get_item<true>(s->qa, s->qa_full, s->qa_free, ic++, it, wt, 753);
+        if (bar_or(bar_team, kTeamThreads, !got)) return;   // the team leaves together or not at all
+        if (it.end) return;
         const int u = it.u;
-        float lo = INFINITY, hi = -INFINITY, run = 0.f;
+        const long long n_last = n0 + it.ntiles;
+        float lo = INFINITY, hi = -INFINITY;
         bool ok = true;
-        // block sums of the previous real tile (backward side): thread r owns channel r
-        auto take_block_sum = [&](int tlp) {
-            const int b = (int)(nS & 1);
-            ok = bwait(&s->bsfull[b], (uint32_t)((nS >> 1) & 1), wt, 752) && ok;
-            tc_fence_after();
-            float d[16];
-            tmem_ld16(tmem + lane_base + kColBsum + 16u * (uint32_t)b, d);
-            tmem_wait_ld(d);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&s->bsempty[b]);
-            ++nS;
-            run += d[0] + d[1] + d[2];
-            const int Rp = it.row0 + (tlp - 1) * kTile, end = Rp + kTile;
-            if (end % blk_len == 0 || end >= N || tlp == it.ntiles) {
-                p.block_sums[((size_t)u * nb + Rp / blk_len) * kD + r] = run;
-                run = 0.f;
-            }
-        };
-        for (int tl = 0; tl <= it.ntiles; ++tl, ++nA) {
-            const int par = (int)(nA & 1);
+        for (int tl = (int)((n0 ^ team) & 1); tl <= it.ntiles; tl += 2) {
+            const long long n = n0 + tl, nW = real0 + tl - 1;   // tile of the CTA; real tile of the CTA
             const bool real = tl > 0;
             const int R = it.row0 + (tl - 1) * kTile, i = R + r;
-            const int wbase = (int)(nA & 3) * kTile;   // ring index of the tile's row 0
-            const uint32_t dmain = tmem + lane_base + (par ? kColMain1 : kColMain0);
-            ok = bwait(&s->tfull[par], (uint32_t)((nA >> 1) & 1), wt, 753) && ok;
+            const int wbase = (int)(n & (kHist - 1)) * kTile;   // ring index of the tile's row 0
+            const int slot4 = (int)(n & (kHist - 1)), prev4 = (int)((n - 1) & (kHist - 1));
+            ok = bwait(&s->tfull[team], (uint32_t)((n >> 1) & 1), wt, 754) && ok;
             tc_fence_after();
             float wi = 0.f, gi = 0.f;
             if (side == 0) {
@@ -503,13 +549,13 @@ __device__ void band_role(unsigned char* wsplit, Smem* s, uint32_t tmem, const K
                 tmem_ld32(dmain + (uint32_t)(32 * q + 64), v);
                 tmem_wait_ld(v, v + 16);
                 const float n2 = select_lane(v, lane);
-                wi = (i >= 0 && i < N) ? 1.0f / fmaxf(sqrtf(n2), kEps) : 0.f;
+                if (i >= 0 && i < N) wi = n2 > 1e-30f ? fast_rsqrt(n2) : 1.0f / fmaxf(sqrtf(n2), kEps);
                 gi = wi * wi * n2;
                 s->w[wbase + r] = wi;
                 s->g[wbase + r] = gi;
                 if (real) {
                     if (i < N) p.inv_norm[(size_t)u * N + i] = wi;
-                    // w as hi + mid + lo in bf16: rows 0..2 of the block-sum product's second operand
+                    // w as hi + mid + lo in bf16: rows 0..2 of the tile-sum product's second operand
                     unsigned char* base = wsplit + (size_t)(nW & 1) * kOperandBytes + (size_t)(r >> 6) * 2048 + (r & 7) * 2;
                     const __nv_bfloat16 hi_ = __float2bfloat16_rn(wi);
                     const float r1 = wi - __bfloat162float(hi_);
@@ -522,19 +568,24 @@ __device__ void band_role(unsigned char* wsplit, Smem* s, uint32_t tmem, const K
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads these writes
                 }
             }
-            if (bar_or(kBarBand, kBandThreads, !ok)) return;   // norms of the tile are in the ring
+            if (bar_or(bar_team, kTeamThreads, !ok)) return;   // the tile's norms are in the ring
+            if (side == 0 && lane == 0) {
+                mbar_arrive(&s->wpub[slot4]);
+                if (real) mbar_arrive(&s->wsready[nW & 1]);
+            }
+            // the previous tile belongs to the other team: its norms, then (below) its carry and restart parts
+            if (real) ok = bwait(&s->wpub[prev4], (uint32_t)(((n - 1) / kHist) & 1), wt, 755) && ok;
             float X, Y, Z;
             if (side == 0) {
-                if (real && lane == 0) mbar_arrive(&s->wsready[nW & 1]);
                 const int c0 = 32 * q;
                 band_sums3(dmain + c0, dmain + c0 + 32, dmain + c0 + 64, s->w, wbase - 64 + c0, wbase - 32 + c0,
                            wbase + c0, lane + 1, X, Y, Z);
-                s->c[par][r] = wi * (X + Y + Z);
+                ts->c[r] = wi * (X + Y + Z);
                 if (q >= 2) {
                     // Gram block of the tile's last 64 rows: the next tile's exact restart value
                     const float bp = wi * (q == 2 ? Z : Y + Z);
                     const float ap = warp_sum(2.f * bp - gi);
-                    if (lane == 0) s->apart[par ^ 1][q - 2] = ap;
+                    if (lane == 0) s->apart[slot4][q - 2] = ap;
                 }
             } else {
                 // forward band: three chunks from column 32 q + 64; columns past 191 are the corner that
@@ -556,31 +607,49 @@ __device__ void band_role(unsigned char* wsplit, Smem* s, uint32_t tmem, const K
                     }
                 }
                 band_sums3(ta[0], ta[1], ta[2], s->w, ia[0], ia[1], ia[2], lane, X, Y, Z);
-                const float wr = s->w[wbase + r];
-                if (q < 2) {
-                    s->fcur[par][r] = wr * (X + Y + Z);
-                } else {
-                    const float wprev = s->w[(wbase - kTile + r) & kWMask];
-                    const float late = q == 2 ? Z : Y + Z, now = q == 2 ? X + Y : X;
-                    s->fprev[par][r - 64] = wprev * (carry + late);
-                    carry = now;
-                }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(&s->tempty[par]);
+                mbar_arrive(&s->tempty[team]);
                 if (side == 1 && q >= 2 && real) mbar_arrive(&s->cempty);
             }
-            if (bar_or(kBarBand, kBandThreads, !ok)) return;   // band sums of the tile are written
-            if (real) ++nW;
+            if (real) ok = bwait(&s->spub[prev4], (uint32_t)(((n - 1) / kHist) & 1), wt, 756) && ok;
+            if (side == 1) {
+                const float wr = s->w[wbase + r];
+                if (q < 2) {
+                    ts->fcur[r] = wr * (X + Y + Z);
+                } else {
+                    const float wprev = s->w[(wbase - kTile + r) & kWMask];
+                    const float late = q == 2 ? Z : Y + Z, now = q == 2 ? X + Y : X;
+                    ts->fprev[r - 64] = wprev * (s->carry[prev4][r - 64] + late);
+                    s->carry[slot4][r - 64] = now;
+                }
+            }
+            if (q >= 2) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&s->spub[slot4]);
+            }
+            if (bar_or(bar_team, kTeamThreads, !ok)) return;   // band sums of the tile are written
             if (side == 0) {
-                if (tl >= 2) take_block_sum(tl - 1);
+                if (real) {
+                    // sum of the tile's normalised keys: thread r owns channel r
+                    const int b = (int)(nW & 1);
+                    ok = bwait(&s->tsfull[b], (uint32_t)((nW >> 1) & 1), wt, 757) && ok;
+                    tc_fence_after();
+                    float d[16];
+                    tmem_ld16(tmem + lane_base + kColTsum + 16u * (uint32_t)b, d);
+                    tmem_wait_ld(d);
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&s->tsempty[b]);
+                    p.tile_sums[((size_t)u * T + R / kTile) * kD + r] = d[0] + d[1] + d[2];
+                }
             } else {
                 // T_i = restart + prefix of (2 c_i - g_ii) - (2 f_{i-64} - g_{i-64,i-64})
-                const float ci = s->c[par][r];
+                const float ci = ts->c[r];
                 const float g0 = s->g[wbase + r];
-                const float fm = r < 64 ? s->fprev[par][r] : s->fcur[par][r - 64];
+                const float fm = r < 64 ? ts->fprev[r] : ts->fcur[r - 64];
                 const float gm = s->g[(wbase + r - 64) & kWMask];
                 float x = 2.f * ci - g0 - (2.f * fm - gm);
 #pragma unroll
@@ -588,57 +657,64 @@ __device__ void band_role(unsigned char* wsplit, Smem* s, uint32_t tmem, const K
                     const float y = __shfl_up_sync(0xffffffffu, x, o);
                     if (lane >= o) x += y;
                 }
-                if (lane == 31) s->wtot[par][q] = x;
-                bar_sync(kBarFwd, 128);
-                float base = s->apart[par][0] + s->apart[par][1];
-                for (int w = 0; w < q; ++w) base += s->wtot[par][w];
+                if (lane == 31) ts->wtot[q] = x;
+                bar_sync(bar_fwd, 128);
+                float base = s->apart[prev4][0] + s->apart[prev4][1];
+                for (int w = 0; w < q; ++w) base += ts->wtot[w];
                 const float Ti = base + x;
                 if (real && i < N) {
-                    const float a_c = -ci / fmaxf(sqrtf(fmaxf(Ti, 0.f)), kEps) + 0.f;
+                    const float a_c = (Ti > 1e-30f ? -ci * fast_rsqrt(Ti) : -ci / fmaxf(sqrtf(fmaxf(Ti, 0.f)), kEps)) + 0.f;
                     p.a_raw[((size_t)u * 3 + 2) * N + i] = a_c;
                     lo = fminf(lo, a_c);
                     hi = fmaxf(hi, a_c);
                 }
             }
+            __threadfence();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s->done[slot4]);
         }
-        // ---- end of the piece
-        if (side == 0) {
-            take_block_sum(it.ntiles);
-        } else {
+        // ---- end of the piece: min/max of the team's tiles
+        if (side == 1) {
             lo = warp_min(lo);
             hi = warp_max(hi);
             if (lane == 0) {
-                s->red[2 * q] = lo;
-                s->red[2 * q + 1] = hi;
+                ts->red[2 * q] = lo;
+                ts->red[2 * q + 1] = hi;
             }
         }
-        __threadfence();
-        if (bar_or(kBarBand, kBandThreads, !ok)) return;
+        const bool owner = (int)(n_last & 1) == team;   // this team took the piece's last tile
+        if (owner) ok = bwait(&s->done[(n_last - 1) & (kHist - 1)], (uint32_t)(((n_last - 1) / kHist) & 1), wt, 758) && ok;
+        if (bar_or(bar_team, kTeamThreads, !ok)) return;
         if (tid == 128) {
             for (int w = 0; w < 4; ++w) {
-                lo = fminf(lo, s->red[2 * w]);
-                hi = fmaxf(hi, s->red[2 * w + 1]);
+                lo = fminf(lo, ts->red[2 * w]);
+                hi = fmaxf(hi, ts->red[2 * w + 1]);
             }
             if (lo <= hi) {
                 atomicMin(&p.mm[(size_t)u * 6 + 4], ord_key(lo));
                 atomicMax(&p.mm[(size_t)u * 6 + 5], ord_key(hi));
             }
         }
-        if (tid == 0) {
-            __threadfence();
-            s->fin_flag = atomicAdd(&p.head_count[u], 1) == p.pieces - 1;
-        }
-        bar_sync(kBarBand, kBandThreads);
-        if (s->fin_flag) {   // every piece of the head is done, by this CTA or by others
-            __threadfence();
-            finalise_head(s, p, u, tid);
-            __threadfence();
-            bar_sync(kBarBand, kBandThreads);
-            if (tid == 0 && !(p.debug & 1)) {
+        if (owner) {
+            // both teams have fenced every write of the piece
+            if (tid == 0) {
                 __threadfence();
-                atomicExch(&p.head_ready[u], 1);
+                ts->fin_flag = atomicAdd(&p.head_count[u], 1) == p.pieces - 1;
+            }
+            bar_sync(bar_team, kTeamThreads);
+            if (ts->fin_flag) {   // every piece of the head is done, by this CTA or by others
+                __threadfence();
+                finalise_head(ts, p, u, tid, bar_team);
+                __threadfence();
+                bar_sync(bar_team, kTeamThreads);
+                if (tid == 0 && !(p.debug & 1)) {
+                    __threadfence();
+                    atomicExch(&p.head_ready[u], 1);
+                }
             }
         }
+        n0 += it.ntiles + 1;
+        real0 += it.ntiles;
     }
 }
 
@@ -649,44 +725,43 @@ __device__ __forceinline__ int ld_acquire(const int* ptr) {
     return v;
 }
 
-// Thread k writes column k of the six anchor rows of every tile (rows 6..15 stay zero): the head sum and the
-// sum of the tile's block, each as hi + mid + lo in bf16.
-__device__ void prep_role(unsigned char* rhs, Smem* s, const KeyPassArgs& p, const Waiter& wt) {
-    const int k = threadIdx.x - kPrepWarp0 * 32, lane = k & 31;
-    const int half = k >> 6, kk = k & 63;
-    long long ic = 0, nB = 0;
-    bool degraded = false;
+// Four warps.  Thread k writes column k of the six anchor rows (rows 6..15 stay zero): the head sum and the
+// sum of the block, each as hi + mid + lo in bf16; thread r reads row r of a tile's accumulator: the key's
+// dots with the head sum and with its block's sum.
+__device__ void second_touch_role(unsigned char* rhs, Smem* s, uint32_t tmem, const KeyPassArgs& p, const Waiter& wt) {
+    const int r = threadIdx.x - kBWarp0 * 32, q = r >> 5, lane = r & 31;
+    const int half = r >> 6, kk = r & 63;
+    const int N = p.N, nb = p.sp.nblocks, tpb = p.sp.block / kTile;
+    long long ic = 0, n = 0, nR = 0;
+    bool degraded = false, ok = true;
     for (;;) {
         Item it;
-        if (!get_item<true>(s, ic++, it, wt, 761)) return;
-        if (it.kind == kItemEnd) return;
-        if (it.kind == kItemA) continue;
+        if (!get_item<true>(s->qb, s->qb_full, s->qb_free, ic++, it, wt, 761)) return;
+        if (it.end) return;
+        const int u = it.u;
         if (!degraded) {
-            uint32_t ns = 64;
             uint32_t spin = 0;
-            while (ld_acquire(&p.head_ready[it.u]) == 0) {
+            while (ld_acquire(&p.head_ready[u]) == 0) {
                 if (*wt.abort) return;
                 if (++spin > p.flag_spin_limit) {
                     set_status(p.status, NKV_ERR_TIMEOUT, 762);
                     degraded = true;   // go on with what the buffers hold, wait for no further flag
                     break;
                 }
-                __nanosleep(ns);
-                if (ns < 1024) ns <<= 1;
+                __nanosleep(spin < 16 ? 64 : 512);
             }
         }
-        float v[2] = {0.f, 0.f};
-        v[0] = __ldcg(&p.head_sum[(size_t)it.u * kD + k]);
-        int cur_blk = -1;
-        for (int tl = 0; tl < it.ntiles; ++tl, ++nB) {
-            const int b = (int)(nB & 1);
-            if (!bwait(&s->rfree[b], (uint32_t)(((nB >> 1) & 1) ^ 1), wt, 763)) return;
-            const int blk = (it.row0 + tl * kTile) / p.sp.block;
-            if (blk != cur_blk) {
-                v[1] = __ldcg(&p.block_sums[((size_t)it.u * p.sp.nblocks + blk) * kD + k]);
-                cur_blk = blk;
-            }
-            unsigned char* base = rhs + (size_t)b * kOperandBytes + (size_t)half * 2048 + (kk & 7) * 2;
+        // the head's anchors, norms and 1/||k|| are final from here on
+        const float rs = __ldcg(&p.inv_s[u]);
+        const float v0 = __ldcg(&p.head_sum[(size_t)u * kD + r]);
+        const int blk0 = it.row0 / p.sp.block, nblk = (it.ntiles + tpb - 1) / tpb;
+        float v1 = __ldcg(&p.block_sums[((size_t)u * nb + blk0) * kD + r]);
+        auto build = [&](int b) {   // split anchors of block blk0 + b; fetches the next block's sum
+            const int rb = (int)((nR + b) & 1);
+            ok = bwait(&s->rfree[rb], (uint32_t)((((nR + b) >> 1) & 1) ^ 1), wt, 763) && ok;
+            const float v[2] = {v0, v1};
+            if (b + 1 < nblk) v1 = __ldcg(&p.block_sums[((size_t)u * nb + blk0 + b + 1) * kD + r]);
+            unsigned char* base = rhs + (size_t)rb * kOperandBytes + (size_t)half * 2048 + (kk & 7) * 2;
 #pragma unroll
             for (int a = 0; a < 2; ++a) {
                 const __nv_bfloat16 hi = __float2bfloat16_rn(v[a]);
@@ -702,50 +777,45 @@ __device__ void prep_role(unsigned char* rhs, Smem* s, const KeyPassArgs& p, con
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
-            if (lane == 0) mbar_arrive(&s->rready[b]);
-        }
-    }
-}
-
-// Thread r reads row r of the accumulator: the key's dots with the head sum and with its block's sum.
-__device__ void epilogue_role(Smem* s, uint32_t tmem, const KeyPassArgs& p, const Waiter& wt) {
-    const int r = threadIdx.x - kEpiWarp0 * 32, q = r >> 5, lane = r & 31;
-    const int N = p.N, nb = p.sp.nblocks;
-    long long ic = 0, nB = 0;
-    for (;;) {
-        Item it;
-        if (!get_item<true>(s, ic++, it, wt, 771)) return;
-        if (it.kind == kItemEnd) return;
-        if (it.kind == kItemA) continue;
-        const int u = it.u;
+            if (lane == 0) mbar_arrive(&s->rready[rb]);
+        };
         float lo_s = INFINITY, hi_s = -INFINITY, lo_e = INFINITY, hi_e = -INFINITY;
-        float rs = 0.f;
-        for (int tl = 0; tl < it.ntiles; ++tl, ++nB) {
-            const int b = (int)(nB & 1);
-            if (!bwait(&s->dfull[b], (uint32_t)((nB >> 1) & 1), wt, 772)) return;
+        build(0);
+        int i = it.row0 + r;
+        float wi = i < N ? __ldcg(&p.inv_norm[(size_t)u * N + i]) : 0.f;
+        float re = __ldcg(&p.inv_e[(size_t)u * nb + blk0]);
+        for (int tl = 0; tl < it.ntiles; ++tl, ++n) {
+            if (tl % tpb == 0 && tl / tpb + 1 < nblk) build(tl / tpb + 1);   // one block ahead of the products
+            // this tile's inputs are in registers; fetch the next tile's while the product runs
+            const int i_cur = i;
+            const float wi_cur = wi, re_cur = re;
+            if (tl + 1 < it.ntiles) {
+                i = it.row0 + (tl + 1) * kTile + r;
+                wi = i < N ? __ldcg(&p.inv_norm[(size_t)u * N + i]) : 0.f;
+                re = __ldcg(&p.inv_e[(size_t)u * nb + (it.row0 + (tl + 1) * kTile) / p.sp.block]);
+            }
+            const int b = (int)(n & 1);
+            if (!bwait(&s->dfull[b], (uint32_t)((n >> 1) & 1), wt, 764)) return;
             tc_fence_after();
-            // the accumulator exists, so the head's flag has been seen: its anchors and norms are final
-            const int i = it.row0 + tl * kTile + r;
-            const float wi = i < N ? __ldcg(&p.inv_norm[(size_t)u * N + i]) : 0.f;
-            const float re = __ldcg(&p.inv_e[(size_t)u * nb + (it.row0 + tl * kTile) / p.sp.block]);
-            if (tl == 0) rs = __ldcg(&p.inv_s[u]);
             float d[16];
             tmem_ld16(tmem + ((uint32_t)(32 * q) << 16) + kColDots + 16u * (uint32_t)b, d);
             tmem_wait_ld(d);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&s->dempty[b]);
-            const float a_s = -((d[0] + d[1] + d[2]) * wi) * rs + 0.f;
-            const float a_e = -((d[3] + d[4] + d[5]) * wi) * re + 0.f;
-            if (i < N) {
-                p.a_raw[((size_t)u * 3 + 0) * N + i] = a_s;
-                p.a_raw[((size_t)u * 3 + 1) * N + i] = a_e;
+            const float a_s = -((d[0] + d[1] + d[2]) * wi_cur) * rs + 0.f;
+            const float a_e = -((d[3] + d[4] + d[5]) * wi_cur) * re_cur + 0.f;
+            if (i_cur < N) {
+                p.a_raw[((size_t)u * 3 + 0) * N + i_cur] = a_s;
+                p.a_raw[((size_t)u * 3 + 1) * N + i_cur] = a_e;
                 lo_s = fminf(lo_s, a_s);
                 hi_s = fmaxf(hi_s, a_s);
                 lo_e = fminf(lo_e, a_e);
                 hi_e = fmaxf(hi_e, a_e);
             }
         }
+        if (!ok) return;
+        nR += nblk;
         lo_s = warp_min(lo_s);
         hi_s = warp_max(hi_s);
         lo_e = warp_min(lo_e);
@@ -771,28 +841,39 @@ key_pass_kernel(const __grid_constant__ CUtensorMap tmap, const KeyPassArgs p) {
 
     if (tid == 0) {
         for (int i = 0; i < kQueue; ++i) {
-            mbar_init(&s->qfull[i], 1);
-            mbar_init(&s->qfree[i], kConsumerWarps);
+            mbar_init(&s->qa_full[i], 1);
+            mbar_init(&s->qa_free[i], kConsumersA);
+            mbar_init(&s->qb_full[i], 1);
+            mbar_init(&s->qb_free[i], kConsumersB);
         }
-        for (int i = 0; i < kSlots; ++i) {
-            mbar_init(&s->full[i], 1);
-            mbar_init(&s->sfree[i], 1);
+        for (int i = 0; i < kSlotsA; ++i) {
+            mbar_init(&s->full_a[i], 1);
+            mbar_init(&s->free_a[i], 1);
+        }
+        for (int i = 0; i < kSlotsB; ++i) {
+            mbar_init(&s->full_b[i], 1);
+            mbar_init(&s->free_b[i], 1);
+        }
+        for (int i = 0; i < kHist; ++i) {
+            mbar_init(&s->wpub[i], 4);
+            mbar_init(&s->spub[i], 4);
+            mbar_init(&s->done[i], 8);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&s->tfull[i], 1);
             mbar_init(&s->tempty[i], 8);
             mbar_init(&s->wsready[i], 4);
-            mbar_init(&s->bsfull[i], 1);
-            mbar_init(&s->bsempty[i], 4);
+            mbar_init(&s->tsfull[i], 1);
+            mbar_init(&s->tsempty[i], 4);
             mbar_init(&s->rready[i], 4);
             mbar_init(&s->rfree[i], 1);
             mbar_init(&s->dfull[i], 1);
             mbar_init(&s->dempty[i], 4);
         }
         mbar_init(&s->cempty, 2);
-        mbar_init(&s->drain, 1);
+        mbar_init(&s->drain_a, 1);
+        mbar_init(&s->drain_b, 1);
         s->abort = 0;
-        s->fin_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // rows of the two 16-row operands that are never written must read as zeros
@@ -801,8 +882,10 @@ key_pass_kernel(const __grid_constant__ CUtensorMap tmap, const KeyPassArgs p) {
         s->w[i] = 0.f;
         s->g[i] = 0.f;
     }
+    for (int i = tid; i < kHist * 64; i += kThreads) (&s->carry[0][0])[i] = 0.f;
+    if (tid < kHist * 2) (&s->apart[0][0])[tid] = 0.f;
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    if (warp == kMmaWarp) tmem_alloc(&s->tmem_base, kTmemCols);
+    if (warp == kMmaAWarp) tmem_alloc(&s->tmem_base, kTmemCols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -811,23 +894,23 @@ key_pass_kernel(const __grid_constant__ CUtensorMap tmap, const KeyPassArgs p) {
     wt.status = p.status;
     wt.abort = &s->abort;
 
-    if (warp == kProducerWarp) {
-        if (lane == 0) producer_role(&tmap, ring, s, p, wt);
-        __syncwarp();
-    } else if (warp == kMmaWarp) {
-        if (lane == 0) mma_role(ring, wsplit, rhs, s, tmem, wt);
-        __syncwarp();
-    } else if (warp >= kPrepWarp0) {
-        prep_role(rhs, s, p, wt);
-    } else if (warp >= kEpiWarp0) {
-        epilogue_role(s, tmem, p, wt);
+    if (warp < 16) {
+        team_role(warp >> 3, wsplit, s, tmem, p, wt);
+    } else if (warp < kProdAWarp) {
+        second_touch_role(rhs, s, tmem, p, wt);
     } else {
-        band_role(wsplit, s, tmem, p, wt);
+        if (lane == 0) {
+            if (warp == kProdAWarp) producer_a(&tmap, ring, s, p, wt);
+            else if (warp == kProdBWarp) producer_b(&tmap, ring, s, p, wt);
+            else if (warp == kMmaAWarp) mma_a(ring, wsplit, s, tmem, wt);
+            else mma_b(ring, rhs, s, tmem, p.sp.block / kTile, wt);
+        }
+        __syncwarp();
     }
 
     tc_fence_before();
     __syncthreads();
-    if (warp == kMmaWarp) tmem_dealloc(tmem, kTmemCols);
+    if (warp == kMmaAWarp) tmem_dealloc(tmem, kTmemCols);
 }
 
 // reset of the per-head min/max keys and of the scheduling words
@@ -860,6 +943,9 @@ cudaError_t configure_keypass_kernels() {
 }
 
 size_t keypass_ctrl_bytes(int64_t units) { return (size_t)(2 * units + 4) * sizeof(int); }
+size_t keypass_tile_sum_bytes(int64_t units, int64_t N) {
+    return (size_t)units * (size_t)((N + kTile - 1) / kTile) * kD * sizeof(float);
+}
 
 // bf16 keys of 128 columns, the paper's window of 64, blocks of whole tiles, and strides a tensor map
 // accepts (multiples of 16 bytes, base 16-byte aligned).
@@ -873,9 +959,9 @@ bool keypass_supported(const TensorView& K, int dtype, const ScoreParams& sp) {
 }
 
 cudaError_t launch_keypass(const TensorView& K, int G, const ScoreParams& sp, const KeyPassOptions& opt,
-                           float* block_sums, float* head_sum, float* inv_s, float* inv_e, float* inv_norm,
-                           float* a_raw, uint32_t* mm, int* ctrl, int* status, int sm_count, cudaStream_t stream,
-                           int64_t* launches) {
+                           float* tile_sums, float* block_sums, float* head_sum, float* inv_s, float* inv_e,
+                           float* inv_norm, float* a_raw, uint32_t* mm, int* ctrl, int* status, int sm_count,
+                           cudaStream_t stream, int64_t* launches) {
     const int units = G * K.H;
     CUtensorMap tmap;
     cudaError_t e = encode_key_map(K, G, kSlabRows, &tmap);
@@ -893,7 +979,7 @@ cudaError_t launch_keypass(const TensorView& K, int G, const ScoreParams& sp, co
     const int T = (K.N + kTile - 1) / kTile;
     const int tiles_per_block = sp.block / kTile;
     // pieces are whole blocks; small calls take smaller pieces so that every SM gets several
-    int tpp = opt.tiles_per_piece > 0 ? opt.tiles_per_piece : 8;
+    int tpp = opt.tiles_per_piece > 0 ? opt.tiles_per_piece : 16;
     if (opt.tiles_per_piece <= 0)
         while (tpp > tiles_per_block && (int64_t)units * ((T + tpp - 1) / tpp) < 4LL * sm_count) tpp >>= 1;
     tpp = (tpp + tiles_per_block - 1) / tiles_per_block * tiles_per_block;
@@ -901,12 +987,10 @@ cudaError_t launch_keypass(const TensorView& K, int G, const ScoreParams& sp, co
     a.pieces = (T + tpp - 1) / tpp;
     const int64_t total = (int64_t)units * a.pieces;
     const unsigned grid = (unsigned)(total < sm_count ? total : sm_count);
-    // the second touch of a head starts once its last piece has had time to finish: one head's pieces plus
-    // one round of the grid behind the first touch
-    a.lag_items = opt.lag_items > 0 ? opt.lag_items : (long long)a.pieces + (long long)grid + grid / 4;
     a.hints = opt.hints;
     a.debug = opt.debug;
-    a.flag_spin_limit = opt.flag_spin_limit > 0 ? (uint32_t)opt.flag_spin_limit : (1u << 20);
+    a.flag_spin_limit = opt.flag_spin_limit > 0 ? (uint32_t)opt.flag_spin_limit : (1u << 21);
+    a.tile_sums = tile_sums;
     a.block_sums = block_sums;
     a.head_sum = head_sum;
     a.inv_s = inv_s;
@@ -914,7 +998,8 @@ cudaError_t launch_keypass(const TensorView& K, int G, const ScoreParams& sp, co
     a.inv_norm = inv_norm;
     a.a_raw = a_raw;
     a.mm = mm;
-    a.next_item = reinterpret_cast<unsigned long long*>(ctrl);
+    a.next_a = reinterpret_cast<unsigned long long*>(ctrl);
+    a.next_b = reinterpret_cast<unsigned long long*>(ctrl) + 1;
     a.head_count = ctrl + 4;
     a.head_ready = ctrl + 4 + units;
     a.status = status;

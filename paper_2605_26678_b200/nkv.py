@@ -431,7 +431,7 @@ def nkv_set_key_passes(mode: str = "auto", h: Optional[Handle] = None) -> None:
     _check(h.lib.nkv_set_key_passes(h.h, KEY_PASS[mode]), "nkv_set_key_passes")
 
 
-DEBUG = {"tiles_per_piece": 0, "lag_items": 1, "l2_hints": 2, "hold_head_flags": 3, "flag_spin_limit": 4,
+DEBUG = {"tiles_per_piece": 0, "l2_hints": 2, "hold_head_flags": 3, "flag_spin_limit": 4,
          "inject_host_status": 5, "separate_passes": 6}
 
 
