@@ -39,7 +39,9 @@
 // Warps of a CTA: two teams of 8 warps take the first-touch tiles in turn (4 warps: norms, backward sums,
 // tile sums; 4 warps: forward sums, prefix scan, a_c), so two tiles are in flight and a team's chain of
 // tensor-memory round trips overlaps the other team's; 4 warps build the split anchors of the second touch
-// and turn its accumulators into a_s, a_e; one TMA producer thread and one MMA issuer thread per pipeline.
+// and turn its accumulators into a_s, a_e; one TMA producer thread and one MMA issuer warp per
+// pipeline.  The teams keep pieces of the accumulators in registers, so after start-up the other warp groups
+// hand registers over to them (setmaxnreg).
 // Keys are staged by TMA in two rings of 128-row slots (64-row slabs, 128-byte swizzle); hand-overs are
 // mbarriers and named barriers inside a team; every wait is bounded.
 #include "nkv_sm100.cuh"
@@ -71,11 +73,15 @@ constexpr uint32_t kColMain0 = 0, kColCorner = 192, kColMain1 = 256, kColTsum = 
 constexpr uint32_t kTmemCols = 512;
 
 // warps: team 0 = 0..7, team 1 = 8..15 (first four backward, last four forward), second touch 16..19,
-// then one thread each of warps 20..23
+// then warps 20..23 (producers: one thread each; issuers: lane 0 issues)
 constexpr int kTeamThreads = 256;
 constexpr int kBWarp0 = 16, kProdAWarp = 20, kProdBWarp = 21, kMmaAWarp = 22, kMmaBWarp = 23;
 constexpr int kThreads = 24 * 32;
-constexpr int kConsumersA = 17, kConsumersB = 5;   // warps (or single threads) that read a pipeline's queue
+constexpr int kConsumersA = 17, kConsumersB = 5;
+constexpr int kLaunchRegs = 80;                    // 65536 / kThreads rounded down to a multiple of 8
+constexpr int kTeamRegs = 96, kOtherRegs = 40;     // registers per thread after the warp groups rebalance them
+// the CTA can only redistribute what it was given at launch; asking for more would wait forever
+static_assert(16 * 32 * kTeamRegs + 8 * 32 * kOtherRegs <= kLaunchRegs * kThreads, "register pool exceeded");   // warps (or single threads) that read a pipeline's queue
 
 struct Item {
     int end, u, g, h, row0, ntiles;
@@ -127,7 +133,7 @@ struct Smem {
     uint64_t cempty;                    // corner accumulator read
     uint64_t wpub[kHist];                   // norms of a tile are in the ring
     uint64_t spub[kHist];                   // carry and restart parts of a tile are written
-    uint64_t done[kHist];                   // every global write of a tile has been issued and fenced
+    uint64_t done[kHist];                   // the other team's global writes of a piece are fenced
     uint64_t wsready[2];                // split norms written
     uint64_t tsfull[2], tsempty[2];     // tile-sum accumulators
     uint64_t rready[2], rfree[2];       // split anchors
@@ -143,17 +149,21 @@ struct Waiter {
     volatile int* abort;
 };
 
-// Bounded wait that also leaves when another role of the CTA has given up.
-__device__ __forceinline__ bool bwait(uint64_t* bar, uint32_t parity, const Waiter& wt, int where) {
-    if (mbar_try_wait(bar, parity)) return true;
+// Bounded wait that also leaves when another role of the CTA has given up.  The polling loop is kept out of
+// line: the kernel's roles run side by side and share the instruction cache.
+__device__ __forceinline__ bool bwait_slow(uint64_t* bar, uint32_t parity, int* status, volatile int* abort, int where) {
     for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (*wt.abort) return false;
+        if (*abort) return false;
         if (spin >= 8) __nanosleep(spin < 64 ? 32 : 128);
     }
-    set_status(wt.status, NKV_ERR_TIMEOUT, where);
-    *wt.abort = 1;
+    set_status(status, NKV_ERR_TIMEOUT, where);
+    *abort = 1;
     return false;
+}
+__device__ __forceinline__ bool bwait(uint64_t* bar, uint32_t parity, const Waiter& wt, int where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return bwait_slow(bar, parity, wt.status, wt.abort, where);
 }
 
 // Descriptor `cnt` of a pipeline's queue.  kWarp: the whole warp calls (one release per warp); else one thread.
@@ -216,7 +226,7 @@ __device__ __forceinline__ void settle_loads(uint64_t* full, int slots, long lon
 }
 
 // First-touch producer (one thread): draws pieces, publishes them, stages halo + tiles.
-__device__ void producer_a(const CUtensorMap* tmap, unsigned char* ring, Smem* s, const KeyPassArgs& p, const Waiter& wt) {
+__device__ __forceinline__ void producer_a(const CUtensorMap* tmap, unsigned char* ring, Smem* s, const KeyPassArgs& p, const Waiter& wt) {
     const uint64_t pol = l2_policy_evict_last();
     const bool hint = (p.hints & 1) != 0;
     long long n = 0, ic = 0;
@@ -261,7 +271,7 @@ __device__ void producer_a(const CUtensorMap* tmap, unsigned char* ring, Smem* s
 }
 
 // Second-touch producer (one thread).
-__device__ void producer_b(const CUtensorMap* tmap, unsigned char* ring, Smem* s, const KeyPassArgs& p, const Waiter& wt) {
+__device__ __forceinline__ void producer_b(const CUtensorMap* tmap, unsigned char* ring, Smem* s, const KeyPassArgs& p, const Waiter& wt) {
     const uint64_t pol = l2_policy_evict_first();
     const bool hint = (p.hints & 2) != 0;
     long long n = 0, ic = 0;
@@ -291,93 +301,115 @@ __device__ void producer_b(const CUtensorMap* tmap, unsigned char* ring, Smem* s
 }
 
 // ---------------------------------------------------------------------------- MMA issuers
-// First touch (one thread).  Tile n of the CTA goes to the accumulator of team n & 1.
-__device__ void mma_a(unsigned char* ring, unsigned char* wsplit, Smem* s, uint32_t tmem, const Waiter& wt) {
+// Offset of K step kk (16 columns) in descriptor units of 16 bytes, for a K-major operand whose two
+// 64-column halves are `half_bytes` apart.
+__device__ __forceinline__ constexpr uint64_t kstep(int kk, uint32_t half_bytes) {
+    return (uint64_t)(((uint32_t)(kk >> 2) * half_bytes + (uint32_t)(kk & 3) * 32u) >> 4);
+}
+
+// Lane 0's value in every lane; also tells the compiler that the value is the same across the warp, so
+// that descriptor arithmetic can stay in the uniform datapath the MMA instruction reads its operands from.
+__device__ __forceinline__ uint32_t uni(uint32_t x) { return __shfl_sync(0xffffffffu, x, 0); }
+__device__ __forceinline__ uint64_t uni(uint64_t x) {
+    return ((uint64_t)uni((uint32_t)(x >> 32)) << 32) | uni((uint32_t)x);
+}
+
+// Products of the first touch (one warp; lane 0 issues).  Tile n of the CTA goes to the accumulator of
+// team n & 1.  After the Gram and corner products of tile n come the tile-sum product of tile n - 1 (its
+// norms are known by then) and the release of that tile's slot, which the products of tile n still read.
+__device__ __forceinline__ void mma_a(unsigned char* ring, unsigned char* wsplit, Smem* s, uint32_t tmem, const Waiter& wt) {
     constexpr uint32_t idesc192 = umma_idesc_bf16(kTile, 192), idesc128 = umma_idesc_bf16(kTile, 128);
     constexpr uint32_t idesc64 = umma_idesc_bf16(kTile, 64);
     constexpr uint32_t idesc_ts = umma_idesc_bf16(kD, 16) | kUmmaAMajorMN;
     const uint32_t ring_a = smem_addr(ring), ws_a = smem_addr(wsplit);
+    const bool leader = (threadIdx.x & 31) == 0;
     long long n = 0, nC = 0, nS = 0, ic = 0;
-    int pend_slot = -1;
-    bool pend_real = false;
-    // The tile whose slot is still read: issue its tile-sum product (real tiles) and release the slot.
+    int prev_slot = -1;
+    bool prev_real = false;
+    // Tile sum of the previous tile (real tiles) and release of its slot.
     auto flush = [&]() -> bool {
-        if (pend_slot < 0) return true;
-        if (pend_real) {
+        if (prev_slot < 0) return true;
+        if (prev_real) {
             const int b = (int)(nS & 1);
             if (!bwait(&s->wsready[b], (uint32_t)((nS >> 1) & 1), wt, 741)) return false;
             if (!bwait(&s->tsempty[b], (uint32_t)(((nS >> 1) & 1) ^ 1), wt, 742)) return false;
             tc_fence_after();
-            const uint32_t a0 = ring_a + (uint32_t)(1 + 2 * pend_slot) * kSlabHalfBytes;
+            const uint64_t rows = uni(umma_desc_sw128_mn(ring_a + (uint32_t)(1 + 2 * prev_slot) * kSlabHalfBytes, kHalfBytes));
+            const uint64_t wdesc = uni(umma_desc_sw128(ws_a + (uint32_t)b * kOperandBytes));
+            const uint32_t dsum = uni(tmem + kColTsum + 16u * (uint32_t)b);
+            if (leader) {
 #pragma unroll
-            for (int kk = 0; kk < kTile / 16; ++kk) {
-                const uint64_t adesc = umma_desc_sw128_mn(a0 + (uint32_t)kk * 2048u, kHalfBytes);
-                const uint64_t bdesc = umma_desc_sw128(ws_a + (uint32_t)b * kOperandBytes + (uint32_t)(kk >> 2) * 2048u +
-                                                       (uint32_t)(kk & 3) * 32u);
-                umma_bf16(tmem + kColTsum + 16u * (uint32_t)b, adesc, bdesc, idesc_ts, kk > 0);
+                for (int kk = 0; kk < kTile / 16; ++kk)
+                    umma_bf16(dsum, rows + (uint64_t)(kk * (2048 >> 4)), wdesc + kstep(kk, 2048u), idesc_ts, kk > 0);
+                umma_commit(&s->tsfull[b]);
             }
-            umma_commit(&s->tsfull[b]);
             ++nS;
         }
-        umma_commit(&s->free_a[pend_slot]);
-        pend_slot = -1;
+        if (leader) umma_commit(&s->free_a[prev_slot]);
+        __syncwarp();
+        prev_slot = -1;
         return true;
     };
     for (;;) {
         Item it;
-        if (!get_item<false>(s->qa, s->qa_full, s->qa_free, ic++, it, wt, 743)) return;
+        if (!get_item<true>(s->qa, s->qa_full, s->qa_free, ic++, it, wt, 743)) return;
         if (it.end) break;
         for (int tl = 0; tl <= it.ntiles; ++tl, ++n) {
             const int slot = (int)(n % kSlotsA), par = (int)(n & 1);
             if (!bwait(&s->full_a[slot], (uint32_t)((n / kSlotsA) & 1), wt, 744)) return;
             if (!bwait(&s->tempty[par], (uint32_t)(((n >> 1) & 1) ^ 1), wt, 745)) return;
-            if (tl > 0 && !bwait(&s->cempty, (uint32_t)((nC & 1) ^ 1), wt, 746)) return;
             tc_fence_after();
-            const uint32_t dmain = tmem + (par ? kColMain1 : kColMain0);
-            const uint32_t a0 = ring_a + (uint32_t)(1 + 2 * slot) * kSlabHalfBytes;
+            const uint32_t dmain = uni(tmem + (par ? kColMain1 : kColMain0));
+            const uint64_t own = uni(umma_desc_sw128(ring_a + (uint32_t)(1 + 2 * slot) * kSlabHalfBytes));
             if (tl == 0) {
                 // halo: Gram of the 128 rows with themselves, columns 64..191 of the accumulator
+                if (leader) {
 #pragma unroll
-                for (int kk = 0; kk < kD / 16; ++kk) {
-                    const uint32_t koff = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
-                    umma_bf16(dmain + 64u, umma_desc_sw128(a0 + koff), umma_desc_sw128(a0 + koff), idesc128, kk > 0);
+                    for (int kk = 0; kk < kD / 16; ++kk)
+                        umma_bf16(dmain + 64u, own + kstep(kk, kHalfBytes), own + kstep(kk, kHalfBytes), idesc128, kk > 0);
                 }
             } else {
-                const uint32_t b0 = ring_a + (uint32_t)(2 * slot) * kSlabHalfBytes;   // the slab before the tile
+                const uint64_t wide = uni(umma_desc_sw128(ring_a + (uint32_t)(2 * slot) * kSlabHalfBytes));   // from the slab before
+                if (leader) {
 #pragma unroll
-                for (int kk = 0; kk < kD / 16; ++kk) {
-                    const uint32_t koff = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
-                    umma_bf16(dmain, umma_desc_sw128(a0 + koff), umma_desc_sw128(b0 + koff), idesc192, kk > 0);
+                    for (int kk = 0; kk < kD / 16; ++kk)
+                        umma_bf16(dmain, own + kstep(kk, kHalfBytes), wide + kstep(kk, kHalfBytes), idesc192, kk > 0);
                 }
-                const uint32_t pa = ring_a + (uint32_t)(1 + 2 * (int)((n - 1) % kSlotsA)) * kSlabHalfBytes;
+                if (!bwait(&s->cempty, (uint32_t)((nC & 1) ^ 1), wt, 746)) return;
+                tc_fence_after();
+                const uint64_t prev = uni(umma_desc_sw128(ring_a + (uint32_t)(1 + 2 * prev_slot) * kSlabHalfBytes));
+                const uint32_t dcorner = uni(tmem + kColCorner);
+                if (leader) {
 #pragma unroll
-                for (int kk = 0; kk < kD / 16; ++kk) {
-                    const uint32_t koff = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
-                    umma_bf16(tmem + kColCorner, umma_desc_sw128(pa + koff), umma_desc_sw128(a0 + koff), idesc64, kk > 0);
+                    for (int kk = 0; kk < kD / 16; ++kk)
+                        umma_bf16(dcorner, prev + kstep(kk, kHalfBytes), own + kstep(kk, kHalfBytes), idesc64, kk > 0);
                 }
                 ++nC;
             }
-            umma_commit(&s->tfull[par]);
+            if (leader) umma_commit(&s->tfull[par]);
+            __syncwarp();
             if (!flush()) return;
-            pend_slot = slot;
-            pend_real = tl > 0;
+            prev_slot = slot;
+            prev_real = tl > 0;
         }
     }
     if (!flush()) return;
     // every product issued has completed before the accumulators are given back
-    umma_commit(&s->drain_a);
+    if (leader) umma_commit(&s->drain_a);
+    __syncwarp();
     bwait(&s->drain_a, 0, wt, 747);
 }
 
-// Second touch (one thread): the tiles of a block share one pair of split anchors.
-__device__ void mma_b(unsigned char* ring, unsigned char* rhs, Smem* s, uint32_t tmem, int tiles_per_block,
+// Second touch (one warp; lane 0 issues): the tiles of a block share one pair of split anchors.
+__device__ __forceinline__ void mma_b(unsigned char* ring, unsigned char* rhs, Smem* s, uint32_t tmem, int tiles_per_block,
                       const Waiter& wt) {
     constexpr uint32_t idesc16 = umma_idesc_bf16(kTile, 16);
     const uint32_t ring_a = smem_addr(ring), rhs_a = smem_addr(rhs);
+    const bool leader = (threadIdx.x & 31) == 0;
     long long n = 0, nR = 0, ic = 0;
     for (;;) {
         Item it;
-        if (!get_item<false>(s->qb, s->qb_full, s->qb_free, ic++, it, wt, 748)) return;
+        if (!get_item<true>(s->qb, s->qb_full, s->qb_free, ic++, it, wt, 748)) return;
         if (it.end) break;
         for (int tl = 0; tl < it.ntiles; ++tl, ++n) {
             const int slot = (int)(n % kSlotsB), b = (int)(n & 1), rb = (int)(nR & 1);
@@ -385,23 +417,24 @@ __device__ void mma_b(unsigned char* ring, unsigned char* rhs, Smem* s, uint32_t
             if (!bwait(&s->full_b[slot], (uint32_t)((n / kSlotsB) & 1), wt, 750)) return;
             if (!bwait(&s->dempty[b], (uint32_t)(((n >> 1) & 1) ^ 1), wt, 751)) return;
             tc_fence_after();
-            const uint32_t a0 = ring_a + (uint32_t)(kSlabsA + 2 * slot) * kSlabHalfBytes;
+            const uint64_t rows = uni(umma_desc_sw128(ring_a + (uint32_t)(kSlabsA + 2 * slot) * kSlabHalfBytes));
+            const uint64_t anchors = uni(umma_desc_sw128(rhs_a + (uint32_t)rb * kOperandBytes));
+            const uint32_t ddots = uni(tmem + kColDots + 16u * (uint32_t)b);
+            const bool last_of_block = (tl + 1) % tiles_per_block == 0 || tl + 1 == it.ntiles;
+            if (leader) {
 #pragma unroll
-            for (int kk = 0; kk < kD / 16; ++kk) {
-                const uint32_t koff = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
-                const uint64_t bdesc = umma_desc_sw128(rhs_a + (uint32_t)rb * kOperandBytes + (uint32_t)(kk >> 2) * 2048u +
-                                                       (uint32_t)(kk & 3) * 32u);
-                umma_bf16(tmem + kColDots + 16u * (uint32_t)b, umma_desc_sw128(a0 + koff), bdesc, idesc16, kk > 0);
+                for (int kk = 0; kk < kD / 16; ++kk)
+                    umma_bf16(ddots, rows + kstep(kk, kHalfBytes), anchors + kstep(kk, 2048u), idesc16, kk > 0);
+                umma_commit(&s->dfull[b]);
+                umma_commit(&s->free_b[slot]);
+                if (last_of_block) umma_commit(&s->rfree[rb]);
             }
-            umma_commit(&s->dfull[b]);
-            umma_commit(&s->free_b[slot]);
-            if ((tl + 1) % tiles_per_block == 0 || tl + 1 == it.ntiles) {
-                umma_commit(&s->rfree[rb]);
-                ++nR;
-            }
+            __syncwarp();
+            if (last_of_block) ++nR;
         }
     }
-    umma_commit(&s->drain_b);
+    if (leader) umma_commit(&s->drain_b);
+    __syncwarp();
     bwait(&s->drain_b, 0, wt, 752);
 }
 
@@ -478,7 +511,7 @@ __device__ __forceinline__ float select_lane(const float* v, int lane) {
 
 // The team that completed a head's last piece: block sums, head sum and the reciprocals of their norms
 // (256 threads, `tid` inside the team, `bar` the team's named barrier).
-__device__ void finalise_head(TeamSmem* ts, const KeyPassArgs& p, int u, int tid, int bar) {
+__device__ __forceinline__ void finalise_head(TeamSmem* ts, const KeyPassArgs& p, int u, int tid, int bar) {
     const int nb = p.sp.nblocks, T = (p.N + kTile - 1) / kTile, tpb = p.sp.block / kTile;
     const float* tsum = p.tile_sums + (size_t)u * T * kD;
     float* bs = p.block_sums + (size_t)u * nb * kD;
@@ -514,7 +547,7 @@ __device__ void finalise_head(TeamSmem* ts, const KeyPassArgs& p, int u, int tid
 }
 
 // One team (8 warps) takes every second first-touch tile of the CTA.
-__device__ void team_role(int team, unsigned char* wsplit, Smem* s, uint32_t tmem, const KeyPassArgs& p,
+__device__ __forceinline__ void team_role(int team, unsigned char* wsplit, Smem* s, uint32_t tmem, const KeyPassArgs& p,
                           const Waiter& wt) {
     const int tid = threadIdx.x - team * kTeamThreads, warp = tid >> 5, lane = tid & 31;
     const int q = warp & 3, side = warp >> 2;   // quarter of the tile's rows; 0 backward band, 1 forward band
@@ -669,9 +702,6 @@ __device__ void team_role(int team, unsigned char* wsplit, Smem* s, uint32_t tme
                     hi = fmaxf(hi, a_c);
                 }
             }
-            __threadfence();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&s->done[slot4]);
         }
         // ---- end of the piece: min/max of the team's tiles
         if (side == 1) {
@@ -682,8 +712,14 @@ __device__ void team_role(int team, unsigned char* wsplit, Smem* s, uint32_t tme
                 ts->red[2 * q + 1] = hi;
             }
         }
-        const bool owner = (int)(n_last & 1) == team;   // this team took the piece's last tile
-        if (owner) ok = bwait(&s->done[(n_last - 1) & (kHist - 1)], (uint32_t)(((n_last - 1) / kHist) & 1), wt, 758) && ok;
+        // every write of the piece is fenced before the piece is counted: the team that did not take the
+        // last tile reports, the other one waits for that report
+        const bool owner = (int)(n_last & 1) == team;
+        const int pslot = (int)((ic - 1) & (kHist - 1));
+        __threadfence();
+        __syncwarp();
+        if (!owner && lane == 0) mbar_arrive(&s->done[pslot]);
+        if (owner) ok = bwait(&s->done[pslot], (uint32_t)(((ic - 1) / kHist) & 1), wt, 758) && ok;
         if (bar_or(bar_team, kTeamThreads, !ok)) return;
         if (tid == 128) {
             for (int w = 0; w < 4; ++w) {
@@ -728,7 +764,7 @@ __device__ __forceinline__ int ld_acquire(const int* ptr) {
 // Four warps.  Thread k writes column k of the six anchor rows (rows 6..15 stay zero): the head sum and the
 // sum of the block, each as hi + mid + lo in bf16; thread r reads row r of a tile's accumulator: the key's
 // dots with the head sum and with its block's sum.
-__device__ void second_touch_role(unsigned char* rhs, Smem* s, uint32_t tmem, const KeyPassArgs& p, const Waiter& wt) {
+__device__ __forceinline__ void second_touch_role(unsigned char* rhs, Smem* s, uint32_t tmem, const KeyPassArgs& p, const Waiter& wt) {
     const int r = threadIdx.x - kBWarp0 * 32, q = r >> 5, lane = r & 31;
     const int half = r >> 6, kk = r & 63;
     const int N = p.N, nb = p.sp.nblocks, tpb = p.sp.block / kTile;
@@ -894,16 +930,22 @@ key_pass_kernel(const __grid_constant__ CUtensorMap tmap, const KeyPassArgs p) {
     wt.status = p.status;
     wt.abort = &s->abort;
 
+    // The teams hold tiles of the accumulators in registers; the other two warp groups (warps 16..19 and
+    // 20..23) give registers up for them.  Every warp of a warp group runs the same instruction here.
+    if (warp < 16) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kTeamRegs));
+    else asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
     if (warp < 16) {
         team_role(warp >> 3, wsplit, s, tmem, p, wt);
     } else if (warp < kProdAWarp) {
         second_touch_role(rhs, s, tmem, p, wt);
+    } else if (warp == kMmaAWarp) {
+        mma_a(ring, wsplit, s, tmem, wt);
+    } else if (warp == kMmaBWarp) {
+        mma_b(ring, rhs, s, tmem, p.sp.block / kTile, wt);
     } else {
         if (lane == 0) {
             if (warp == kProdAWarp) producer_a(&tmap, ring, s, p, wt);
-            else if (warp == kProdBWarp) producer_b(&tmap, ring, s, p, wt);
-            else if (warp == kMmaAWarp) mma_a(ring, wsplit, s, tmem, wt);
-            else mma_b(ring, rhs, s, tmem, p.sp.block / kTile, wt);
+            else producer_b(&tmap, ring, s, p, wt);
         }
         __syncwarp();
     }
