@@ -139,19 +139,105 @@ def test_positive_rescaling_invariance(N, d):
     assert np.array_equal(h1.a_star, h2.a_star)
 
 
-def test_minmax_range_and_affine_shift():
-    """Normalised scales span exactly [0,1]; a common shift of the raw anomaly
-    (the '1 - cos' convention) cannot change anything downstream."""
+def test_minmax_uses_the_heads_own_extremes():
+    """The oracle's lo / hi are the extremes of its own raw anomalies, every normalised scale
+    attains 0 and 1, and the head statistics are consistent with them (Section 2.3)."""
     rng = np.random.default_rng(11)
     K = _rand_keys(rng, 200, 16)
-    ref = bf.final_score(K)
-    for k in range(3):
-        assert ref["an"][k].min() == 0.0 and ref["an"][k].max() == 1.0
     h = oracle.score_head(K)
+    assert np.array_equal(h.lo, h.a_raw.min(1)) and np.array_equal(h.hi, h.a_raw.max(1))
     an = (h.a_raw - h.lo[:, None]) / (h.hi - h.lo)[:, None]
-    shifted = ((h.a_raw + 1.0) - (h.lo + 1.0)[:, None]) / (h.hi - h.lo)[:, None]
-    assert np.allclose(an, shifted, atol=1e-15)
-    assert np.allclose(1.0 + np.array([-1.0]), 0.0)
+    for k in range(3):
+        assert an[k].min() == 0.0 and an[k].max() == 1.0
+    # the reliability gap of a scale is a difference of means of values in [0, 1]
+    assert np.all(h.delta >= 0.0) and np.all(h.delta <= 1.0)
+
+
+def _two_direction_case():
+    """Keys alternate between two orthogonal directions (N = 100, one block, W = 64).  Then a_s and a_e are
+    constant (their normalised scales are identically 0) and the window anomaly is known in closed form:
+    a_c(i) = -p / sqrt(p^2 + q^2) with p keys of i's own direction and q of the other in the window."""
+    N, d = 100, 8
+    K = np.zeros((N, d), np.float32)
+    K[0::2, 0] = 5.0
+    K[1::2, 1] = 0.25
+    i = np.arange(N)
+    n = np.minimum(i + 1, 64)
+    p_own = (n + 1) // 2
+    q = n - p_own
+    a_c = -p_own / np.sqrt(p_own.astype(np.float64) ** 2 + q ** 2)
+    return K, a_c
+
+
+def test_surprise_gate_chain_closed_form():
+    """Section 2.4 and Appendix A on an input where every quantity follows by hand.
+
+    With a_tilde_s = a_tilde_e = 0 and x = a_tilde_c: the population std of (0, 0, x) is x sqrt(2)/3, so the
+    surprise is proportional to x and its per-head min-max is x itself; centring and rectifying give
+    s' = max(0, x - mean x); the gate is sigma(kappa (s' - tau)); Delta_s = Delta_e = 0 and Delta_c is the
+    gap of x; the blend is w_c x, the winner is x, so a_star = (1 - alpha) w_c x + alpha x."""
+    K, a_c = _two_direction_case()
+    N = len(a_c)
+    x = (a_c - a_c.min()) / (a_c.max() - a_c.min())
+    m = 10                                              # max(1, floor(0.10 * 100))
+    srt = np.sort(x)
+    delta_c = srt[-m:].mean() - srt[:m].mean()
+    z = np.log(np.array([0.4, 0.4, 0.2])) + 3.0 * np.array([0.0, 0.0, delta_c])
+    w = np.exp(z - z.max())
+    w /= w.sum()
+    s_prime = np.maximum(0.0, x - x.mean())
+    alpha = 1.0 / (1.0 + np.exp(-10.0 * (s_prime - 0.60)))
+    want = (1.0 - alpha) * w[2] * x + alpha * x
+
+    h = oracle.score_head(K)
+    assert np.allclose(h.delta, [0.0, 0.0, delta_c], atol=1e-12)
+    assert np.allclose(h.w, w, atol=1e-12)
+    # surprise statistics: min 0, max sqrt(2)/3 (at x = 1), mean of the normalised surprise = mean x
+    assert abs(h.s_min) < 1e-12 and abs(h.s_max - math.sqrt(2.0) / 3.0) < 1e-12
+    assert abs(h.s_mean - x.mean()) < 1e-12
+    assert np.all(np.isinf(h.a_star[:4]))
+    assert np.allclose(h.a_star[4:], want[4:].astype(np.float32), atol=1e-7)
+
+    # the gate grows with the surprise: alpha = (a_star - w_c x) / (x - w_c x) where x > 0
+    pos = np.arange(N)[4:][x[4:] > 1e-6]
+    a64 = h.a_star.astype(np.float64)
+    alpha_seen = (a64[pos] - w[2] * x[pos]) / (x[pos] - w[2] * x[pos])
+    order = np.argsort(x[pos], kind="stable")
+    assert np.all(np.diff(alpha_seen[order]) >= -1e-6)
+
+    # plausible misreadings of Appendix A give visibly different scores on this input, so the
+    # comparison above would catch them: threshold applied to the normalised surprise before
+    # centring, and rectifying before centring
+    alt1 = 1.0 / (1.0 + np.exp(-10.0 * (x - 0.60)))
+    alt2 = 1.0 / (1.0 + np.exp(-10.0 * ((np.maximum(0.0, x) - x.mean()) - 0.60)))
+    for alt in (alt1, alt2):
+        other = (1.0 - alt) * w[2] * x + alt * x
+        assert np.max(np.abs(other[4:] - want[4:])) > 5e-4    # 5000 times the tolerance of the comparison
+
+
+def test_gate_parameters_move_the_closed_form():
+    """The same input with other (beta, tau, kappa, priors): every constant enters where Section 2.4 puts it."""
+    K, a_c = _two_direction_case()
+    x = (a_c - a_c.min()) / (a_c.max() - a_c.min())
+    p = oracle.default_params()
+    p.beta, p.tau, p.kappa = 1.5, 0.2, 4.0
+    p.prior[0], p.prior[1], p.prior[2] = 0.5, 0.2, 0.3
+    srt = np.sort(x)
+    delta_c = srt[-10:].mean() - srt[:10].mean()
+    z = np.log(np.array([0.5, 0.2, 0.3])) + 1.5 * np.array([0.0, 0.0, delta_c])
+    w = np.exp(z - z.max())
+    w /= w.sum()
+    alpha = 1.0 / (1.0 + np.exp(-4.0 * (np.maximum(0.0, x - x.mean()) - 0.2)))
+    want = (1.0 - alpha) * w[2] * x + alpha * x
+    h = oracle.score_head(K, p)
+    assert np.allclose(h.w, w, atol=1e-12)
+    assert np.allclose(h.a_star[4:], want[4:].astype(np.float32), atol=1e-7)
+    # with the gate half open the two misreadings of the centring order are far away
+    alt1 = 1.0 / (1.0 + np.exp(-4.0 * (x - 0.2)))
+    alt2 = 1.0 / (1.0 + np.exp(-4.0 * ((np.maximum(0.0, x) - x.mean()) - 0.2)))
+    for alt in (alt1, alt2):
+        other = (1.0 - alt) * w[2] * x + alt * x
+        assert np.max(np.abs(other[4:] - want[4:])) > 2e-2
 
 
 def test_weights_softmax_properties():
