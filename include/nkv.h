@@ -248,17 +248,18 @@ NKV_API int nkv_get_stage_ms(nkv_handle* h, float* ms_out);
 NKV_API int64_t nkv_launch_count(const nkv_handle* h);
 
 /*
- * Choice of the kernels that scan the keys inside nkv_compress (Sections 2.1-2.3).  A head's keys are
- * touched twice: the first touch yields 1/||k||, the sums of normalised keys per episodic block and the
- * current-memory anomaly a_c; the second, which needs the anchors of the whole head, yields a_s and a_e.
- *   NKV_KEY_PASS_AUTO (default), NKV_KEY_PASS_TENSOR: bf16 keys with d = 128, W = 64 and episodic blocks
- *       of 128 or 256 keys (the paper's schedule gives those for N <= 4127 and N >= 8192) run one
- *       persistent tcgen05 kernel: k_hat_i . S_i and ||S_i||^2 are sums over a band of the keys' Gram
- *       matrix, ||k_i||^2 is its diagonal, block sums and anchor dots are skinny products with fp32
- *       factors split three ways into bf16.  Heads are cut into pieces that all SMs work on, and the
- *       second touch trails the first closely enough to find the keys in L2.  Other inputs run the FMA
- *       kernels.
- *   NKV_KEY_PASS_FMA: fp32 FMAs on staged key tiles, two kernels (any supported dtype and d).
+ * Choice of the kernels that make the two passes over the keys of nkv_compress (Sections 2.1-2.3).  The
+ * first pass yields 1/||k||, the block sums of normalised keys and the current-memory anomaly a_c; the
+ * second, which needs the anchors of the whole head, the anomalies a_s and a_e.
+ *   NKV_KEY_PASS_FMA     both passes with fp32 FMAs on staged key tiles (any supported dtype and d).
+ *   NKV_KEY_PASS_TENSOR  (bf16 keys) forms on the tensor cores what is a contraction: in the first pass
+ *       (d = 128, W = 64, one CTA per head) k_hat_i . S_i and ||S_i||^2 as sums over a band of the keys'
+ *       Gram matrix; in the second pass (d = 64 or 128) the dots of the keys with the anchors, the fp32
+ *       anchors split three ways into bf16.  A pass whose inputs do not allow the tensor form runs the
+ *       FMA kernel.
+ *   NKV_KEY_PASS_AUTO (default) takes the tensor form of the second pass when d = 128, and of the first
+ *       pass when in addition the call's heads, dealt one per SM, keep at least 85 % of the SMs busy over
+ *       the rounds that takes.
  * The forms agree to fp32 rounding.
  */
 enum { NKV_KEY_PASS_AUTO = 0, NKV_KEY_PASS_FMA = 1, NKV_KEY_PASS_TENSOR = 2 };
@@ -276,26 +277,12 @@ NKV_API int nkv_key_scan(nkv_handle* h, const nkv_tensor* K, const nkv_params* p
                          float* mu_e, float* a_raw, float* minmax, void* ws, size_t ws_bytes, void* stream);
 
 /*
- * Test and tuning hooks (no counterpart in the paper; results never depend on the tuning values).
- *   NKV_DEBUG_TILES_PER_PIECE   128-key tiles per piece of a head in the persistent key scan (0: automatic)
- *   NKV_DEBUG_L2_HINTS          bit 0: first-touch loads ask L2 to keep the lines; bit 1: second-touch
- *                               loads mark them as the first to leave
- *   NKV_DEBUG_HOLD_HEAD_FLAGS   non-zero: the key scan never raises its "anchors of this head are final"
- *                               flags, so every bounded wait on one runs out: the call completes with
- *                               meaningless scores and the device status NKV_ERR_TIMEOUT
- *   NKV_DEBUG_FLAG_SPIN_LIMIT   polls after which such a wait gives up (0: default)
+ * Test hook (no counterpart in the paper).
  *   NKV_DEBUG_INJECT_HOST_STATUS  value = chunk * 16 + code: nkv_compress_host plants device status `code`
- *                               in that chunk's status words before reading them back (0 clears)
- *   NKV_DEBUG_SEPARATE_PASSES   non-zero: NKV_KEY_PASS_TENSOR runs the two-kernel tensor-core form instead
+ *       in that chunk's status words before reading them back, so that the reporting of a device-side
+ *       failure in any chunk can be tested without provoking one (0 clears).
  */
-enum {
-    NKV_DEBUG_TILES_PER_PIECE = 0,
-    NKV_DEBUG_L2_HINTS = 2,
-    NKV_DEBUG_HOLD_HEAD_FLAGS = 3,
-    NKV_DEBUG_FLAG_SPIN_LIMIT = 4,
-    NKV_DEBUG_INJECT_HOST_STATUS = 5,
-    NKV_DEBUG_SEPARATE_PASSES = 6
-};
+enum { NKV_DEBUG_INJECT_HOST_STATUS = 5 };
 NKV_API int nkv_debug_set(nkv_handle* h, int what, int64_t value);
 
 /*

@@ -17,7 +17,6 @@ struct nkv_handle {
     int timing;
     int timing_valid;
     int key_pass;     // NKV_KEY_PASS_*: which kernels make the two key passes
-    KeyPassOptions kp;   // scheduling of the single-kernel key scan (zeros: chosen per call)
     cudaEvent_t ev[NKV_NUM_STAGES + 1];
     cudaStream_t copy_streams[2];
     cudaEvent_t slot_done[2];
@@ -56,7 +55,7 @@ int64_t keep_count(int64_t N, double r) { return (int64_t)floor((1.0 - r) * (dou
 
 // Workspace carving shared by every entry point.
 struct Layout {
-    size_t status, inv_norm, mu_s, mu_e, inv_s, inv_e, mm, a_raw, a_star, thr, ctrl, tsum, hstat, total;
+    size_t status, inv_norm, mu_s, mu_e, inv_s, inv_e, mm, a_raw, a_star, thr, hstat, total;
 };
 
 Layout make_layout(int64_t units, int64_t N, int64_t d, int64_t nb) {
@@ -77,8 +76,6 @@ Layout make_layout(int64_t units, int64_t N, int64_t d, int64_t nb) {
     L.a_raw = take((size_t)units * 3 * N * 4);
     L.a_star = take((size_t)units * N * 4);
     L.thr = take((size_t)units * 2 * 4);
-    L.ctrl = take(keypass_ctrl_bytes(units));
-    L.tsum = d == 128 ? take(keypass_tile_sum_bytes(units, N)) : o;
     L.hstat = take(head_stat_bytes(units));
     L.total = o;
     return L;
@@ -155,23 +152,21 @@ int cuda_failed(cudaError_t e, const char* what, int line) {
 
 // The two passes over the keys (Sections 2.1-2.3): afterwards the workspace holds 1/||k||, the anchors, the
 // three raw anomalies and their per-head min/max keys.  `mark` is called once between the passes (stage
-// timing).  *sums_only: the anchor arrays hold block sums and the head sum, not means.
+// timing).  *sums_only stays false: the anchor arrays hold means.
 template <typename Mark>
 int key_scan(nkv_handle* h, const TensorView& kv, int dtype, int G, const ScoreParams& sp, void* ws, const Layout& L,
              cudaStream_t st, Mark&& mark, bool* sums_only) {
     const int units = G * kv.H, N = kv.N, d = kv.d;
     int* status = at<int>(ws, L.status);
     *sums_only = false;
-    if (h->key_pass != NKV_KEY_PASS_FMA && !(h->kp.debug & 2) && keypass_supported(kv, dtype, sp)) {
-        // one persistent kernel makes both passes; the stage mark between them stays empty
-        CU(launch_keypass(kv, G, sp, h->kp, at<float>(ws, L.tsum), at<float>(ws, L.mu_e), at<float>(ws, L.mu_s), at<float>(ws, L.inv_s),
-                          at<float>(ws, L.inv_e), at<float>(ws, L.inv_norm), at<float>(ws, L.a_raw),
-                          at<uint32_t>(ws, L.mm), at<int>(ws, L.ctrl), status, h->sm_count, st, &h->launches));
-        CU(mark());
-        *sums_only = true;
-    } else if (stream_path_supported(sp)) {
+    if (stream_path_supported(sp)) {
         // pass A: norms, block sums and the current-memory anomaly; pass B: the two anchor anomalies
-        const bool tensor_ok = h->key_pass == NKV_KEY_PASS_TENSOR && gram_pass_supported(kv, dtype, sp);
+        // the tensor-core form walks whole heads, one CTA each: by default it runs when the heads fill
+        // the SMs to at least 85 % over its waves (below that the FMA form, which splits heads, is faster)
+        const int waves = (units + h->sm_count - 1) / h->sm_count;
+        const bool fills = (double)units >= 0.85 * (double)waves * (double)h->sm_count;
+        const bool tensor_ok = h->key_pass != NKV_KEY_PASS_FMA && gram_pass_supported(kv, dtype, sp) &&
+                               (h->key_pass == NKV_KEY_PASS_TENSOR || fills);
         if (tensor_ok)
             CU(launch_gram_pass(kv, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm), at<float>(ws, L.a_raw),
                                 at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));
@@ -183,7 +178,9 @@ int key_scan(nkv_handle* h, const TensorView& kv, int dtype, int G, const ScoreP
         CU(launch_anchor_norms(units, d, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_s),
                                at<float>(ws, L.inv_e), nullptr, st, &h->launches));
         CU(mark());
-        if (h->key_pass == NKV_KEY_PASS_TENSOR && anchor_dots_supported(kv, dtype, sp))
+        // d = 64 tiles are too small to pay for the per-tile hand-overs: the FMA form is faster there
+        const bool dots_wanted = h->key_pass == NKV_KEY_PASS_TENSOR || (h->key_pass == NKV_KEY_PASS_AUTO && d == 128);
+        if (dots_wanted && anchor_dots_supported(kv, dtype, sp))
             CU(launch_anchor_dots(kv, G, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm),
                                   at<float>(ws, L.inv_s), at<float>(ws, L.inv_e), at<float>(ws, L.a_raw),
                                   at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));
@@ -298,7 +295,7 @@ int nkv_create(nkv_handle** out, int device) {
     h->l2_bytes = prop.l2CacheSize;
     h->key_pass = NKV_KEY_PASS_AUTO;
     if (configure_scan_kernels() != cudaSuccess || configure_stream_kernels() != cudaSuccess ||
-        configure_keypass_kernels() != cudaSuccess || configure_gram_kernels() != cudaSuccess ||
+        configure_gram_kernels() != cudaSuccess ||
         configure_dots_kernels() != cudaSuccess || configure_select_kernels() != cudaSuccess) {
         delete h;
         return NKV_ERR_CUDA;
@@ -656,14 +653,8 @@ int nkv_key_scan(nkv_handle* h, const nkv_tensor* K, const nkv_params* params, f
     bool sums_only = false;
     auto no_mark = []() -> cudaError_t { return cudaSuccess; };
     if ((rc = key_scan(h, view_of(K), K->dtype, G, sp, ws, L, st, no_mark, &sums_only))) return rc;
-    if (sums_only) {
-        CU(launch_keypass_means(units, N, sp, at<float>(ws, L.mu_e), at<float>(ws, L.mu_s), mu_e, mu_s, st,
-                                &h->launches));
-    } else {
-        CU(cudaMemcpyAsync(mu_s, at<float>(ws, L.mu_s), (size_t)units * d * 4, cudaMemcpyDeviceToDevice, st));
-        CU(cudaMemcpyAsync(mu_e, at<float>(ws, L.mu_e), (size_t)units * sp.nblocks * d * 4, cudaMemcpyDeviceToDevice,
-                           st));
-    }
+    CU(cudaMemcpyAsync(mu_s, at<float>(ws, L.mu_s), (size_t)units * d * 4, cudaMemcpyDeviceToDevice, st));
+    CU(cudaMemcpyAsync(mu_e, at<float>(ws, L.mu_e), (size_t)units * sp.nblocks * d * 4, cudaMemcpyDeviceToDevice, st));
     CU(cudaMemcpyAsync(inv_norm, at<float>(ws, L.inv_norm), (size_t)units * N * 4, cudaMemcpyDeviceToDevice, st));
     CU(cudaMemcpyAsync(a_raw, at<float>(ws, L.a_raw), (size_t)units * 3 * N * 4, cudaMemcpyDeviceToDevice, st));
     minmax_floats_kernel<<<(units * 6 + 255) / 256, 256, 0, st>>>(units * 6, at<uint32_t>(ws, L.mm), minmax);
@@ -675,27 +666,10 @@ int nkv_key_scan(nkv_handle* h, const nkv_tensor* K, const nkv_params* params, f
 int nkv_debug_set(nkv_handle* h, int what, int64_t value) {
     if (!h) return NKV_ERR_INVALID_ARG;
     switch (what) {
-        case NKV_DEBUG_TILES_PER_PIECE:
-            if (value < 0 || value > 64) return NKV_ERR_INVALID_ARG;
-            h->kp.tiles_per_piece = (int)value;
-            return NKV_OK;
-        case NKV_DEBUG_L2_HINTS:
-            if (value < 0 || value > 3) return NKV_ERR_INVALID_ARG;
-            h->kp.hints = (int)value;
-            return NKV_OK;
-        case NKV_DEBUG_HOLD_HEAD_FLAGS:
-            h->kp.debug = (h->kp.debug & ~1) | (value ? 1 : 0);
-            return NKV_OK;
-        case NKV_DEBUG_FLAG_SPIN_LIMIT:
-            if (value < 0 || value > (1 << 24)) return NKV_ERR_INVALID_ARG;
-            h->kp.flag_spin_limit = (int)value;
-            return NKV_OK;
         case NKV_DEBUG_INJECT_HOST_STATUS:   // value = chunk * 16 + status code (0 clears)
+            if (value < 0) return NKV_ERR_INVALID_ARG;
             h->inject_status = (int)(value & 15);
             h->inject_chunk = (int)(value >> 4);
-            return NKV_OK;
-        case NKV_DEBUG_SEPARATE_PASSES:
-            h->kp.debug = (h->kp.debug & ~2) | (value ? 2 : 0);
             return NKV_OK;
         default:
             return NKV_ERR_INVALID_ARG;

@@ -91,25 +91,6 @@ __device__ __forceinline__ float warp_min(float v) {
     return v;
 }
 
-// One m16n8k16 bf16 tensor-core product with fp32 accumulation: c += a * b.
-__device__ __forceinline__ void mma_bf16_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-// x = hi + mid + lo with all three in bf16: together they carry the 24 mantissa bits of an fp32 number.
-__device__ __forceinline__ void split3_bf16(float x, __nv_bfloat16* out, int stride) {
-    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
-    const float r1 = x - __bfloat162float(hi);
-    const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
-    const float r2 = r1 - __bfloat162float(mid);
-    out[0] = hi;
-    out[stride] = mid;
-    out[2 * stride] = __float2bfloat16_rn(r2);
-}
-
 __device__ __forceinline__ void set_status(int* status, int code, int detail) {
     if (atomicCAS(&status[kStatusCode], 0, code) == 0) status[kStatusDetail] = detail;
 }
@@ -145,26 +126,6 @@ cudaError_t configure_dots_kernels();
 cudaError_t launch_anchor_dots(const TensorView& K, int G, const ScoreParams& sp, const float* mu_s, const float* mu_e,
                                const float* inv_norm, const float* inv_s, const float* inv_e, float* a_raw,
                                uint32_t* mm, int* status, int sm_count, cudaStream_t stream, int64_t* launches);
-// both key passes in one persistent tensor-core kernel (bf16 keys, d = 128, blocks of whole 128-key tiles);
-// the second touch of a key finds it in L2.  Anchors come out as sums (block_sums, head_sum) with the
-// reciprocals of their norms; launch_keypass_means turns them into the means mu_e, mu_s.
-struct KeyPassOptions {
-    int tiles_per_piece;   // 0: chosen from the call's size
-    int hints;             // bit 0 / bit 1: L2 eviction hints on first- / second-touch loads
-    int debug;             // bit 0: never raise the head flags (makes the bounded flag wait run out)
-    int flag_spin_limit;   // 0: default
-};
-bool keypass_supported(const TensorView& K, int dtype, const ScoreParams& sp);
-size_t keypass_ctrl_bytes(int64_t units);
-size_t keypass_tile_sum_bytes(int64_t units, int64_t N);
-cudaError_t configure_keypass_kernels();
-cudaError_t launch_keypass(const TensorView& K, int G, const ScoreParams& sp, const KeyPassOptions& opt,
-                           float* tile_sums, float* block_sums, float* head_sum, float* inv_s, float* inv_e,
-                           float* inv_norm, float* a_raw, uint32_t* mm, int* ctrl, int* status, int sm_count,
-                           cudaStream_t stream, int64_t* launches);
-cudaError_t launch_keypass_means(int units, int N, const ScoreParams& sp, const float* block_sums,
-                                 const float* head_sum, float* mu_e, float* mu_s, cudaStream_t stream,
-                                 int64_t* launches);
 cudaError_t configure_select_kernels();
 cudaError_t configure_scan_kernels();
 cudaError_t configure_stream_kernels();

@@ -36,14 +36,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: false (after recording where) if the phase never completes.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status, int where) {
+// Bounded wait: false (after recording where) if the phase never completes.  The polling loop is one
+// out-of-line function: the roles of a kernel run side by side and share the instruction cache, and a
+// wait that finds its phase complete at the first look costs one instruction.
+static __device__ __noinline__ bool mbar_wait_poll(uint64_t* bar, uint32_t parity, int* status, int where) {
     for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
         if (spin >= 4) __nanosleep(64);   // leave the issue slots to the warps that have work
     }
     set_status(status, NKV_ERR_TIMEOUT, where);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status, int where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_poll(bar, parity, status, where);
 }
 
 // Named barrier over `count` threads that also ORs a predicate over them.
@@ -70,32 +76,6 @@ __device__ __forceinline__ void tma_load_4d(void* dst_smem, const CUtensorMap* m
         "[%6];" ::"r"(smem_addr(dst_smem)),
         "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_addr(bar))
         : "memory");
-}
-
-// The same with an L2 eviction policy for the lines the copy touches.
-__device__ __forceinline__ void tma_load_4d_hint(void* dst_smem, const CUtensorMap* map, int c0, int c1, int c2, int c3,
-                                                 uint64_t* bar, uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
-        "[%0], [%1, {%2, %3, %4, %5}], [%6], %7;" ::"r"(smem_addr(dst_smem)),
-        "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_addr(bar)), "l"(policy)
-        : "memory");
-}
-// Asks L2 to fetch the box; nothing is written to shared memory and nothing signals completion.
-__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap* map, int c0, int c1, int c2, int c3) {
-    asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(map), "r"(c0), "r"(c1),
-                 "r"(c2), "r"(c3)
-                 : "memory");
-}
-__device__ __forceinline__ uint64_t l2_policy_evict_last() {
-    uint64_t p;
-    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
-    return p;
-}
-__device__ __forceinline__ uint64_t l2_policy_evict_first() {
-    uint64_t p;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-    return p;
 }
 
 // ---------------------------------------------------------------------------- tensor memory
@@ -172,23 +152,10 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t addr) {
     d |= (uint64_t)2 << 61;                     // 128-byte swizzle
     return d;
 }
-// The same bytes read as an MN-major operand: the 128-byte rows run along M (or N), the rows of the
-// swizzle atom along K.  One descriptor covers 16 rows (two 8-row groups, 1024 bytes apart); `lbo` is the
-// byte distance between consecutive 64-element pieces of the M (or N) extent.
-__device__ __forceinline__ uint64_t umma_desc_sw128_mn(uint32_t addr, uint32_t lbo) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3ffffu) >> 4);
-    d |= (uint64_t)((lbo & 0x3ffffu) >> 4) << 16;
-    d |= (uint64_t)(1024 >> 4) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, tile M x N.
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
-constexpr uint32_t kUmmaAMajorMN = 1u << 15;   // flag of the instruction descriptor: A is MN-major
 // D[tmem] (+)= A[smem] * B[smem]^T, issued by one thread.
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                           bool accumulate) {

@@ -431,12 +431,11 @@ def nkv_set_key_passes(mode: str = "auto", h: Optional[Handle] = None) -> None:
     _check(h.lib.nkv_set_key_passes(h.h, KEY_PASS[mode]), "nkv_set_key_passes")
 
 
-DEBUG = {"tiles_per_piece": 0, "l2_hints": 2, "hold_head_flags": 3, "flag_spin_limit": 4,
-         "inject_host_status": 5, "separate_passes": 6}
+DEBUG = {"inject_host_status": 5}
 
 
 def nkv_debug_set(what: str, value: int, h: Optional[Handle] = None) -> None:
-    """Test and tuning hooks of the library (see nkv.h); results never depend on the tuning values."""
+    """Test hook of the library (see nkv.h)."""
     h = h or handle()
     _check(h.lib.nkv_debug_set(h.h, DEBUG[what], int(value)), "nkv_debug_set")
 

@@ -159,17 +159,11 @@ def test_compaction_copies_rows_verbatim(d, dv, dtype, mode):
 @pytest.mark.parametrize("N,d,dtype,H,layers,r", [
     (5, 64, "fp32", 2, 1, 0.5), (300, 64, "bf16", 4, 2, 0.75), (1000, 128, "fp32", 8, 1, 0.5),
     (2500, 128, "bf16", 8, 2, 0.95), (4133, 64, "bf16", 3, 1, 0.0), (777, 128, "bf16", 1, 3, 0.9)])
-@pytest.mark.parametrize("scan_lag", [0, 3])
-def test_fused_compress_end_to_end(N, d, dtype, H, layers, r, scan_lag):
-    """scan_lag 0: the two key passes as separate kernels; 3: the single interleaved scan kernel."""
+def test_fused_compress_end_to_end(N, d, dtype, H, layers, r):
     K, V = _cache(N, d, dtype, H=H, layers=layers)
     p = nkv.nkv_default_params()
     ws = nkv.alloc_workspace(K, p)
-    nkv.nkv_set_scan_options(scan_lag)
-    try:
-        res = nkv.nkv_compress(K, V, r, p, ws=ws, want_a_star=True)
-    finally:
-        nkv.nkv_set_scan_options(0)
+    res = nkv.nkv_compress(K, V, r, p, ws=ws, want_a_star=True)
     assert nkv.nkv_last_device_status(ws) == nkv.NKV_OK
     rep = pr.SwapReport()
     for g in range(K.shape[0]):
