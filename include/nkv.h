@@ -21,7 +21,8 @@
  *     0-based.  All pointers in nkv_tensor and all array arguments are DEVICE
  *     pointers unless an argument says "host".  Strides are in elements; d is
  *     contiguous, stride_n must equal d, every row start is 16-byte aligned.
- *     d is 64 or 128, dtype bf16 or fp32, 1 <= window <= 64.
+ *     d is 64 or 128, dtype bf16 or fp32, 2 <= window <= 64 (with a window of one key the
+ *     current anchor is the key itself and that scale carries no information).
  *   - Every buffer is caller-owned.  No entry point except nkv_create,
  *     nkv_destroy and nkv_compress_host allocates, frees or synchronises; work
  *     is enqueued on the given stream (a cudaStream_t passed as void*, NULL =
@@ -81,7 +82,8 @@ typedef struct nkv_params {
     int32_t block_max;
     int32_t gate_mode;  /* nkv_gate_mode */
     double top_frac;    /* p of the reliability gap, 0.10 */
-    double prior[3];    /* (w_s^0, w_e^0, w_c^0) = (0.4, 0.4, 0.2); entries > 0 */
+    double prior[3];    /* (w_s^0, w_e^0, w_c^0) = (0.4, 0.4, 0.2); entries >= 0, not all 0; a zero
+                           switches its scale off (single-anchor and no-current ablations) */
     double beta;        /* 3.0 */
     double tau;         /* 0.60 */
     double kappa;       /* 10.0 */

@@ -36,8 +36,13 @@ bool params_ok(const nkv_params* p) {
     if (!p) return false;
     if (p->n_sink < 0 || p->block_div < 1 || p->block_min < 1 || p->block_max < p->block_min) return false;
     if (!(p->top_frac > 0.0 && p->top_frac <= 1.0)) return false;
-    for (int k = 0; k < 3; ++k)
-        if (!(p->prior[k] > 0.0) || !isfinite(p->prior[k])) return false;
+    // a prior of zero switches its scale off (the single-anchor and no-current ablations); one must remain
+    double prior_sum = 0.0;
+    for (int k = 0; k < 3; ++k) {
+        if (!(p->prior[k] >= 0.0) || !isfinite(p->prior[k])) return false;
+        prior_sum += p->prior[k];
+    }
+    if (!(prior_sum > 0.0)) return false;
     if (!isfinite(p->beta) || !isfinite(p->tau) || !isfinite(p->kappa)) return false;
     if (!(p->safeguard >= 0.0 && p->safeguard <= 1.0)) return false;
     if (p->gate_mode < NKV_GATE_SURPRISE || p->gate_mode > NKV_GATE_MAX) return false;
@@ -114,7 +119,9 @@ TensorView view_of(const nkv_tensor* t) {
 
 int resolve_params(const nkv_params* p, int64_t N, ScoreParams* sp) {
     if (!params_ok(p)) return NKV_ERR_INVALID_ARG;
-    if (p->window < 1 || p->window > kMaxWindow) return NKV_ERR_UNSUPPORTED;
+    // W = 1 makes the current anchor the key itself: a_c is the constant -1 and its per-head min-max would
+    // normalise rounding noise, so the smallest window is 2
+    if (p->window < 2 || p->window > kMaxWindow) return NKV_ERR_UNSUPPORTED;
     sp->window = p->window;
     sp->n_sink = p->n_sink;
     sp->block = (int)block_size(N, p);

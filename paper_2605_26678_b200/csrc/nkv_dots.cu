@@ -44,6 +44,7 @@ struct Smem {
     uint64_t kfree[kMaxSlots];  // tile and right-hand side consumed by the MMAs
     uint64_t tfull[kStages];    // accumulator written
     uint64_t tempty[kStages];   // accumulator read (one arrival per reading warp)
+    uint64_t drain;             // products issued before a give-up have completed
     uint32_t tmem_base;
 };
 template <int D>
@@ -72,7 +73,14 @@ __device__ void dots_producer(const CUtensorMap* tmap, unsigned char* tiles, Sme
     for (long long t = tr.first; t < tr.last; ++t, ++n) {
         const int slot = (int)(n % C::kSlots);
         const long long fill = n / C::kSlots;
-        if (fill > 0 && !mbar_wait(&s->kfree[slot], (uint32_t)((fill - 1) & 1), status, 711)) return;
+        if (fill > 0 && !mbar_wait(&s->kfree[slot], (uint32_t)((fill - 1) & 1), status, 711)) {
+            // giving up: the copies already armed still land in this CTA's shared memory, so stay (bounded)
+            // until they have
+            for (long long m = n > C::kSlots ? n - C::kSlots : 0; m < n; ++m)
+                for (uint32_t spin = 0; spin < (1u << 16) && !mbar_try_wait(&s->full[m % C::kSlots], (uint32_t)((m / C::kSlots) & 1)); ++spin)
+                    __nanosleep(256);
+            return;
+        }
         const int u = (int)(t / tr.tiles_per_unit);
         const int i0 = (int)(t - (long long)u * tr.tiles_per_unit) * kTile;
         const int g = u / H, h = u - g * H;
@@ -94,9 +102,14 @@ __device__ void dots_mma(unsigned char* tiles, unsigned char* rhs, Smem* s, uint
     for (long long t = tr.first; t < tr.last; ++t, ++n) {
         const int slot = (int)(n % C::kSlots), stage = (int)(n % kStages);
         const uint32_t fpar = (uint32_t)((n / C::kSlots) & 1), upar = (uint32_t)((n / kStages) & 1);
-        if (!mbar_wait(&s->full[slot], fpar, status, 712)) return;
-        if (!mbar_wait(&s->rready[slot], fpar, status, 713)) return;
-        if (!mbar_wait(&s->tempty[stage], upar ^ 1u, status, 714)) return;
+        if (!mbar_wait(&s->full[slot], fpar, status, 712) || !mbar_wait(&s->rready[slot], fpar, status, 713) ||
+            !mbar_wait(&s->tempty[stage], upar ^ 1u, status, 714)) {
+            // products already issued keep reading shared memory and writing tensor memory: wait (bounded)
+            // for them before the CTA frees both
+            umma_commit(&s->drain);
+            for (uint32_t spin = 0; spin < (1u << 16) && !mbar_try_wait(&s->drain, 0); ++spin) __nanosleep(256);
+            return;
+        }
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
@@ -259,6 +272,7 @@ anchor_dots_kernel(const __grid_constant__ CUtensorMap tmap, ScoreParams sp, int
             mbar_init(&s->tfull[i], 1);
             mbar_init(&s->tempty[i], 4);
         }
+        mbar_init(&s->drain, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = tid; i < C::kSlots * C::kRhsBytes / 16; i += kThreads) reinterpret_cast<uint4*>(rhs)[i] = make_uint4(0, 0, 0, 0);

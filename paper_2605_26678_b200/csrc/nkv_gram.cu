@@ -72,6 +72,7 @@ struct Smem {
     uint64_t wready[kWReady];    // norms of a span written
     uint64_t cready[kCfRing];    // band sums of a tile written
     uint64_t cfree[kCfRing];     // band sums of a tile consumed
+    uint64_t drain;              // products issued before a give-up have completed
     uint32_t tmem_base;
 };
 constexpr size_t kSmemBytes = 1024 + kRingBytes + sizeof(Smem);
@@ -126,7 +127,17 @@ __device__ void producer_role(const CUtensorMap* tmap, unsigned char* ring, Smem
             int p;
             uint32_t fc;
             slab_slot(q, p, fc);
-            if (fc > 0 && !mbar_wait(&s->sfree[p], (fc - 1) & 1u, status, 701)) return;
+            if (fc > 0 && !mbar_wait(&s->sfree[p], (fc - 1) & 1u, status, 701)) {
+                // giving up: the copies already armed still land in this CTA's shared memory, so stay (bounded)
+                // until the last ring of them has
+                for (long long m = q > kRing ? q - kRing : 0; m < q; ++m) {
+                    int pm;
+                    uint32_t fm;
+                    slab_slot(m, pm, fm);
+                    for (uint32_t spin = 0; spin < (1u << 16) && !mbar_try_wait(&s->full[pm], fm & 1u); ++spin) __nanosleep(256);
+                }
+                return;
+            }
             mbar_expect_tx(&s->full[p], (p == 0 ? 4 : 2) * kSlabHalfBytes);
             for (int copy = 0; copy < (p == 0 ? 2 : 1); ++copy) {
                 unsigned char* dst = ring + (size_t)(copy ? kRing : p) * kSlabHalfBytes;
@@ -139,6 +150,13 @@ __device__ void producer_role(const CUtensorMap* tmap, unsigned char* ring, Smem
 
 // MMA issuer (one thread).  Tile tau of a head: A = slabs 2 tau + 1, 2 tau + 2 (the tile's rows),
 // B = slabs 2 tau .. 2 tau + 3 as two pairs, two MMAs of N = 128 per 16-wide K step.
+// Products already issued keep reading shared memory and writing tensor memory: a role that gives up
+// waits (bounded) for them before the CTA frees both.
+__device__ __forceinline__ void drain_products(Smem* s) {
+    umma_commit(&s->drain);
+    for (uint32_t spin = 0; spin < (1u << 16) && !mbar_try_wait(&s->drain, 0); ++spin) __nanosleep(256);
+}
+
 __device__ void mma_role(unsigned char* ring, Smem* s, uint32_t tmem_base, int units, int T, int* status) {
     constexpr uint32_t idesc = umma_idesc_bf16(kTile, 128);
     const uint32_t ring_addr = smem_addr(ring);
@@ -149,10 +167,10 @@ __device__ void mma_role(unsigned char* ring, Smem* s, uint32_t tmem_base, int u
             uint32_t fc;
             for (int lam = tau == 0 ? 0 : 2 * tau + 2; lam <= 2 * tau + 3; ++lam) {
                 slab_slot(hb + lam, p, fc);
-                if (!mbar_wait(&s->full[p], fc & 1u, status, 702)) return;
+                if (!mbar_wait(&s->full[p], fc & 1u, status, 702)) return drain_products(s);
             }
             const int st = (int)(gt & 1);
-            if (!mbar_wait(&s->tempty[st], (uint32_t)(((gt >> 1) & 1) ^ 1), status, 703)) return;
+            if (!mbar_wait(&s->tempty[st], (uint32_t)(((gt >> 1) & 1) ^ 1), status, 703)) return drain_products(s);
             tc_fence_after();
             int pa;
             slab_slot(hb + 2 * tau + 1, pa, fc);
@@ -486,6 +504,7 @@ gram_pass_kernel(const __grid_constant__ CUtensorMap tmap, ScoreParams sp, int u
             mbar_init(&s->tfull[i], 1);
             mbar_init(&s->tempty[i], 1);
         }
+        mbar_init(&s->drain, 1);
         for (int i = 0; i < kWReady; ++i) mbar_init(&s->wready[i], 1);
         for (int i = 0; i < kCfRing; ++i) {
             mbar_init(&s->cready[i], 1);

@@ -3,8 +3,8 @@
 Tolerances (fp32 scores): |delta| <= 1e-4 absolute or 1e-4 relative.  Integer outputs
 (budgets, positions, ranks) and compacted bytes are compared exactly; when the GPU's own
 scores feed the integer stages, a token may legitimately swap in or out only if its oracle
-score lies within the tolerance of a threshold that the selection used, and such swaps are
-counted.
+score lies within the tolerance (plus the observed score difference of that token) of a
+threshold that the selection used, and such swaps are counted.
 """
 from __future__ import annotations
 
@@ -66,38 +66,46 @@ class SwapReport:
 
 
 def compare_selection(a_star_oracle: np.ndarray, sel: "oracle.GroupSelection", gpu_budgets: np.ndarray,
-                      gpu_idx: np.ndarray, gpu_offsets: np.ndarray, report: SwapReport, tol=TOL):
-    """One group: exact match, or every differing token is a near-tie of a used threshold."""
+                      gpu_idx: np.ndarray, gpu_offsets: np.ndarray, report: SwapReport, tol=TOL, n_safe=None,
+                      a_star_gpu=None):
+    """One group: exact match, or every differing token is a near-tie of a threshold the selection used.
+
+    The thresholds are, per head, the smallest retained score and the n_safe-th best score (the safeguard
+    threshold), and the smallest score retained anywhere in the group (the cross-head competition).  A token
+    may change sides only if its oracle score is within tol + |gpu - oracle| of one of them: two scores that
+    each carry at most `tol` of error can swap only when they are that close."""
     H, N = a_star_oracle.shape
-    # thresholds the oracle's selection used: per head the smallest retained score, and the
-    # smallest score retained through cross-head competition anywhere in the group
-    finite_max = float(np.nanmax(np.where(np.isfinite(a_star_oracle), a_star_oracle, -np.inf)))
-    head_thr, all_thr = [], []
+    finite = np.where(np.isfinite(a_star_oracle), a_star_oracle, -np.inf)
+    finite_max = float(finite.max())
+    head_thr = []
     for h in range(H):
         rows = sel.idx[sel.offsets[h]:sel.offsets[h + 1]]
         t = float(a_star_oracle[h, rows].min()) if len(rows) else np.inf
-        if np.isinf(t):
-            t = finite_max
-        head_thr.append(t)
-    group_thr = min(head_thr)
+        thr = [finite_max if np.isinf(t) else t]
+        if n_safe is not None and 0 < n_safe <= N:
+            t2 = float(np.sort(a_star_oracle[h])[::-1][n_safe - 1])
+            thr.append(finite_max if np.isinf(t2) else t2)
+        head_thr.append(thr)
+    group_thr = min(t[0] for t in head_thr)
     for h in range(H):
         report.heads += 1
         want = set(sel.idx[sel.offsets[h]:sel.offsets[h + 1]].tolist())
         got = set(gpu_idx[gpu_offsets[h]:gpu_offsets[h + 1]].tolist())
         assert len(got) == gpu_budgets[h], "head %d: %d positions for budget %d" % (h, len(got), gpu_budgets[h])
+        diff = want ^ got
         if gpu_budgets[h] != sel.budgets[h]:
             report.budget_mismatch_heads += 1
-        diff = want ^ got
+            assert diff, "head %d: budgets differ but the position sets do not" % h
         if not diff:
             continue
         report.heads_with_swaps += 1
         report.swapped_tokens += len(diff)
         for i in diff:
             s = float(a_star_oracle[h, i])
-            near = min(abs(s - head_thr[h]), abs(s - group_thr))
-            # safeguard thresholds of other sizes also act; the nearest used threshold is what matters
-            assert near <= 4 * tol * max(1.0, abs(s)), (
-                "head %d token %d (score %.7f) changed sides but is %.3g away from the thresholds %.7f / %.7f"
+            near = min([abs(s - t) for t in head_thr[h]] + [abs(s - group_thr)])
+            seen = abs(float(a_star_gpu[h, i]) - s) if a_star_gpu is not None else tol
+            assert near <= (tol + seen) * max(1.0, abs(s)), (
+                "head %d token %d (score %.7f) changed sides but is %.3g away from the thresholds %s / %.7f"
                 % (h, i, s, near, head_thr[h], group_thr))
 
 
@@ -116,7 +124,8 @@ def check_group_against_oracle(K: torch.Tensor, V: torch.Tensor, res: "nkv.Compr
     H = K.shape[1]
     assert b.sum() == ref.sel.budgets.sum() == offs[H]
     assert np.array_equal(offs[1:] - offs[:-1], b)
-    compare_selection(ref.a_star, ref.sel, b, idx, offs, report)
+    compare_selection(ref.a_star, ref.sel, b, idx, offs, report, n_safe=nkv.nkv_safeguard_count(K.shape[2], r, params),
+                      a_star_gpu=None if res.a_star is None else res.a_star[g].cpu().numpy())
     # integer stages are exact given the GPU's own scores
     if res.a_star is not None:
         own = oracle.budget_select(res.a_star[g].cpu().numpy(), r, op)

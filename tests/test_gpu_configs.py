@@ -57,7 +57,8 @@ def _check_groups(cfg, K, V, groups, ratios, params):
             pr.assert_close(res.a_star[g].cpu().numpy(), a_ref, "a_star group %d" % g)
             sel = oracle.budget_select(a_ref, r, op)
             bud, idx, offs = pr.gpu_group_outputs(res, g)
-            pr.compare_selection(a_ref, sel, bud, idx, offs, rep)
+            pr.compare_selection(a_ref, sel, bud, idx, offs, rep, n_safe=nkv.nkv_safeguard_count(K.shape[2], r, params),
+                                 a_star_gpu=res.a_star[g].cpu().numpy())
             own = oracle.budget_select(res.a_star[g].cpu().numpy(), r, op)
             assert np.array_equal(own.budgets, bud) and np.array_equal(own.idx, idx)
             Kr, Vr = pr.raw_rows(K[g]), pr.raw_rows(V[g])
@@ -86,7 +87,9 @@ def test_benchmark_config_matches_oracle(name, groups):
     params = nkv.nkv_default_params()
     reports = _check_groups(cfg, K, V, groups, cfg.ratios, params)
     for r, rep in reports.items():
-        # swaps are tokens whose oracle score is within 4e-4 of a threshold (asserted inside); keep them rare
-        assert rep.swapped_tokens <= 4 * rep.heads, "too many near-tie swaps at r=%s" % r
+        # swaps are tokens whose oracle score is within tolerance of a threshold (asserted inside); the scores
+        # agree to about 1e-6, so at most a token or two per head may sit that close to a threshold
+        assert rep.swapped_tokens <= 2 * rep.heads, "too many near-tie swaps at r=%s" % r
+        assert rep.budget_mismatch_heads <= rep.heads_with_swaps
     del K, V
     torch.cuda.empty_cache()

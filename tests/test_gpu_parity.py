@@ -67,6 +67,59 @@ def test_scores_match_oracle(N, d, dtype):
         assert torch.isinf(a_star[0, h, :min(4, N)]).all()
 
 
+KEY_SCAN_CASES = [("fma", 1, 64, "fp32"), ("fma", 63, 128, "bf16"), ("fma", 257, 128, "bf16"), ("fma", 1000, 128, "fp32"),
+                  ("fma", 4133, 64, "bf16"), ("fma", 6000, 128, "bf16"), ("tensor", 100, 128, "bf16"),
+                  ("tensor", 257, 128, "bf16"), ("tensor", 2500, 128, "bf16"), ("tensor", 4352, 128, "bf16"),
+                  ("tensor", 8200, 128, "bf16"), ("tensor", 4133, 64, "bf16"), ("auto", 3000, 128, "bf16")]
+
+
+@pytest.mark.parametrize("mode,N,d,dtype", KEY_SCAN_CASES)
+def test_key_scan_intermediates_match_oracle(mode, N, d, dtype):
+    """The kernels nkv_compress times, stage by stage: 1/||k||, the anchors, the three raw anomalies and their
+    per-head extremes straight out of the key scan, for the FMA and the tensor-core form."""
+    K, _ = _cache(N, d, dtype, H=3)
+    p = nkv.nkv_default_params()
+    ws = nkv.alloc_workspace(K, p)
+    nkv.nkv_set_key_passes(mode)
+    try:
+        inv_norm, mu_s, mu_e, a_raw, minmax = nkv.nkv_key_scan(K, p, ws=ws)
+    finally:
+        nkv.nkv_set_key_passes("auto")
+    assert nkv.nkv_last_device_status(ws) == nkv.NKV_OK
+    for h in range(K.shape[1]):
+        ref = oracle.score_head(K[0, h].cpu())
+        pr.assert_close(inv_norm[0, h].cpu().numpy(), ref.inv_norm, "inv_norm", 1e-5)
+        pr.assert_close(mu_s[0, h].cpu().numpy(), ref.mu_s, "mu_s", 1e-5)
+        pr.assert_close(mu_e[0, h].cpu().numpy(), ref.mu_e, "mu_e", 1e-5)
+        pr.assert_close(a_raw[0, h].cpu().numpy(), ref.a_raw, "a_raw", 1e-5)
+        mm = minmax[0, h].cpu().numpy()
+        pr.assert_close(mm[0::2], ref.lo, "lo", 1e-5)
+        pr.assert_close(mm[1::2], ref.hi, "hi", 1e-5)
+
+
+@pytest.mark.parametrize("prior,gate", [((1.0, 0.0, 0.0), nkv.NKV_GATE_AVERAGE), ((0.5, 0.5, 0.0), nkv.NKV_GATE_AVERAGE),
+                                        ((0.5, 0.5, 0.0), nkv.NKV_GATE_SURPRISE), ((0.0, 0.0, 1.0), nkv.NKV_GATE_MAX)])
+def test_ablation_priors_switch_scales_off(prior, gate):
+    """Single-anchor scoring (the "w/o continuum" row of the ablation table) and scoring without the current
+    memory (the components table): a prior of zero removes a scale from the blend."""
+    K, V = _cache(1500, 128, "bf16", H=2)
+    p = nkv.nkv_default_params()
+    p.gate_mode = gate
+    for k in range(3):
+        p.prior[k] = prior[k]
+    res = nkv.nkv_compress(K, V, 0.75, p, want_a_star=True)
+    torch.cuda.synchronize()
+    for h in range(K.shape[1]):
+        ref = oracle.score_head(K[0, h].cpu(), pr.oracle_params(p))
+        assert [w == 0.0 for w in ref.w] == [x == 0.0 for x in prior]
+        pr.assert_close(res.a_star[0, h].cpu().numpy(), ref.a_star, "a_star")
+    if prior == (1.0, 0.0, 0.0):   # key distinctiveness: min-max of -cos(k_hat, mean k_hat)
+        a = res.a_star[0, 0, 4:].cpu().numpy()
+        ref = oracle.score_head(K[0, 0].cpu())
+        want = (ref.a_raw[0] - ref.lo[0]) / (ref.hi[0] - ref.lo[0])
+        pr.assert_close(a, want[4:], "single-anchor score")
+
+
 @pytest.mark.parametrize("gate,window,n_sink,prior", [
     (nkv.NKV_GATE_AVERAGE, 64, 4, (0.4, 0.4, 0.2)), (nkv.NKV_GATE_MAX, 64, 0, (0.4, 0.4, 0.2)),
     (nkv.NKV_GATE_SURPRISE, 2, 4, (0.2, 0.3, 0.5)), (nkv.NKV_GATE_SURPRISE, 17, 8, (0.4, 0.4, 0.2)),
@@ -130,9 +183,13 @@ def test_safeguard_one_gives_uniform_budgets():
 
 
 @pytest.mark.parametrize("d,dv,dtype,mode", [(128, 128, "bf16", "out"), (64, 64, "fp32", "out"),
-                                             (128, 128, "fp32", "in"), (64, 64, "bf16", "in")])
+                                             (128, 128, "fp32", "in"), (64, 64, "bf16", "in"),
+                                             (128, 64, "bf16", "out"), (64, 128, "fp32", "out"),
+                                             (128, 64, "bf16", "in")])
 def test_compaction_copies_rows_verbatim(d, dv, dtype, mode):
     K, V = _cache(900, d, dtype, H=3, layers=2)
+    if dv != d:   # values of another width (the paper's V in R^{N x d_v}): same rows, other row length
+        V = _cache(900, dv, dtype, H=3, layers=2, seed=12)[1]
     s = _random_scores(2, 3, 900, seed=5, ties="none")
     sel = [oracle.budget_select(s[g], 0.6) for g in range(2)]
     idx = torch.from_numpy(np.stack([x.idx for x in sel])).to(DEV)
@@ -254,11 +311,17 @@ def test_argument_errors_are_reported_not_thrown():
     with pytest.raises(nkv.NkvError) as e:
         nkv.nkv_compress(K[..., :48].contiguous(), V[..., :48].contiguous(), 0.5)
     assert e.value.status == nkv.NKV_ERR_UNSUPPORTED
+    for bad_window in (65, 1, 0):
+        p = nkv.nkv_default_params()
+        p.window = bad_window
+        with pytest.raises(nkv.NkvError) as e:
+            nkv.nkv_compress(K, V, 0.5, p)
+        assert e.value.status == nkv.NKV_ERR_UNSUPPORTED
     p = nkv.nkv_default_params()
-    p.window = 65
+    p.prior[0] = p.prior[1] = p.prior[2] = 0.0
     with pytest.raises(nkv.NkvError) as e:
         nkv.nkv_compress(K, V, 0.5, p)
-    assert e.value.status == nkv.NKV_ERR_UNSUPPORTED
+    assert e.value.status == nkv.NKV_ERR_INVALID_ARG
     with pytest.raises(nkv.NkvError) as e:
         nkv.nkv_compress(K, V, 0.5, ws=torch.empty(1024, dtype=torch.uint8, device=DEV))
     assert e.value.status == nkv.NKV_ERR_WORKSPACE
@@ -285,3 +348,39 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     assert torch.equal(out.idx, dev.idx.cpu()) and torch.equal(out.budgets, dev.budgets.cpu())
     assert torch.equal(out.head_offsets, dev.head_offsets.cpu())
     assert torch.equal(out.k_out, dev.k_out.cpu()) and torch.equal(out.v_out, dev.v_out.cpu())
+
+
+def test_too_many_heads_is_an_argument_error():
+    """More than 65535 heads in one call is refused before anything is launched."""
+    K = torch.zeros((8200, 8, 1, 64), dtype=torch.bfloat16, device=DEV)
+    before = nkv.nkv_launch_count()
+    with pytest.raises(nkv.NkvError) as e:
+        nkv.nkv_compress(K, K, 0.0)
+    assert e.value.status == nkv.NKV_ERR_UNSUPPORTED
+    assert nkv.nkv_launch_count() == before
+
+
+def test_host_entry_point_reports_a_device_status_of_any_chunk():
+    """A device-side status raised while any chunk runs comes back from nkv_compress_host: the status words
+    of every chunk are copied out before the chunk's slot is reused.  The status is planted by the library's
+    test hook, nothing on the device misbehaves."""
+    K, V = _cache(600, 64, "bf16", H=2, layers=6)
+    Kh, Vh = K.cpu().pin_memory(), V.cpu().pin_memory()
+    G, H, N, d = K.shape
+    k = nkv.nkv_keep_per_head(N, 0.5)
+    out = nkv.Compressed(torch.empty((G, H * k, d), dtype=K.dtype).pin_memory(),
+                         torch.empty((G, H * k, d), dtype=K.dtype).pin_memory(),
+                         torch.empty((G, H * k), dtype=torch.int32).pin_memory(),
+                         torch.empty((G, H + 1), dtype=torch.int32).pin_memory(),
+                         torch.empty((G, H), dtype=torch.int32).pin_memory(), None)
+    staging = torch.empty(nkv.nkv_host_staging_bytes(H, N, d, nkv.NKV_BF16, 0.5, 2), dtype=torch.uint8, device=DEV)
+    nkv.nkv_compress_host(Kh, Vh, 0.5, out, staging, 2)           # three chunks, all fine
+    for chunk, code in ((0, nkv.NKV_ERR_TIMEOUT), (1, nkv.NKV_ERR_DEVICE_CHECK), (2, nkv.NKV_ERR_TIMEOUT)):
+        nkv.nkv_debug_set("inject_host_status", chunk * 16 + code)
+        try:
+            with pytest.raises(nkv.NkvError) as e:
+                nkv.nkv_compress_host(Kh, Vh, 0.5, out, staging, 2)
+            assert e.value.status == code
+        finally:
+            nkv.nkv_debug_set("inject_host_status", 0)
+    nkv.nkv_compress_host(Kh, Vh, 0.5, out, staging, 2)           # and fine again
