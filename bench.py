@@ -50,7 +50,7 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="nkv", choices=["nkv", "reference"])
-    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(wl.CONFIGS))
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(wl.ALL_CONFIGS))
     ap.add_argument("--ratio", type=float, default=None)
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
@@ -408,7 +408,7 @@ def run_e2e(args, cfg, r, K, V, h, params, dist, dev, world):
 
 def main():
     args = parse_args()
-    cfg = wl.CONFIGS[args.workload]
+    cfg = wl.ALL_CONFIGS[args.workload]
     r = args.ratio if args.ratio is not None else (DEFAULT_RATIO if DEFAULT_RATIO in cfg.ratios else cfg.ratios[0])
     if args.impl == "reference":
         run_reference(args, cfg, r)

@@ -21,7 +21,7 @@
  *     0-based.  All pointers in nkv_tensor and all array arguments are DEVICE
  *     pointers unless an argument says "host".  Strides are in elements; d is
  *     contiguous, stride_n must equal d, every row start is 16-byte aligned.
- *     d is 64 or 128, dtype bf16 or fp32, 2 <= window <= 64 (with a window of one key the
+ *     d is 64 or 128, dtype bf16, fp16 or fp32 (fp16 keys run the FMA form of the key passes), 2 <= window <= 64 (with a window of one key the
  *     current anchor is the key itself and that scale carries no information).
  *   - Every buffer is caller-owned.  No entry point except nkv_create,
  *     nkv_destroy and nkv_compress_host allocates, frees or synchronises; work
@@ -63,7 +63,7 @@ typedef enum nkv_status {
     NKV_ERR_DEVICE_CHECK = 6  /* device status: a kernel self-check failed */
 } nkv_status;
 
-typedef enum nkv_dtype { NKV_BF16 = 0, NKV_F32 = 1 } nkv_dtype;
+typedef enum nkv_dtype { NKV_BF16 = 0, NKV_F32 = 1, NKV_F16 = 2 } nkv_dtype;
 
 /* Routing rule (Section 2.4); AVERAGE and MAX are the router-ablation variants. */
 typedef enum nkv_gate_mode { NKV_GATE_SURPRISE = 0, NKV_GATE_AVERAGE = 1, NKV_GATE_MAX = 2 } nkv_gate_mode;

@@ -18,7 +18,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "nkv_oracle.c")
 _LIB = os.path.join(_HERE, "libnkv_oracle.so")
 
-BF16, F32 = 0, 1
+BF16, F32, F16 = 0, 1, 2
 GATE_SURPRISE, GATE_AVERAGE, GATE_MAX = 0, 1, 2
 
 
@@ -113,7 +113,7 @@ def _ptr(a: Optional[np.ndarray]):
 
 
 def _as_bytes_2d(x) -> (np.ndarray, int):
-    """[N, d] array of bf16 (torch) / fp32 (torch or numpy) -> (contiguous numpy view, dtype code)."""
+    """[N, d] array of bf16 / fp16 (torch), fp16 / fp32 (numpy) -> (contiguous numpy view, dtype code)."""
     try:
         import torch
     except Exception:  # pragma: no cover
@@ -124,13 +124,17 @@ def _as_bytes_2d(x) -> (np.ndarray, int):
             return x.view(torch.int16).numpy().view(np.uint16), BF16
         if x.dtype == torch.float32:
             return x.numpy(), F32
-        raise TypeError("oracle accepts bf16 or fp32 keys, got %s" % x.dtype)
+        if x.dtype == torch.float16:
+            return x.view(torch.int16).numpy().view(np.uint16), F16
+        raise TypeError("oracle accepts bf16, fp16 or fp32 keys, got %s" % x.dtype)
     x = np.ascontiguousarray(x)
     if x.dtype == np.float32:
         return x, F32
     if x.dtype == np.uint16:
         return x, BF16
-    raise TypeError("oracle accepts float32 or raw-bf16 (uint16) arrays, got %s" % x.dtype)
+    if x.dtype == np.float16:
+        return x.view(np.uint16), F16
+    raise TypeError("oracle accepts float32, float16 or raw-bf16 (uint16) arrays, got %s" % x.dtype)
 
 
 @dataclass

@@ -3,7 +3,7 @@
  *
  * A plain, slow, single-threaded CPU statement of what the compression path
  * computes, written from the paper's definitions in the paper's order.  All
- * floating point is double; inputs (bf16 or fp32 bytes) are widened exactly.
+ * floating point is double; inputs (bf16, fp16 or fp32 bytes) are widened exactly.
  * There is no blocking, fusion, running sum or reordering: the sliding-window
  * mean is summed directly for every token and ranks come from full sorts.
  *
@@ -37,6 +37,7 @@
 #include <string.h>
 
 #define NKVO_BF16 0
+#define NKVO_F16 2
 #define NKVO_F32 1
 
 #define NKVO_GATE_SURPRISE 0
@@ -79,6 +80,15 @@ void nkvo_default_params(nkvo_params* p) {
 static double widen(const void* base, int dtype, int64_t index) {
     if (dtype == NKVO_F32) {
         return (double)((const float*)base)[index];
+    } else if (dtype == NKVO_F16) {
+        /* IEEE binary16: 1 sign, 5 exponent (bias 15), 10 fraction bits; every value is exact in double */
+        uint16_t h = ((const uint16_t*)base)[index];
+        int sign = h >> 15, e = (h >> 10) & 31, f = h & 1023;
+        double v;
+        if (e == 0) v = ldexp((double)f, -24);
+        else if (e == 31) v = f ? NAN : INFINITY;
+        else v = ldexp((double)(1024 + f), e - 25);
+        return sign ? -v : v;
     } else {
         uint32_t bits = ((uint32_t)((const uint16_t*)base)[index]) << 16;
         float f;

@@ -88,12 +88,12 @@ Layout make_layout(int64_t units, int64_t N, int64_t d, int64_t nb) {
 
 int check_tensor(const nkv_tensor* t) {
     if (!t || !t->ptr) return NKV_ERR_INVALID_ARG;
-    if (t->dtype != NKV_BF16 && t->dtype != NKV_F32) return NKV_ERR_UNSUPPORTED;
+    if (t->dtype != NKV_BF16 && t->dtype != NKV_F32 && t->dtype != NKV_F16) return NKV_ERR_UNSUPPORTED;
     if (t->d != 64 && t->d != 128) return NKV_ERR_UNSUPPORTED;
     if (t->G < 1 || t->H < 1 || t->N < 1) return NKV_ERR_INVALID_ARG;
     if (t->N > (int64_t)1 << 24 || t->G * t->H > (int64_t)1 << 24) return NKV_ERR_UNSUPPORTED;
     if (t->stride_n != t->d) return NKV_ERR_UNSUPPORTED;
-    const int64_t eb = t->dtype == NKV_BF16 ? 2 : 4;
+    const int64_t eb = t->dtype == NKV_F32 ? 4 : 2;
     if (t->stride_h < t->N * t->d || t->stride_g < t->H * t->N * t->d) {
         // strides may be permuted (for instance heads outermost); only require non-overlap of rows
         if (t->stride_h < 1 || t->stride_g < 1) return NKV_ERR_INVALID_ARG;
@@ -438,7 +438,7 @@ int nkv_compact(nkv_handle* h, const nkv_tensor* K, const nkv_tensor* V, const i
     if ((rc = check_tensor(V))) return rc;
     if (V->G != K->G || V->H != K->H || V->N != K->N) return NKV_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
-    const int kb = K->dtype == NKV_BF16 ? 2 : 4, vb = V->dtype == NKV_BF16 ? 2 : 4;
+    const int kb = K->dtype == NKV_F32 ? 4 : 2, vb = V->dtype == NKV_F32 ? 4 : 2;
     if (mode == NKV_OUT_OF_PLACE) {
         if (!K_out || !V_out || ((uintptr_t)K_out) % 16 || ((uintptr_t)V_out) % 16) return NKV_ERR_INVALID_ARG;
         CU(launch_gather(view_of(K), kb, view_of(V), vb, (int)K->G, idx, head_offsets, idx_capacity, K_out, V_out,
@@ -476,7 +476,7 @@ int nkv_compress(nkv_handle* h, const nkv_tensor* K, const nkv_tensor* V, double
     if ((rc = check_ws(ws, ws_bytes, L.total))) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     const TensorView kv = view_of(K), vv = view_of(V);
-    const int kb = K->dtype == NKV_BF16 ? 2 : 4, vb = V->dtype == NKV_BF16 ? 2 : 4;
+    const int kb = K->dtype == NKV_F32 ? 4 : 2, vb = V->dtype == NKV_F32 ? 4 : 2;
     float* a_star = a_star_opt ? a_star_opt : at<float>(ws, L.a_star);
     int* status = at<int>(ws, L.status);
     const bool timing = h->timing != 0;
@@ -514,7 +514,7 @@ int nkv_host_staging_bytes(const nkv_handle* h, int64_t H, int64_t N, int64_t d,
     if (!(r >= 0.0 && r < 1.0)) return NKV_ERR_INVALID_ARG;
     const int64_t keep = keep_count(N, r);
     if (keep < 1) return NKV_ERR_INVALID_ARG;
-    const size_t eb = dtype == NKV_BF16 ? 2 : 4;
+    const size_t eb = dtype == NKV_F32 ? 4 : 2;
     const int64_t b = block_size(N, params);
     const size_t c = (size_t)groups_per_chunk;
     size_t slot = 0;
@@ -546,7 +546,7 @@ int nkv_compress_host(nkv_handle* h, const nkv_tensor* Kh, const nkv_tensor* Vh,
     if ((rc = check_ws(dev, dev_bytes, need))) return rc;
     const int64_t G = Kh->G, H = Kh->H, N = Kh->N, d = Kh->d;
     const int64_t keep = keep_count(N, r);
-    const size_t eb = Kh->dtype == NKV_BF16 ? 2 : 4;
+    const size_t eb = Kh->dtype == NKV_F32 ? 4 : 2;
     const int64_t b = block_size(N, params);
     const size_t c = (size_t)groups_per_chunk;
     const size_t slot_bytes = need / 2;

@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -48,7 +49,7 @@ __device__ __forceinline__ float ord_float(uint32_t k) {
     return __uint_as_float(b);
 }
 
-// 16-byte chunk -> fp32 values.  bf16: 8 values, fp32: 4 values.
+// 16-byte chunk -> fp32 values.  bf16 and fp16: 8 values, fp32: 4 values.
 template <typename T> struct Elem;
 template <> struct Elem<__nv_bfloat16> {
     static constexpr int kPerChunk = 8;
@@ -58,6 +59,19 @@ template <> struct Elem<__nv_bfloat16> {
         v[2] = __uint_as_float(q.y << 16); v[3] = __uint_as_float(q.y & 0xffff0000u);
         v[4] = __uint_as_float(q.z << 16); v[5] = __uint_as_float(q.z & 0xffff0000u);
         v[6] = __uint_as_float(q.w << 16); v[7] = __uint_as_float(q.w & 0xffff0000u);
+    }
+};
+template <> struct Elem<__half> {
+    static constexpr int kPerChunk = 8;
+    static constexpr int kBytes = 2;
+    __device__ __forceinline__ static void unpack(const uint4& q, float* v) {
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[j]));
+            v[2 * j] = f.x;
+            v[2 * j + 1] = f.y;
+        }
     }
 };
 template <> struct Elem<float> {

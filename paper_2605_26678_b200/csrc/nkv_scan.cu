@@ -365,6 +365,8 @@ cudaError_t configure_scan_kernels() {
     cudaError_t e;
     if ((e = set_scan_attr<__nv_bfloat16, 64>()) != cudaSuccess) return e;
     if ((e = set_scan_attr<__nv_bfloat16, 128>()) != cudaSuccess) return e;
+    if ((e = set_scan_attr<__half, 64>()) != cudaSuccess) return e;
+    if ((e = set_scan_attr<__half, 128>()) != cudaSuccess) return e;
     if ((e = set_scan_attr<float, 64>()) != cudaSuccess) return e;
     if ((e = set_scan_attr<float, 128>()) != cudaSuccess) return e;
     return cudaSuccess;
@@ -374,6 +376,8 @@ cudaError_t configure_scan_kernels() {
     do {                                                               \
         if ((dtype) == NKV_BF16 && (d) == 64) { CALL(__nv_bfloat16, 64); }  \
         else if ((dtype) == NKV_BF16 && (d) == 128) { CALL(__nv_bfloat16, 128); } \
+        else if ((dtype) == NKV_F16 && (d) == 64) { CALL(__half, 64); }  \
+        else if ((dtype) == NKV_F16 && (d) == 128) { CALL(__half, 128); } \
         else if ((dtype) == NKV_F32 && (d) == 64) { CALL(float, 64); }  \
         else if ((dtype) == NKV_F32 && (d) == 128) { CALL(float, 128); } \
         else return cudaErrorInvalidValue;                             \
@@ -423,6 +427,7 @@ cudaError_t launch_window_means(const TensorView& K, int dtype, int G, const Sco
                                 float* mu_c, cudaStream_t stream, int64_t* launches) {
     const unsigned grid = (unsigned)K.N * (unsigned)(G * K.H);
     if (dtype == NKV_BF16) window_means_kernel<__nv_bfloat16><<<grid, K.d, 0, stream>>>(K, sp, inv_norm, mu_c);
+    else if (dtype == NKV_F16) window_means_kernel<__half><<<grid, K.d, 0, stream>>>(K, sp, inv_norm, mu_c);
     else window_means_kernel<float><<<grid, K.d, 0, stream>>>(K, sp, inv_norm, mu_c);
     ++*launches;
     return cudaGetLastError();

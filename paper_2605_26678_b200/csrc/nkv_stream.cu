@@ -81,7 +81,7 @@ __device__ __forceinline__ float hsum2(F2 x) {
     return a + b;
 }
 
-// 16-byte chunk -> packed pairs.  bf16: 4 pairs (8 values), fp32: 2 pairs (4 values).
+// 16-byte chunk -> packed pairs.  bf16 and fp16: 4 pairs (8 values), fp32: 2 pairs (4 values).
 template <typename T> struct Pairs;
 template <> struct Pairs<__nv_bfloat16> {
     static constexpr int kPairs = 4;
@@ -90,6 +90,17 @@ template <> struct Pairs<__nv_bfloat16> {
         p[1] = pack2(__uint_as_float(q.y << 16), __uint_as_float(q.y & 0xffff0000u));
         p[2] = pack2(__uint_as_float(q.z << 16), __uint_as_float(q.z & 0xffff0000u));
         p[3] = pack2(__uint_as_float(q.w << 16), __uint_as_float(q.w & 0xffff0000u));
+    }
+};
+template <> struct Pairs<__half> {
+    static constexpr int kPairs = 4;
+    __device__ __forceinline__ static void unpack(const uint4& q, F2* p) {
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[j]));
+            p[j] = pack2(f.x, f.y);
+        }
     }
 };
 template <> struct Pairs<float> {
@@ -581,6 +592,8 @@ __global__ void stream_init_kernel(int units, uint32_t* mm, float* block_sums, l
 template <typename T, int D> struct Tiles;
 template <> struct Tiles<__nv_bfloat16, 128> { static constexpr int A = 256, B = 256; };
 template <> struct Tiles<__nv_bfloat16, 64> { static constexpr int A = 512, B = 512; };
+template <> struct Tiles<__half, 128> { static constexpr int A = 256, B = 256; };
+template <> struct Tiles<__half, 64> { static constexpr int A = 512, B = 512; };
 template <> struct Tiles<float, 128> { static constexpr int A = 128, B = 128; };
 template <> struct Tiles<float, 64> { static constexpr int A = 256, B = 256; };
 
@@ -598,6 +611,8 @@ cudaError_t configure_stream_kernels() {
     cudaError_t e;
     if ((e = set_attrs<__nv_bfloat16, 64>()) != cudaSuccess) return e;
     if ((e = set_attrs<__nv_bfloat16, 128>()) != cudaSuccess) return e;
+    if ((e = set_attrs<__half, 64>()) != cudaSuccess) return e;
+    if ((e = set_attrs<__half, 128>()) != cudaSuccess) return e;
     if ((e = set_attrs<float, 64>()) != cudaSuccess) return e;
     if ((e = set_attrs<float, 128>()) != cudaSuccess) return e;
     return cudaSuccess;
@@ -609,6 +624,8 @@ bool stream_path_supported(const ScoreParams& sp) { return sp.block % kSeg == 0;
     do {                                                                     \
         if ((dtype) == NKV_BF16 && (d) == 64) { CALL(__nv_bfloat16, 64); }   \
         else if ((dtype) == NKV_BF16 && (d) == 128) { CALL(__nv_bfloat16, 128); } \
+        else if ((dtype) == NKV_F16 && (d) == 64) { CALL(__half, 64); }      \
+        else if ((dtype) == NKV_F16 && (d) == 128) { CALL(__half, 128); }    \
         else if ((dtype) == NKV_F32 && (d) == 64) { CALL(float, 64); }       \
         else if ((dtype) == NKV_F32 && (d) == 128) { CALL(float, 128); }     \
         else return cudaErrorInvalidValue;                                   \

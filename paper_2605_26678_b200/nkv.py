@@ -23,7 +23,7 @@ LIB_PATH = os.path.join(_PKG, "libnkv.so")
 NKV_OK = 0
 NKV_ERR_INVALID_ARG, NKV_ERR_UNSUPPORTED, NKV_ERR_WORKSPACE = 1, 2, 3
 NKV_ERR_CUDA, NKV_ERR_TIMEOUT, NKV_ERR_DEVICE_CHECK = 4, 5, 6
-NKV_BF16, NKV_F32 = 0, 1
+NKV_BF16, NKV_F32, NKV_F16 = 0, 1, 2
 NKV_GATE_SURPRISE, NKV_GATE_AVERAGE, NKV_GATE_MAX = 0, 1, 2
 NKV_OUT_OF_PLACE, NKV_IN_PLACE = 0, 1
 NKV_HEAD_STATS = 16
@@ -164,6 +164,8 @@ def _dtype_code(t: torch.Tensor) -> int:
         return NKV_BF16
     if t.dtype == torch.float32:
         return NKV_F32
+    if t.dtype == torch.float16:
+        return NKV_F16
     raise NkvError(NKV_ERR_UNSUPPORTED, "dtype %s" % t.dtype)
 
 

@@ -50,9 +50,9 @@ def assert_close(got, want, what, tol=TOL):
 
 
 def raw_rows(x: torch.Tensor) -> np.ndarray:
-    """bf16 -> uint16 view, fp32 -> float32, on host."""
+    """bf16 / fp16 -> uint16 view, fp32 -> float32, on host."""
     x = x.detach().cpu().contiguous()
-    if x.dtype == torch.bfloat16:
+    if x.dtype in (torch.bfloat16, torch.float16):
         return x.view(torch.int16).numpy().view(np.uint16)
     return x.numpy()
 

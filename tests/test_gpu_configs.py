@@ -1,4 +1,5 @@
-"""The five benchmark configurations at full size, in the launch configuration the bench times.
+"""The five benchmark configurations and the other model shapes at full size, in the launch configuration the
+bench times.
 
 The fused call runs on the whole synthetic cache; the oracle recomputes sampled layer groups
 (all of them for the small configuration) and everything about those groups is compared:
@@ -80,9 +81,13 @@ def _check_groups(cfg, K, V, groups, ratios, params):
     ("cfg3_llama32_1b_32k", [0, 15]),
     ("cfg4_qwen3_4b_32k_b4", [0, 143]),
     ("cfg5_qwen3_8b_128k", [20]),
+    ("shape_qwen3_0p6b_16k", [3]),
+    ("shape_qwen3_8b_16k_fp16", [0, 35]),
+    ("shape_qwen3_32b_8k", [0, 63]),
+    ("shape_llama32_3b_32k", [27]),
 ])
 def test_benchmark_config_matches_oracle(name, groups):
-    cfg = wl.CONFIGS[name]
+    cfg = wl.ALL_CONFIGS[name]
     K, V = wl.make_cache(cfg, DEV)
     params = nkv.nkv_default_params()
     reports = _check_groups(cfg, K, V, groups, cfg.ratios, params)

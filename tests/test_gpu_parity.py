@@ -28,7 +28,8 @@ def _cache(N, d, dtype, H=2, layers=1, seed=11, seg=(32, 96)):
 
 
 SHAPES = [(1, 64, "fp32"), (3, 64, "bf16"), (63, 128, "bf16"), (64, 64, "fp32"), (65, 128, "fp32"),
-          (200, 64, "bf16"), (257, 128, "bf16"), (1000, 128, "fp32"), (4133, 64, "bf16"), (6000, 128, "bf16")]
+          (200, 64, "bf16"), (257, 128, "bf16"), (1000, 128, "fp32"), (4133, 64, "bf16"), (6000, 128, "bf16"),
+          (300, 64, "fp16"), (4133, 128, "fp16")]
 
 
 @pytest.mark.parametrize("N,d,dtype", SHAPES)
@@ -70,7 +71,8 @@ def test_scores_match_oracle(N, d, dtype):
 KEY_SCAN_CASES = [("fma", 1, 64, "fp32"), ("fma", 63, 128, "bf16"), ("fma", 257, 128, "bf16"), ("fma", 1000, 128, "fp32"),
                   ("fma", 4133, 64, "bf16"), ("fma", 6000, 128, "bf16"), ("tensor", 100, 128, "bf16"),
                   ("tensor", 257, 128, "bf16"), ("tensor", 2500, 128, "bf16"), ("tensor", 4352, 128, "bf16"),
-                  ("tensor", 8200, 128, "bf16"), ("tensor", 4133, 64, "bf16"), ("auto", 3000, 128, "bf16")]
+                  ("tensor", 8200, 128, "bf16"), ("tensor", 4133, 64, "bf16"), ("auto", 3000, 128, "bf16"),
+                  ("auto", 2500, 128, "fp16"), ("tensor", 777, 64, "fp16")]
 
 
 @pytest.mark.parametrize("mode,N,d,dtype", KEY_SCAN_CASES)
@@ -185,7 +187,7 @@ def test_safeguard_one_gives_uniform_budgets():
 @pytest.mark.parametrize("d,dv,dtype,mode", [(128, 128, "bf16", "out"), (64, 64, "fp32", "out"),
                                              (128, 128, "fp32", "in"), (64, 64, "bf16", "in"),
                                              (128, 64, "bf16", "out"), (64, 128, "fp32", "out"),
-                                             (128, 64, "bf16", "in")])
+                                             (128, 64, "bf16", "in"), (128, 128, "fp16", "out")])
 def test_compaction_copies_rows_verbatim(d, dv, dtype, mode):
     K, V = _cache(900, d, dtype, H=3, layers=2)
     if dv != d:   # values of another width (the paper's V in R^{N x d_v}): same rows, other row length
@@ -215,7 +217,8 @@ def test_compaction_copies_rows_verbatim(d, dv, dtype, mode):
 
 @pytest.mark.parametrize("N,d,dtype,H,layers,r", [
     (5, 64, "fp32", 2, 1, 0.5), (300, 64, "bf16", 4, 2, 0.75), (1000, 128, "fp32", 8, 1, 0.5),
-    (2500, 128, "bf16", 8, 2, 0.95), (4133, 64, "bf16", 3, 1, 0.0), (777, 128, "bf16", 1, 3, 0.9)])
+    (2500, 128, "bf16", 8, 2, 0.95), (4133, 64, "bf16", 3, 1, 0.0), (777, 128, "bf16", 1, 3, 0.9),
+    (3000, 128, "fp16", 4, 2, 0.85), (900, 64, "fp16", 2, 1, 0.25)])
 def test_fused_compress_end_to_end(N, d, dtype, H, layers, r):
     K, V = _cache(N, d, dtype, H=H, layers=layers)
     p = nkv.nkv_default_params()
@@ -326,7 +329,7 @@ def test_argument_errors_are_reported_not_thrown():
         nkv.nkv_compress(K, V, 0.5, ws=torch.empty(1024, dtype=torch.uint8, device=DEV))
     assert e.value.status == nkv.NKV_ERR_WORKSPACE
     with pytest.raises(nkv.NkvError) as e:
-        nkv.nkv_compress(K.half(), V.half(), 0.5)
+        nkv.nkv_compress(K.double(), V.double(), 0.5)
     assert e.value.status == nkv.NKV_ERR_UNSUPPORTED
 
 
