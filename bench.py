@@ -36,18 +36,46 @@ METRIC = "keys_compressed_per_sec"
 UNIT = "keys/s"
 DEFAULT_WORKLOAD = "cfg4_qwen3_4b_32k_b4"
 DEFAULT_RATIO = 0.75
-# DRAM bytes per key (dram__bytes_read.sum + dram__bytes_write.sum of one launch / keys of the launch)
-# from the ncu capture summarised in profiles/ (cfg2, bf16, d = 128; traffic grows with the number of
-# keys).  Only kernels unchanged since their capture are listed.
-NCU_DRAM_BYTES_PER_KEY = {("anchors", "bf16", 128): (604.288256e6 + 25.738752e6) / 2359296}
+# DRAM bytes per key of each kernel (dram__bytes_read.sum + dram__bytes_write.sum of one launch / keys of the
+# launch) come from the ncu capture summarised in profiles/; the file lists kernel, storage, head_dim, bytes
+# per key and the digest of the kernel's source file at capture time.  A kernel whose source has changed since
+# reports no traffic.
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_bytes_per_key.txt")
+STAGE_KERNEL = {"anchors": ("gram_pass_kernel", "nkv_gram.cu"), "score": ("anchor_dots_kernel", "nkv_dots.cu"),
+                "compact": ("gather_kernel", "nkv_compact.cu"), "head": ("scale_stats_kernel", "nkv_select.cu"),
+                "budget": ("budget_kernel", "nkv_select.cu"), "select": ("select_kernel", "nkv_select.cu")}
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+
+
+def source_digest(name):
+    import hashlib
+    path = os.path.join(ROOT, "paper_2605_26678_b200", "csrc", name)
+    try:
+        with open(path, "rb") as f:
+            return hashlib.sha256(f.read()).hexdigest()[:16]
+    except OSError:
+        return None
+
+
+def measured_traffic_per_key(kernel, source, storage, head_dim):
+    """Bytes per key from the tracked ncu summary, or None if absent or taken on another version of the kernel."""
+    try:
+        with open(TRAFFIC_FILE) as f:
+            for line in f:
+                parts = line.split()
+                if len(parts) >= 5 and not line.startswith("#") and parts[0] == kernel and parts[1] == storage \
+                        and int(parts[2]) == head_dim:
+                    return float(parts[3]) if parts[4] == source_digest(source) else None
+    except OSError:
+        pass
+    return None
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="nkv", choices=["nkv", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(wl.ALL_CONFIGS))
@@ -55,6 +83,7 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-config-table", action="store_true", help="skip the per-configuration table")
     ap.add_argument("--key-passes", default="auto", choices=["auto", "fma", "tensor"],
                     help="kernels of the two key passes (library default: auto)")
     return ap.parse_args()
@@ -146,6 +175,17 @@ def whole_job_throughput(ms_local, steps, keys_per_rank, world, dist=None, devic
     return keys_per_rank * world / (ms_per_step * 1e-3), ms_per_step
 
 
+def bench_config(cfg, r, key_passes):
+    """The `config` object of the JSON line (the same for both arms)."""
+    return {"workload": "%s r=%.2f" % (cfg.name, r), "groups": cfg.groups, "kv_heads": cfg.kv_heads,
+            "seq_len": cfg.seq_len, "head_dim": cfg.head_dim, "storage": cfg.dtype,
+            "keys_per_step_per_gpu": cfg.keys, "kv_bytes_per_gpu": cfg.kv_bytes(),
+            "l2": "inputs (%.1f GB) are far larger than the 126 MB L2; no flush needed" % (
+                cfg.kv_bytes() / 1e9) if cfg.kv_bytes() > 1e9 else "inputs fit L2: warm-cache number",
+            "key_passes": key_passes,
+            "parallelism": "independent sequences per GPU (replicas), no collective"}
+
+
 def algorithmic_bytes(cfg, r):
     """Bytes the method must move through HBM for one step (per GPU)."""
     from paper_2605_26678_b200 import nkv
@@ -166,15 +206,17 @@ def algorithmic_bytes(cfg, r):
 # ----------------------------------------------------------------------------------------------
 # CPU oracle legs
 # ----------------------------------------------------------------------------------------------
-def oracle_throughput(cfg, r, groups_kv, threads):
+def oracle_throughput(cfg, r, groups_kv, threads, keep=None):
     """Times the oracle over the given [(K[H,N,d], V[H,N,d])] host groups with `threads` workers."""
     import oracle
     oracle.lib()
     t0 = time.perf_counter()
     with ThreadPoolExecutor(max_workers=threads) as ex:
-        list(ex.map(lambda kv: oracle.compress_group(kv[0], kv[1], r), groups_kv))
+        results = list(ex.map(lambda kv: oracle.compress_group(kv[0], kv[1], r), groups_kv))
     dt = time.perf_counter() - t0
     keys = len(groups_kv) * cfg.kv_heads * cfg.seq_len
+    if keep is not None:
+        keep.extend(results)
     return keys / dt, dt
 
 
@@ -208,7 +250,7 @@ def run_reference(args, cfg, r):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / max(1, args.steps),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "%s r=%.2f" % (cfg.name, r), "note": "CPU oracle on a bounded sample"},
+        "config": bench_config(cfg, r, args.key_passes),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": min(threads, len(groups)), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -278,7 +320,7 @@ def run_nkv(args, cfg, r):
     # ---- per-stage device time (events recorded on the launching stream inside the library) --
     nkv.nkv_set_timing(True, h)
     stage_ms = [[] for _ in range(nkv.NKV_NUM_STAGES)]
-    for _ in range(args.steps):
+    for _ in range(min(args.steps, 20)):
         step()
         for i, v in enumerate(nkv.nkv_get_stage_ms(h)):
             stage_ms[i].append(v)
@@ -288,15 +330,16 @@ def run_nkv(args, cfg, r):
     peak, peak_src = measured_peak()
     dominant = max(stage_avg, key=stage_avg.get)
     dom_gbs = stage_bytes[dominant] / (stage_avg[dominant] * 1e-3) / 1e9
+    kernel_name, kernel_src = STAGE_KERNEL[dominant]
+    per_key = measured_traffic_per_key(kernel_name, kernel_src, cfg.dtype, cfg.head_dim)
     roofline = {
-        "bound": "hbm", "kernel": dominant, "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
+        "bound": "hbm", "kernel": kernel_name, "stage": dominant, "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
         "frac": dom_gbs / peak,
-        "traffic": (NCU_DRAM_BYTES_PER_KEY[(dominant, cfg.dtype, cfg.head_dim)] * cfg.keys
-                    if (dominant, cfg.dtype, cfg.head_dim) in NCU_DRAM_BYTES_PER_KEY else None),
+        "traffic": per_key * cfg.keys if per_key is not None else None,
         "peak_source": peak_src,
         "algorithmic_bytes_per_launch": stage_bytes[dominant], "ms_per_launch": stage_avg[dominant],
         "stages_ms": stage_avg,
-        "stages_gbs": {s: stage_bytes[s] / (stage_avg[s] * 1e-3) / 1e9 for s in stage_avg if stage_avg[s] > 0},
+        "stages_gbs": {s: stage_bytes[s] / (stage_avg[s] * 1e-3) / 1e9 for s in stage_avg if stage_avg[s] > 1e-3},
     }
     pipe_gbs = bytes_min / (ms_per_step * 1e-3) / 1e9
     pipeline = {
@@ -317,10 +360,11 @@ def run_nkv(args, cfg, r):
         cores = os.cpu_count() or 1
         threads = min(cores, 32)
         done_groups, spent, g0 = 0, 0.0, 0
+        oracle_groups = []   # the oracle's results for groups 0, 1, ...: reused for the near-tie count
         while g0 < cfg.groups and spent < 12.0:
             wave = list(range(g0, min(cfg.groups, g0 + threads)))
             data = [(K[g].cpu(), V[g].cpu()) for g in wave]
-            _, dt = oracle_throughput(cfg, r, data, threads)
+            _, dt = oracle_throughput(cfg, r, data, threads, keep=oracle_groups if g0 == 0 else None)
             spent += dt
             done_groups += len(wave)
             g0 += len(wave)
@@ -329,24 +373,124 @@ def run_nkv(args, cfg, r):
                "sample": "%d of %d layer groups (%d keys) in %.1f s, %d worker threads" % (
                    done_groups, cfg.groups, done_groups * cfg.kv_heads * cfg.seq_len, spent, threads)}
 
+    # ---- near-tie swaps: the timed call's retained sets against the oracle's on the groups it just did ----
+    swaps = None
+    if cpu is not None and oracle_groups:
+        swaps = near_tie_swaps(K, V, r, params, ws, h, oracle_groups)
+
+    # ---- the other configurations (one GPU, rank 0 only; the headline line above is unaffected) ----
+    table = None
+    if rank == 0 and world == 1 and not args.no_config_table:
+        del K, V, out, ws
+        torch.cuda.empty_cache()
+        table = config_table(args, cfg, r, ms_per_step, h, peak)
+
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": "%s r=%.2f" % (cfg.name, r), "groups": cfg.groups, "kv_heads": cfg.kv_heads,
-                       "seq_len": cfg.seq_len, "head_dim": cfg.head_dim, "storage": cfg.dtype,
-                       "keys_per_step_per_gpu": cfg.keys, "kv_bytes_per_gpu": cfg.kv_bytes(),
-                       "l2": "inputs (%.1f GB) are far larger than the 126 MB L2; no flush needed" % (
-                           cfg.kv_bytes() / 1e9) if cfg.kv_bytes() > 1e9 else "inputs fit L2: warm-cache number",
-                       "key_passes": args.key_passes,
-                       "parallelism": "independent sequences per GPU (replicas), no collective"},
+            "config": bench_config(cfg, r, args.key_passes),
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "pipeline": pipeline,
-            "cpu_baseline": cpu,
+            "cpu_baseline": cpu, "near_tie_swaps": swaps, "configs": table,
         }
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def near_tie_swaps(K, V, r, params, ws, h, oracle_groups):
+    """Retained sets of the CUDA path against the oracle's on the first groups of the workload: heads whose
+    sets differ, tokens that changed sides, and how far (in score) the farthest of them is from the threshold
+    it crossed.  The oracle results are the ones the CPU baseline leg just produced."""
+    import numpy as np
+    from paper_2605_26678_b200 import nkv
+    res = nkv.nkv_compress(K, V, r, params, ws=ws, want_a_star=True, h=h)
+    torch.cuda.synchronize()
+    heads = with_swaps = tokens = 0
+    worst_score = worst_gap = 0.0
+    for g, ref in enumerate(oracle_groups):
+        a_gpu = res.a_star[g].cpu().numpy()
+        idx = res.idx[g].cpu().numpy()
+        offs = res.head_offsets[g].cpu().numpy()
+        fin = np.isfinite(ref.a_star)
+        worst_score = max(worst_score, float(np.abs(a_gpu[fin] - ref.a_star[fin]).max()))
+        for hd in range(K.shape[1]):
+            heads += 1
+            want = set(ref.sel.idx[ref.sel.offsets[hd]:ref.sel.offsets[hd + 1]].tolist())
+            got = set(idx[offs[hd]:offs[hd + 1]].tolist())
+            diff = want ^ got
+            if not diff:
+                continue
+            with_swaps += 1
+            tokens += len(diff)
+            thr = float(ref.a_star[hd, sorted(want)].min()) if want else 0.0
+            worst_gap = max(worst_gap, max(abs(float(ref.a_star[hd, i]) - thr) for i in diff))
+    return {"groups_checked": len(oracle_groups), "heads_checked": heads, "heads_with_swaps": with_swaps,
+            "swapped_tokens": tokens, "max_score_difference": worst_score,
+            "max_distance_of_a_swapped_token_from_its_heads_threshold": worst_gap}
+
+
+def time_steps(step, steps, flush=None):
+    """Milliseconds per step: back to back (flush None), or each step timed alone after `flush()`."""
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    if flush is None:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+    total = 0.0
+    for _ in range(steps):
+        flush()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        step()
+        e1.record()
+        torch.cuda.synchronize()
+        total += e0.elapsed_time(e1)
+    return total / steps
+
+
+def config_table(args, head_cfg, head_r, head_ms, h, peak):
+    """ms, keys/s and pipeline fraction of every benchmark configuration (and of the other ratios of the
+    headline one).  Caches that fit L2 are timed twice: warm (back to back) and cold (a buffer larger than L2
+    is overwritten before every step)."""
+    from paper_2605_26678_b200 import nkv
+    dev = torch.device("cuda", torch.cuda.current_device())
+    params = nkv.nkv_default_params()
+    flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    rows = {}
+    for name, cfg in wl.CONFIGS.items():
+        K, V = wl.make_cache(cfg, dev, groups_per_call=4)
+        ws = nkv.alloc_workspace(K, params)
+        for r in cfg.ratios:
+            if name == head_cfg.name and r == head_r:
+                ms = head_ms
+                cold = None
+            else:
+                out = nkv.alloc_outputs(K, V, r)
+                step = lambda: nkv.nkv_compress(K, V, r, params, out=out, ws=ws, h=h)
+                small = cfg.kv_bytes() < (4 << 30)
+                ms = time_steps(step, 50 if small else 10)
+                cold = time_steps(step, 20, flush=lambda: flush_buf.fill_(1)) if small else None
+                del out
+            _, bytes_min = algorithmic_bytes(cfg, r)
+            row = {"ms_per_step": ms, "keys_per_s": cfg.keys / (ms * 1e-3),
+                   "pipeline_frac_of_measured": bytes_min / (ms * 1e-3) / 1e9 / peak,
+                   "ms_per_sequence": ms / cfg.batch}
+            if cold is not None:
+                row["l2"] = "warm (back to back); cold = every step after a 512 MB overwrite"
+                row["ms_per_step_cold"] = cold
+                row["pipeline_frac_of_measured_cold"] = bytes_min / (cold * 1e-3) / 1e9 / peak
+            rows["%s r=%.2f" % (name, r)] = row
+        del K, V, ws
+        torch.cuda.empty_cache()
+    return rows
 
 
 def run_e2e(args, cfg, r, K, V, h, params, dist, dev, world):
