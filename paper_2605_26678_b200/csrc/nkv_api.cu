@@ -60,10 +60,10 @@ int64_t keep_count(int64_t N, double r) { return (int64_t)floor((1.0 - r) * (dou
 
 // Workspace carving shared by every entry point.
 struct Layout {
-    size_t status, inv_norm, mu_s, mu_e, inv_s, inv_e, mm, a_raw, a_star, thr, hstat, total;
+    size_t status, inv_norm, mu_s, mu_e, inv_s, inv_e, mm, a_raw, a_star, thr, hstat, bscr, total;
 };
 
-Layout make_layout(int64_t units, int64_t N, int64_t d, int64_t nb) {
+Layout make_layout(int64_t G, int64_t units, int64_t N, int64_t d, int64_t nb) {
     Layout L;
     size_t o = 0;
     auto take = [&](size_t bytes) {
@@ -82,6 +82,7 @@ Layout make_layout(int64_t units, int64_t N, int64_t d, int64_t nb) {
     L.a_star = take((size_t)units * N * 4);
     L.thr = take((size_t)units * 2 * 4);
     L.hstat = take(head_stat_bytes(units));
+    L.bscr = take(budget_scratch_bytes(G, units / G));   // the heads per group divide the units
     L.total = o;
     return L;
 }
@@ -344,7 +345,7 @@ int nkv_workspace_bytes(const nkv_handle* h, int64_t G, int64_t H, int64_t N, in
     (void)dtype;
     if (!h || !out_bytes || G < 1 || H < 1 || N < 1 || d < 1 || !params_ok(params)) return NKV_ERR_INVALID_ARG;
     const int64_t b = block_size(N, params);
-    *out_bytes = make_layout(G * H, N, d, (N + b - 1) / b).total;
+    *out_bytes = make_layout(G, G * H, N, d, (N + b - 1) / b).total;
     return NKV_OK;
 }
 
@@ -375,7 +376,7 @@ int nkv_score(nkv_handle* h, const nkv_tensor* K, const float* mu_s, const float
     ScoreParams sp;
     if ((rc = resolve_params(params, K->N, &sp))) return rc;
     const int units = (int)(K->G * K->H);
-    const Layout L = make_layout(units, K->N, K->d, sp.nblocks);
+    const Layout L = make_layout(K->G, units, K->N, K->d, sp.nblocks);
     if ((rc = check_ws(ws, ws_bytes, L.total))) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     const TensorView kv = view_of(K);
@@ -403,8 +404,10 @@ int nkv_budget(nkv_handle* h, const float* a_star, int64_t G, int64_t H, int64_t
     if (rc) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     CU(cudaMemsetAsync(ws, 0, kStatusWords * sizeof(int), st));
+    const size_t scr_off = thr_off + align_up((size_t)G * H * 8);
+    void* scratch = ws_bytes >= scr_off + budget_scratch_bytes(G, H) ? at<unsigned char>(ws, scr_off) : nullptr;
     CU(launch_budget((int)G, (int)H, (int)N, (int)k, (int)n_safe, a_star, budgets, at<uint32_t>(ws, thr_off),
-                     at<int>(ws, 0), st, &h->launches));
+                     at<int>(ws, 0), scratch, st, &h->launches));
     return NKV_OK;
 }
 
@@ -472,7 +475,7 @@ int nkv_compress(nkv_handle* h, const nkv_tensor* K, const nkv_tensor* V, double
     const int64_t n_safe = nkv_safeguard_count(K->N, r, params);
     const int G = (int)K->G, H = (int)K->H, N = (int)K->N, d = (int)K->d;
     const int units = G * H;
-    const Layout L = make_layout(units, N, d, sp.nblocks);
+    const Layout L = make_layout(G, units, N, d, sp.nblocks);
     if ((rc = check_ws(ws, ws_bytes, L.total))) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     const TensorView kv = view_of(K), vv = view_of(V);
@@ -494,7 +497,8 @@ int nkv_compress(nkv_handle* h, const nkv_tensor* K, const nkv_tensor* V, double
     CU(launch_head_scores(units, N, sp, at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), a_star, nullptr,
                           at<float>(ws, L.hstat), status, st, &h->launches));
     CU(mark());
-    CU(launch_budget(G, H, N, (int)keep, (int)n_safe, a_star, budgets, at<uint32_t>(ws, L.thr), status, st,
+    CU(launch_budget(G, H, N, (int)keep, (int)n_safe, a_star, budgets, at<uint32_t>(ws, L.thr), status,
+                     at<unsigned char>(ws, L.bscr), st,
                      &h->launches));
     CU(mark());
     CU(launch_select(G, H, N, (int64_t)H * keep, a_star, budgets, at<uint32_t>(ws, L.thr), idx, head_offsets, status,
@@ -523,7 +527,7 @@ int nkv_host_staging_bytes(const nkv_handle* h, int64_t H, int64_t N, int64_t d,
     slot += align_up(c * H * keep * 4);              // idx
     slot += align_up(c * (H + 1) * 4);               // head_offsets
     slot += align_up(c * H * 4);                     // budgets
-    slot += make_layout(c * H, N, d, (N + b - 1) / b).total;
+    slot += make_layout(c, c * H, N, d, (N + b - 1) / b).total;
     *out_bytes = 2 * slot;
     return NKV_OK;
 }
@@ -553,7 +557,7 @@ int nkv_compress_host(nkv_handle* h, const nkv_tensor* Kh, const nkv_tensor* Vh,
     const size_t kv_bytes = align_up(c * H * N * d * eb), out_bytes = align_up(c * H * keep * d * eb);
     const size_t idx_bytes = align_up(c * H * keep * 4), off_bytes = align_up(c * (H + 1) * 4),
                  bud_bytes = align_up(c * H * 4);
-    const size_t ws_need = make_layout(c * H, N, d, (N + b - 1) / b).total;
+    const size_t ws_need = make_layout(c, c * H, N, d, (N + b - 1) / b).total;
 
     int result = NKV_OK;
     int chunk_index = 0;
@@ -653,7 +657,7 @@ int nkv_key_scan(nkv_handle* h, const nkv_tensor* K, const nkv_params* params, f
     ScoreParams sp;
     if ((rc = resolve_params(params, K->N, &sp))) return rc;
     const int G = (int)K->G, N = (int)K->N, d = (int)K->d, units = (int)(K->G * K->H);
-    const Layout L = make_layout(units, N, d, sp.nblocks);
+    const Layout L = make_layout(G, units, N, d, sp.nblocks);
     if ((rc = check_ws(ws, ws_bytes, L.total))) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     CU(cudaMemsetAsync(at<int>(ws, L.status), 0, kStatusWords * sizeof(int), st));

@@ -151,8 +151,10 @@ size_t head_stat_bytes(int64_t units);   // scratch of launch_head_scores (`hsta
 cudaError_t launch_head_scores(int units, int N, const ScoreParams& sp, const float* a_raw,
                                const uint32_t* minmax_keys, float* a_star, float* head_stats_opt, float* hstat,
                                int* status, cudaStream_t stream, int64_t* launches);
+size_t budget_scratch_bytes(int64_t G, int64_t H);   // scratch of the parallel form of launch_budget
 cudaError_t launch_budget(int G, int H, int N, int keep, int n_safe, const float* a_star, int32_t* budgets,
-                          uint32_t* sel_thresholds, int* status, cudaStream_t stream, int64_t* launches);
+                          uint32_t* sel_thresholds, int* status, void* scratch_or_null, cudaStream_t stream,
+                          int64_t* launches);
 cudaError_t launch_select(int G, int H, int N, int64_t idx_capacity, const float* a_star, const int32_t* budgets,
                           const uint32_t* sel_thresholds_or_null, int32_t* idx, int32_t* head_offsets, int* status,
                           cudaStream_t stream, int64_t* launches);

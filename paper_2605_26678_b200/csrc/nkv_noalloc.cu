@@ -64,7 +64,7 @@ extern "C" int nkv_budget_static(const float* a_star, int64_t G, int64_t H, int6
     int64_t launches = 0;
     unsigned char* base = reinterpret_cast<unsigned char*>(scratch);
     if (nkv::launch_budget((int)G, (int)H, (int)N, (int)keep, (int)n_safe, a_star, budgets,
-                           reinterpret_cast<uint32_t*>(base + kStatusBytes), reinterpret_cast<int*>(base), st,
+                           reinterpret_cast<uint32_t*>(base + kStatusBytes), reinterpret_cast<int*>(base), nullptr, st,
                            &launches) != cudaSuccess)
         return NKV_ERR_CUDA;
     return NKV_OK;

@@ -304,7 +304,10 @@ __device__ __forceinline__ float block_reduce_f(SelectShared& S, float v, int op
 // turns out wrong (rank outside the list, list overflow) the full-histogram path runs instead, so the
 // result is always exact.
 // ------------------------------------------------------------------------------------------
-constexpr int kSampleMin = 1024, kSampleMax = 32768;   // sample positions: n / 8, clamped
+constexpr int kSampleMin = 1024, kSampleMax = 32768;   // sample positions: n / 8 (n / 4 for long inputs), clamped
+// The bracket that one sample rank error of 4 sigma spans grows with n / positions: beyond 64k elements a
+// denser sample keeps it inside the candidate buffers.
+__device__ __forceinline__ int sample_positions(int n) { return min(max(n > 65536 ? n / 4 : n / 8, kSampleMin), kSampleMax); }
 constexpr int kCandSmall = 4096;                       // bracket capacity of the per-head kernels
 constexpr int kCandLarge = 12288;                      // ... of the per-group kernel (dynamic shared memory)
 
@@ -338,7 +341,7 @@ __device__ void block_select_bracket(SelectShared& S, BracketShared<CAP>& X, con
     bool use_bracket = n > kCandCap && n_eff > 0;
     if (use_bracket) {
         // 1. histogram of a strided sample (rejected elements are skipped)
-        const int positions = min(max(n / 8, kSampleMin), kSampleMax);
+        const int positions = sample_positions(n);
         for (int b = tid; b < kBins; b += nt) S.hist[b] = 0;
         __syncthreads();
         int mine = 0;
@@ -543,7 +546,7 @@ __device__ bool two_tail_sums(SelectShared& S, BracketShared<CAP>& X, const floa
     const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
     if (n <= CAP || 2 * m >= n) return false;
     // 1. histogram of a strided sample
-    const int positions = min(max(n / 8, kSampleMin), kSampleMax);
+    const int positions = sample_positions(n);
     for (int b = tid; b < kBins; b += nt) S.hist[b] = 0;
     __syncthreads();
     for (int i0 = 0; i0 < positions; i0 += 4 * nt) {   // four loads in flight per thread
@@ -672,7 +675,8 @@ constexpr int kStatThreads = 256;
 
 // scale_stats: one CTA per (head, task).  Tasks 0..2: the reliability gap of one scale (exact sums of
 // the m largest and m smallest values); task 3: min, max and sum of the surprise over the head.
-__global__ void __launch_bounds__(kStatThreads, 4) scale_stats_kernel(int N, ScoreParams sp, const float* __restrict__ a_raw,
+template <int kT>
+__global__ void __launch_bounds__(kT, kT == 256 ? 4 : 1) scale_stats_kernel(int N, ScoreParams sp, const float* __restrict__ a_raw,
                                                                    const uint32_t* __restrict__ mm,
                                                                    float* __restrict__ hstat, int* status) {
     __shared__ SelectShared S;
@@ -900,7 +904,8 @@ struct PoolSrc {       // all (head, token) pairs of a group whose key does not 
 // safeguard: one CTA per head.  The n_safe best tokens of each head are kept unconditionally:
 // thr[2u] = ordered key of the n_safe-th best score, thr[2u+1] = how many tokens tied at that key
 // belong to the safeguard.  (The group kernel below overwrites both words with the final threshold.)
-__global__ void __launch_bounds__(kStatThreads, 4) safeguard_kernel(int N, int n_safe, const float* __restrict__ a_star,
+template <int kT>
+__global__ void __launch_bounds__(kT, kT == 256 ? 4 : 1) safeguard_kernel(int N, int n_safe, const float* __restrict__ a_star,
                                                                  uint32_t* __restrict__ thr, int* status) {
     __shared__ SelectShared S;
     __shared__ BracketShared<kCandSmall> X;
@@ -924,7 +929,9 @@ __global__ void __launch_bounds__(kStatThreads, 4) safeguard_kernel(int N, int n
 __global__ void __launch_bounds__(kThreads) budget_kernel(int H, int N, int keep, int n_safe,
                                                           const float* __restrict__ a_star,
                                                           int32_t* __restrict__ budgets, uint32_t* __restrict__ thr,
-                                                          int* status) {
+                                                          int* status, const int* __restrict__ only_flagged) {
+    // after the parallel form: only the groups it left over
+    if (only_flagged && only_flagged[blockIdx.x * 4 + 3] == 0) return;
     __shared__ SelectShared S;
     extern __shared__ __align__(16) unsigned char budget_dyn[];
     BracketShared<kCandLarge>& X = *reinterpret_cast<BracketShared<kCandLarge>*>(budget_dyn);
@@ -1022,6 +1029,197 @@ __global__ void __launch_bounds__(kThreads) budget_kernel(int H, int N, int keep
             thr[((int64_t)g * H + h) * 2 + 1] = q;
         }
         if (total != H * keep || remaining != 0) set_status(status, NKV_ERR_DEVICE_CHECK, 201);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// budget, parallel form: the cross-head competition of a group as a histogram over all of its
+// heads, so that the streaming work is spread over many CTAs and only a small candidate list
+// is finished by one CTA per group.
+// ------------------------------------------------------------------------------------------
+constexpr int kBudgetCand = 8192;    // candidates per group (the scores that share the threshold's bin)
+constexpr int kBudgetChunk = 8192;   // scores per CTA of the two streaming steps
+constexpr int kBudgetMeta = 4;       // per group: threshold bin, rank wanted inside it, candidates, needs the one-CTA kernel
+
+// final scores lie in [0, 1] (sinks: +inf): 2048 value-linear bins, monotone in the score
+__device__ __forceinline__ int score_bin(float v) { return min(max(__float2int_rz(v * (float)kBins), 0), kBins - 1); }
+
+// step 1: per head, the histogram of its pool (scores at or below the head's safeguard threshold)
+__global__ void __launch_bounds__(256) budget_hist_kernel(int N, const float* __restrict__ a_star,
+                                                          const uint32_t* __restrict__ thr, int* __restrict__ bhist) {
+    __shared__ int hist[kBins];
+    const int u = blockIdx.y, j0 = blockIdx.x * kBudgetChunk, j1 = min(N, j0 + kBudgetChunk);
+    for (int b = threadIdx.x; b < kBins; b += blockDim.x) hist[b] = 0;
+    __syncthreads();
+    const uint32_t T = thr[(int64_t)u * 2];
+    const float* v = a_star + (int64_t)u * N;
+    for (int j = j0 + threadIdx.x; j < j1; j += blockDim.x) {
+        const float x = v[j];
+        if (ord_key(x) <= T) atomicAdd(&hist[score_bin(x)], 1);
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b < kBins; b += blockDim.x)
+        if (hist[b]) atomicAdd(&bhist[(int64_t)u * kBins + b], hist[b]);
+}
+
+// step 2: per group, the bin that holds the rank the competition stops at
+__global__ void __launch_bounds__(256) budget_find_kernel(int H, int keep, int n_safe, const uint32_t* __restrict__ thr,
+                                                          const int* __restrict__ bhist, int* __restrict__ bmeta) {
+    __shared__ SelectShared S;
+    const int g = blockIdx.x;
+    const int rest = H * keep - H * n_safe;
+    if (rest <= 0) {
+        if (threadIdx.x == 0) bmeta[g * kBudgetMeta] = -1;
+        return;
+    }
+    for (int b = threadIdx.x; b < kBins; b += blockDim.x) {
+        int c = 0;
+        for (int h = 0; h < H; ++h) {
+            const int64_t u = (int64_t)g * H + h;
+            c += bhist[u * kBins + b];
+            // of the scores tied at the safeguard threshold, thr[2u+1] belong to the safeguard, not to the pool
+            if (score_bin(ord_float(thr[u * 2])) == b) c -= (int)thr[u * 2 + 1];
+        }
+        S.hist[b] = c;
+    }
+    if (threadIdx.x == 0) {
+        S.bin = -1;
+        S.above = 0;
+    }
+    __syncthreads();
+    find_bin_desc(S, rest);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        bmeta[g * kBudgetMeta] = S.bin;                 // -1: fewer pool scores than slots (cannot happen: rest <= pool)
+        bmeta[g * kBudgetMeta + 1] = rest - S.above;    // rank wanted among the bin's scores, from the top
+    }
+}
+
+// step 3: the pool scores of that bin, with their heads, into the group's candidate list
+__global__ void __launch_bounds__(256) budget_collect_kernel(int H, int N, const float* __restrict__ a_star,
+                                                             const uint32_t* __restrict__ thr, int* __restrict__ bmeta,
+                                                             float* __restrict__ cand_v, unsigned char* __restrict__ cand_h) {
+    const int u = blockIdx.y, g = u / H, h = u - g * H;
+    const int bin = bmeta[g * kBudgetMeta];
+    if (bin < 0) return;
+    const int j0 = blockIdx.x * kBudgetChunk, j1 = min(N, j0 + kBudgetChunk);
+    const uint32_t T = thr[(int64_t)u * 2];
+    const float* v = a_star + (int64_t)u * N;
+    const int lane = threadIdx.x & 31;
+    for (int jb = j0; jb < j1; jb += blockDim.x) {
+        const int j = jb + threadIdx.x;
+        const float x = j < j1 ? v[j] : 0.f;
+        const bool mine = j < j1 && ord_key(x) <= T && score_bin(x) == bin;
+        const unsigned ballot = __ballot_sync(0xffffffffu, mine);
+        if (ballot) {
+            int base = 0;
+            if (lane == 0) base = atomicAdd(&bmeta[g * kBudgetMeta + 2], __popc(ballot));
+            base = __shfl_sync(0xffffffffu, base, 0);
+            const int pos = base + __popc(ballot & ((1u << lane) - 1u));
+            if (mine && pos < kBudgetCand) {
+                cand_v[(int64_t)g * kBudgetCand + pos] = x;
+                cand_h[(int64_t)g * kBudgetCand + pos] = (unsigned char)h;
+            }
+        }
+    }
+}
+
+// step 4: one CTA per group finishes exactly on the candidates and turns counts into budgets.  A group whose
+// candidate list overflowed (scores packed into one bin) is left to budget_kernel.
+__global__ void __launch_bounds__(kThreads) budget_finish_kernel(int H, int keep, int n_safe,
+                                                                 const int* __restrict__ bhist, int* __restrict__ bmeta,
+                                                                 const float* __restrict__ cand_v,
+                                                                 const unsigned char* __restrict__ cand_h,
+                                                                 int32_t* __restrict__ budgets, uint32_t* __restrict__ thr,
+                                                                 int* status) {
+    __shared__ SelectShared S;
+    extern __shared__ __align__(16) unsigned char finish_dyn[];
+    float* cv = reinterpret_cast<float*>(finish_dyn);
+    unsigned char* ch = finish_dyn + kBudgetCand * sizeof(float);
+    __shared__ uint32_t T[kMaxCorr];
+    __shared__ int corr[kMaxCorr], cnt_mid[kMaxCorr], cnt_eq[kMaxCorr];
+    const int g = blockIdx.x, tid = threadIdx.x;
+    const int bin = bmeta[g * kBudgetMeta], need = bmeta[g * kBudgetMeta + 1], nc = bmeta[g * kBudgetMeta + 2];
+    if (bin >= 0 && nc > kBudgetCand) {
+        if (tid == 0) bmeta[g * kBudgetMeta + 3] = 1;
+        return;
+    }
+    if (tid < H) {
+        T[tid] = thr[((int64_t)g * H + tid) * 2];
+        corr[tid] = (int)thr[((int64_t)g * H + tid) * 2 + 1];
+    }
+    if (tid == 0) S.ncorr = 0;
+    __syncthreads();
+    const int rest = H * keep - H * n_safe;
+    uint32_t tau = 0xffffffffu;
+    if (bin >= 0) {
+        for (int j = tid; j < nc; j += blockDim.x) {
+            cv[j] = cand_v[(int64_t)g * kBudgetCand + j];
+            ch[j] = cand_h[(int64_t)g * kBudgetCand + j];
+        }
+        if (tid == 0) {
+            // safeguard ties that sit among the candidates do not compete
+            int n = 0;
+            for (int h = 0; h < H; ++h)
+                if (corr[h] > 0 && score_bin(ord_float(T[h])) == bin) {
+                    S.corr_v[n] = ord_float(T[h]);
+                    S.corr_m[n] = corr[h];
+                    ++n;
+                }
+            S.ncorr = n;
+        }
+        __syncthreads();
+        SmemSrc src{cv};
+        block_select_desc(S, src, nc, need, (float)bin / (float)kBins, (float)kBins * (float)kBins, status);
+        tau = S.theta;
+        __syncthreads();
+    }
+    // per head: pool scores above tau (whole bins above the threshold's bin plus candidates) and equal to it
+    for (int h = 0; h < H; ++h) {
+        int mid = 0, eq = 0;
+        if (bin >= 0) {
+            const int* hh = bhist + ((int64_t)g * H + h) * kBins;
+            for (int b = bin + 1 + tid; b < kBins; b += blockDim.x) mid += hh[b];
+            for (int j = tid; j < nc; j += blockDim.x)
+                if (ch[j] == h) {
+                    const uint32_t key = ord_key(cv[j]);
+                    mid += key > tau;
+                    eq += key == tau;
+                }
+        }
+        mid = block_sum_int(S, mid);
+        __syncthreads();
+        eq = block_sum_int(S, eq);
+        if (tid == 0) {
+            cnt_mid[h] = mid;
+            cnt_eq[h] = eq;
+        }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        int taken_gt = 0;
+        for (int h = 0; h < H; ++h) taken_gt += cnt_mid[h] - (T[h] > tau ? corr[h] : 0);
+        int remaining = rest - taken_gt;
+        int total = 0;
+        for (int h = 0; h < H; ++h) {
+            const int pool_eq = cnt_eq[h] - (T[h] == tau ? corr[h] : 0);
+            const int t = max(0, min(pool_eq, remaining));
+            remaining -= t;
+            const int B = n_safe + cnt_mid[h] - (T[h] > tau ? corr[h] : 0) + t;
+            budgets[(int64_t)g * H + h] = B;
+            total += B;
+            uint32_t theta, q;
+            if (tau < T[h]) {
+                theta = tau;
+                q = (uint32_t)t;
+            } else {
+                theta = T[h];
+                q = (uint32_t)(corr[h] + t);
+            }
+            thr[((int64_t)g * H + h) * 2] = theta;
+            thr[((int64_t)g * H + h) * 2 + 1] = q;
+        }
+        if (total != H * keep || remaining != 0) set_status(status, NKV_ERR_DEVICE_CHECK, 202);
     }
 }
 
@@ -1162,7 +1360,9 @@ __global__ void __launch_bounds__(256) ranks_kernel(int N, const float* __restri
 cudaError_t launch_head_scores(int units, int N, const ScoreParams& sp, const float* a_raw,
                                const uint32_t* minmax_keys, float* a_star, float* head_stats_opt, float* hstat,
                                int* status, cudaStream_t stream, int64_t* launches) {
-    scale_stats_kernel<<<units * 4, kStatThreads, 0, stream>>>(N, sp, a_raw, minmax_keys, hstat, status);
+    // long heads: four times the threads per head (the per-head work is one CTA's)
+    if (N >= 65536) scale_stats_kernel<1024><<<units * 4, 1024, 0, stream>>>(N, sp, a_raw, minmax_keys, hstat, status);
+    else scale_stats_kernel<kStatThreads><<<units * 4, kStatThreads, 0, stream>>>(N, sp, a_raw, minmax_keys, hstat, status);
     ++*launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -1184,21 +1384,50 @@ cudaError_t configure_select_kernels() {
     if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
     e = cudaFuncSetAttribute(budget_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)sizeof(BracketShared<kCandLarge>));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(budget_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBudgetCand * 5);
     if (e == cudaSuccess && dev >= 0 && dev < 64) done[dev] = true;
     return e;
 }
 
+size_t budget_scratch_bytes(int64_t G, int64_t H) {
+    return (size_t)G * H * kBins * sizeof(int) + (size_t)G * 256 + (size_t)G * kBudgetCand * 5;
+}
+
+// `scratch` (budget_scratch_bytes, 256-byte aligned) or null: with it, calls large enough to pay for the extra
+// launches run the parallel form of the group competition.
 cudaError_t launch_budget(int G, int H, int N, int keep, int n_safe, const float* a_star, int32_t* budgets,
-                          uint32_t* sel_thresholds, int* status, cudaStream_t stream, int64_t* launches) {
+                          uint32_t* sel_thresholds, int* status, void* scratch, cudaStream_t stream,
+                          int64_t* launches) {
     if (H > kMaxCorr) return cudaErrorInvalidValue;
     cudaError_t cfg = configure_select_kernels();
     if (cfg != cudaSuccess) return cfg;
-    safeguard_kernel<<<G * H, kStatThreads, 0, stream>>>(N, n_safe, a_star, sel_thresholds, status);
+    if (N >= 65536) safeguard_kernel<1024><<<G * H, 1024, 0, stream>>>(N, n_safe, a_star, sel_thresholds, status);
+    else safeguard_kernel<kStatThreads><<<G * H, kStatThreads, 0, stream>>>(N, n_safe, a_star, sel_thresholds, status);
     ++*launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    const int* flagged = nullptr;
+    if (scratch && (int64_t)H * N >= 200000 && (int64_t)G * H <= 65535) {
+        unsigned char* base = static_cast<unsigned char*>(scratch);
+        int* bhist = reinterpret_cast<int*>(base);
+        int* bmeta = reinterpret_cast<int*>(base + (size_t)G * H * kBins * sizeof(int));
+        float* cand_v = reinterpret_cast<float*>(base + (size_t)G * H * kBins * sizeof(int) + (size_t)G * 256);
+        unsigned char* cand_h = reinterpret_cast<unsigned char*>(cand_v + (size_t)G * kBudgetCand);
+        e = cudaMemsetAsync(base, 0, (size_t)G * H * kBins * sizeof(int) + (size_t)G * 256, stream);
+        if (e != cudaSuccess) return e;
+        const dim3 grid((unsigned)((N + kBudgetChunk - 1) / kBudgetChunk), (unsigned)(G * H));
+        budget_hist_kernel<<<grid, 256, 0, stream>>>(N, a_star, sel_thresholds, bhist);
+        budget_find_kernel<<<G, 256, 0, stream>>>(H, keep, n_safe, sel_thresholds, bhist, bmeta);
+        budget_collect_kernel<<<grid, 256, 0, stream>>>(H, N, a_star, sel_thresholds, bmeta, cand_v, cand_h);
+        budget_finish_kernel<<<G, kThreads, kBudgetCand * 5, stream>>>(H, keep, n_safe, bhist, bmeta, cand_v, cand_h, budgets,
+                                                                      sel_thresholds, status);
+        *launches += 4;
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        flagged = bmeta;
+    }
     budget_kernel<<<G, kThreads, sizeof(BracketShared<kCandLarge>), stream>>>(H, N, keep, n_safe, a_star, budgets,
-                                                                                 sel_thresholds, status);
+                                                                                 sel_thresholds, status, flagged);
     ++*launches;
     return cudaGetLastError();
 }

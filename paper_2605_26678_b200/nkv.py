@@ -285,7 +285,9 @@ def nkv_budget(a_star: torch.Tensor, r: float, params: Optional[Params] = None,
     a_star = a_star.contiguous()
     G, H, N = a_star.shape
     budgets = torch.empty((G, H), dtype=torch.int32, device=a_star.device)
-    ws = ws if ws is not None else torch.empty(4096 + 16 * G * H, dtype=torch.uint8, device=a_star.device)
+    # status words, thresholds and the scratch of the parallel form of the group competition
+    ws = ws if ws is not None else torch.empty(8192 + 16 * G * H + G * H * 8192 + G * (256 + 5 * 8192), dtype=torch.uint8,
+                                               device=a_star.device)
     _check(h.lib.nkv_budget(h.h, _p(a_star), G, H, N, float(r), ctypes.byref(params), _p(budgets), _p(ws),
                             ws.numel(), _stream()), "nkv_budget")
     return budgets

@@ -159,7 +159,10 @@ def _random_scores(G, H, N, seed, ties):
 
 @pytest.mark.parametrize("G,H,N,r,ties", [
     (1, 1, 10, 0.5, "none"), (2, 3, 100, 0.75, "none"), (1, 8, 1000, 0.75, "many"), (2, 4, 5000, 0.95, "dense"),
-    (1, 8, 3000, 0.5, "all"), (1, 2, 4097, 0.0, "none"), (3, 8, 2048, 0.9, "dense"), (1, 5, 40, 0.95, "none")])
+    (1, 8, 3000, 0.5, "all"), (1, 2, 4097, 0.0, "none"), (3, 8, 2048, 0.9, "dense"), (1, 5, 40, 0.95, "none"),
+    # large enough for the parallel form of the group competition; "dense" and "all" overflow its candidate list
+    (2, 8, 20000, 0.75, "none"), (2, 8, 12000, 0.5, "many"), (1, 8, 16384, 0.95, "dense"), (1, 8, 9000, 0.5, "all"),
+    (3, 5, 14001, 0.9, "none")])
 def test_budget_and_select_bit_exact_on_oracle_scores(G, H, N, r, ties):
     s = _random_scores(G, H, N, seed=N + H, ties=ties)
     a_star = torch.from_numpy(s).to(DEV)
