@@ -158,15 +158,35 @@ int cuda_failed(cudaError_t e, const char* what, int line) {
         if (e__ != cudaSuccess) return cuda_failed(e__, #expr, __LINE__); \
     } while (0)
 
+// The workspace arrays of a run of groups that starts at group g0 (unit u0 = g0 * H).
+struct Bufs {
+    float *inv_norm, *mu_s, *mu_e, *inv_s, *inv_e, *a_raw, *hstat;
+    uint32_t *mm, *thr;
+    unsigned char* bscr;
+};
+Bufs bufs_at(void* ws, const Layout& L, int64_t g0, int64_t H, int64_t N, int64_t d, int64_t nb) {
+    const int64_t u0 = g0 * H;
+    Bufs b;
+    b.inv_norm = at<float>(ws, L.inv_norm) + u0 * N;
+    b.mu_s = at<float>(ws, L.mu_s) + u0 * d;
+    b.mu_e = at<float>(ws, L.mu_e) + u0 * nb * d;
+    b.inv_s = at<float>(ws, L.inv_s) + u0;
+    b.inv_e = at<float>(ws, L.inv_e) + u0 * nb;
+    b.a_raw = at<float>(ws, L.a_raw) + u0 * 3 * N;
+    b.hstat = at<float>(ws, L.hstat) + head_stat_bytes(u0) / sizeof(float);
+    b.mm = at<uint32_t>(ws, L.mm) + u0 * 6;
+    b.thr = at<uint32_t>(ws, L.thr) + u0 * 2;
+    b.bscr = at<unsigned char>(ws, L.bscr) + (g0 ? budget_scratch_bytes(g0, H) : 0);   // every term is linear in G
+    return b;
+}
+
 // The two passes over the keys (Sections 2.1-2.3): afterwards the workspace holds 1/||k||, the anchors, the
 // three raw anomalies and their per-head min/max keys.  `mark` is called once between the passes (stage
-// timing).  *sums_only stays false: the anchor arrays hold means.
+// timing).
 template <typename Mark>
-int key_scan(nkv_handle* h, const TensorView& kv, int dtype, int G, const ScoreParams& sp, void* ws, const Layout& L,
-             cudaStream_t st, Mark&& mark, bool* sums_only) {
+int key_scan(nkv_handle* h, const TensorView& kv, int dtype, int G, const ScoreParams& sp, const Bufs& B, int* status,
+             cudaStream_t st, Mark&& mark) {
     const int units = G * kv.H, N = kv.N, d = kv.d;
-    int* status = at<int>(ws, L.status);
-    *sums_only = false;
     if (stream_path_supported(sp)) {
         // pass A: norms, block sums and the current-memory anomaly; pass B: the two anchor anomalies
         // the tensor-core form walks whole heads, one CTA each: by default it runs when the heads fill
@@ -176,36 +196,36 @@ int key_scan(nkv_handle* h, const TensorView& kv, int dtype, int G, const ScoreP
         const bool tensor_ok = h->key_pass != NKV_KEY_PASS_FMA && gram_pass_supported(kv, dtype, sp) &&
                                (h->key_pass == NKV_KEY_PASS_TENSOR || fills);
         if (tensor_ok)
-            CU(launch_gram_pass(kv, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm), at<float>(ws, L.a_raw),
-                                at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));
+            CU(launch_gram_pass(kv, G, sp, B.mu_e, B.inv_norm, B.a_raw,
+                                B.mm, status, h->sm_count, st, &h->launches));
         else
-            CU(launch_stream_a(kv, dtype, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm),
-                               at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), status, h->sm_count, st,
+            CU(launch_stream_a(kv, dtype, G, sp, B.mu_e, B.inv_norm,
+                               B.a_raw, B.mm, status, h->sm_count, st,
                                &h->launches));
-        CU(launch_anchor_means(units, N, d, sp, at<float>(ws, L.mu_e), at<float>(ws, L.mu_s), st, &h->launches));
-        CU(launch_anchor_norms(units, d, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_s),
-                               at<float>(ws, L.inv_e), nullptr, st, &h->launches));
+        CU(launch_anchor_means(units, N, d, sp, B.mu_e, B.mu_s, st, &h->launches));
+        CU(launch_anchor_norms(units, d, sp, B.mu_s, B.mu_e, B.inv_s,
+                               B.inv_e, nullptr, st, &h->launches));
         CU(mark());
         // d = 64 tiles are too small to pay for the per-tile hand-overs: the FMA form is faster there
         const bool dots_wanted = h->key_pass == NKV_KEY_PASS_TENSOR || (h->key_pass == NKV_KEY_PASS_AUTO && d == 128);
         if (dots_wanted && anchor_dots_supported(kv, dtype, sp))
-            CU(launch_anchor_dots(kv, G, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm),
-                                  at<float>(ws, L.inv_s), at<float>(ws, L.inv_e), at<float>(ws, L.a_raw),
-                                  at<uint32_t>(ws, L.mm), status, h->sm_count, st, &h->launches));
+            CU(launch_anchor_dots(kv, G, sp, B.mu_s, B.mu_e, B.inv_norm,
+                                  B.inv_s, B.inv_e, B.a_raw,
+                                  B.mm, status, h->sm_count, st, &h->launches));
         else
-            CU(launch_stream_b(kv, dtype, G, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e),
-                               at<float>(ws, L.inv_norm), at<float>(ws, L.inv_s), at<float>(ws, L.inv_e),
-                               at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), status, h->sm_count, st,
+            CU(launch_stream_b(kv, dtype, G, sp, B.mu_s, B.mu_e,
+                               B.inv_norm, B.inv_s, B.inv_e,
+                               B.a_raw, B.mm, status, h->sm_count, st,
                                &h->launches));
     } else {
-        CU(launch_anchor_sums(kv, dtype, G, sp, at<float>(ws, L.mu_e), at<float>(ws, L.inv_norm), st, &h->launches));
-        CU(launch_anchor_means(units, N, d, sp, at<float>(ws, L.mu_e), at<float>(ws, L.mu_s), st, &h->launches));
-        CU(launch_anchor_norms(units, d, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e), at<float>(ws, L.inv_s),
-                               at<float>(ws, L.inv_e), at<uint32_t>(ws, L.mm), st, &h->launches));
+        CU(launch_anchor_sums(kv, dtype, G, sp, B.mu_e, B.inv_norm, st, &h->launches));
+        CU(launch_anchor_means(units, N, d, sp, B.mu_e, B.mu_s, st, &h->launches));
+        CU(launch_anchor_norms(units, d, sp, B.mu_s, B.mu_e, B.inv_s,
+                               B.inv_e, B.mm, st, &h->launches));
         CU(mark());
-        CU(launch_scan_scores(kv, dtype, G, sp, at<float>(ws, L.mu_s), at<float>(ws, L.mu_e),
-                              at<float>(ws, L.inv_norm), at<float>(ws, L.inv_s), at<float>(ws, L.inv_e),
-                              at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), st, &h->launches));
+        CU(launch_scan_scores(kv, dtype, G, sp, B.mu_s, B.mu_e,
+                              B.inv_norm, B.inv_s, B.inv_e,
+                              B.a_raw, B.mm, st, &h->launches));
     }
     return NKV_OK;
 }
@@ -491,22 +511,40 @@ int nkv_compress(nkv_handle* h, const nkv_tensor* K, const nkv_tensor* V, double
 
     CU(cudaMemsetAsync(status, 0, kStatusWords * sizeof(int), st));
     CU(mark());
-    bool sums_only = false;
-    if ((rc = key_scan(h, kv, K->dtype, G, sp, ws, L, st, mark, &sums_only))) return rc;
-    CU(mark());
-    CU(launch_head_scores(units, N, sp, at<float>(ws, L.a_raw), at<uint32_t>(ws, L.mm), a_star, nullptr,
-                          at<float>(ws, L.hstat), status, st, &h->launches));
-    CU(mark());
-    CU(launch_budget(G, H, N, (int)keep, (int)n_safe, a_star, budgets, at<uint32_t>(ws, L.thr), status,
-                     at<unsigned char>(ws, L.bscr), st,
-                     &h->launches));
-    CU(mark());
-    CU(launch_select(G, H, N, (int64_t)H * keep, a_star, budgets, at<uint32_t>(ws, L.thr), idx, head_offsets, status,
-                     st, &h->launches));
-    CU(mark());
-    CU(launch_gather(kv, kb, vv, vb, G, idx, head_offsets, (int64_t)H * keep, K_out, V_out, h->sm_count, st,
-                     &h->launches));
-    CU(mark());
+    // One run of groups: the key scan on `ks`, everything after it on `ss`.
+    auto run = [&](int g0, int gc, cudaStream_t ks, cudaStream_t ss, cudaEvent_t scanned) -> int {
+        const Bufs B = bufs_at(ws, L, g0, H, N, d, sp.nblocks);
+        TensorView kc = kv, vc = vv;
+        kc.ptr = static_cast<const unsigned char*>(kv.ptr) + (size_t)g0 * kv.stride_g * kb;
+        vc.ptr = static_cast<const unsigned char*>(vv.ptr) + (size_t)g0 * vv.stride_g * vb;
+        float* as = a_star + (size_t)g0 * H * N;
+        int32_t* bud = budgets + (size_t)g0 * H;
+        int32_t* ix = idx + (size_t)g0 * H * keep;
+        int32_t* ho = head_offsets + (size_t)g0 * (H + 1);
+        int rc2 = key_scan(h, kc, K->dtype, gc, sp, B, status, ks, mark);
+        if (rc2) return rc2;
+        CU(mark());
+        if (ss != ks) {
+            CU(cudaEventRecord(scanned, ks));
+            CU(cudaStreamWaitEvent(ss, scanned, 0));
+        }
+        CU(launch_head_scores(gc * H, N, sp, B.a_raw, B.mm, as, nullptr, B.hstat, status, ss, &h->launches));
+        CU(mark());
+        CU(launch_budget(gc, H, N, (int)keep, (int)n_safe, as, bud, B.thr, status, B.bscr, ss, &h->launches));
+        CU(mark());
+        CU(launch_select(gc, H, N, (int64_t)H * keep, as, bud, B.thr, ix, ho, status, ss, &h->launches));
+        CU(mark());
+        CU(launch_gather(kc, kb, vc, vb, gc, ix, ho, (int64_t)H * keep,
+                         static_cast<unsigned char*>(K_out) + (size_t)g0 * H * keep * kv.d * kb,
+                         static_cast<unsigned char*>(V_out) + (size_t)g0 * H * keep * vv.d * vb, h->sm_count, ss,
+                         &h->launches));
+        CU(mark());
+        return NKV_OK;
+    };
+    // Running a call as two halves on two streams (the score side of one half beside the second key pass and
+    // the compaction of the other) measured no faster: the first key pass leaves no registers for a second
+    // kernel on its SMs, and beside the second pass the score kernels get a quarter of their CTAs.
+    if ((rc = run(0, G, st, st, nullptr))) return rc;
     if (timing) h->timing_valid = 1;
     return NKV_OK;
 }
@@ -661,9 +699,10 @@ int nkv_key_scan(nkv_handle* h, const nkv_tensor* K, const nkv_params* params, f
     if ((rc = check_ws(ws, ws_bytes, L.total))) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     CU(cudaMemsetAsync(at<int>(ws, L.status), 0, kStatusWords * sizeof(int), st));
-    bool sums_only = false;
     auto no_mark = []() -> cudaError_t { return cudaSuccess; };
-    if ((rc = key_scan(h, view_of(K), K->dtype, G, sp, ws, L, st, no_mark, &sums_only))) return rc;
+    if ((rc = key_scan(h, view_of(K), K->dtype, G, sp, bufs_at(ws, L, 0, K->H, N, d, sp.nblocks), at<int>(ws, L.status), st,
+                       no_mark)))
+        return rc;
     CU(cudaMemcpyAsync(mu_s, at<float>(ws, L.mu_s), (size_t)units * d * 4, cudaMemcpyDeviceToDevice, st));
     CU(cudaMemcpyAsync(mu_e, at<float>(ws, L.mu_e), (size_t)units * sp.nblocks * d * 4, cudaMemcpyDeviceToDevice, st));
     CU(cudaMemcpyAsync(inv_norm, at<float>(ws, L.inv_norm), (size_t)units * N * 4, cudaMemcpyDeviceToDevice, st));

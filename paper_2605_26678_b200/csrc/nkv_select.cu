@@ -1408,7 +1408,8 @@ cudaError_t launch_budget(int G, int H, int N, int keep, int n_safe, const float
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const int* flagged = nullptr;
-    if (scratch && (int64_t)H * N >= 200000 && (int64_t)G * H <= 65535) {
+    // with a group per SM or so the one-CTA kernel already fills the GPU and reads the scores once
+    if (scratch && (int64_t)H * N >= 200000 && G <= 64) {
         unsigned char* base = static_cast<unsigned char*>(scratch);
         int* bhist = reinterpret_cast<int*>(base);
         int* bmeta = reinterpret_cast<int*>(base + (size_t)G * H * kBins * sizeof(int));
