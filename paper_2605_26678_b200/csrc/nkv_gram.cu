@@ -51,11 +51,12 @@ constexpr int kThreads = 22 * 32;
 constexpr int kWRing = 2048;                  // per-row scalars kept in rings of 2048 rows
 constexpr int kCfRing = 4;                    // band -> scan hand-over buffers
 constexpr int kWReady = 8;                    // norms -> band hand-over barriers
+constexpr int kPpRing = 4;                    // norms -> scan hand-over buffers (segment sums of a span)
 constexpr uint32_t kTmemCols = 512;           // two accumulators of 256 columns
 constexpr int kBarNorm = 1, kBarBand = 2, kBarScan = 3;   // named barriers
 
 struct Smem {
-    float pp[2][16 * kD];        // sums of normalised keys of the 16 eight-row segments of a span
+    float pp[kPpRing][16 * kD];  // sums of normalised keys of the 16 eight-row segments of a span
     float w[kWRing];             // 1/||k|| by row (0 outside the head)
     float g[kWRing];             // g_ii by row
     float c[kCfRing][kTile];     // backward band sums of a tile
@@ -72,6 +73,7 @@ struct Smem {
     uint64_t wready[kWReady];    // norms of a span written
     uint64_t cready[kCfRing];    // band sums of a tile written
     uint64_t cfree[kCfRing];     // band sums of a tile consumed
+    uint64_t ppfree[kPpRing];    // segment sums of a span consumed
     uint64_t drain;              // products issued before a give-up have completed
     uint32_t tmem_base;
 };
@@ -264,50 +266,30 @@ __device__ __forceinline__ float segment_range_sum(const float* v, int a, int b)
 }
 
 // Span tau of a head covers rows [128 tau + 64, 128 tau + 192), tau = -1 .. T-1: always 64 rows ahead of
-// what the band sums of tile tau need.
-__device__ void norms_role(const unsigned char* ring, Smem* s, ScoreParams sp, int units, int N, int T,
-                           float* __restrict__ block_sums, int* status) {
+// what the band sums of tile tau need.  The segment sums of a span go to the scan group, which adds them up
+// into block sums (one thread per column) while this group is already on the next span.
+__device__ void norms_role(const unsigned char* ring, Smem* s, int units, int N, int T, int* status) {
     const int t = threadIdx.x - kNormWarp0 * 32;
     const int grp = t >> 4, l = t & 15;
-    const int b = sp.block;
     long long hb = 0, gs = 0;
     int rb = 64;   // ring index of the head's row 0 (see ring_advance)
     for (int u = blockIdx.x; u < units; u += gridDim.x) {
-        float run = 0.f;   // running block sum of column t (t < 128)
-        int blk = 0, blk_end = min(b, N);   // block being summed and the row it ends before
         for (int tau = -1; tau < T; ++tau, ++gs) {
             int p0, p1;
             uint32_t fc0, fc1;
             slab_slot(hb + 2 * tau + 2, p0, fc0);
             slab_slot(hb + 2 * tau + 3, p1, fc1);
-            bool ok = mbar_wait(&s->full[p0], fc0 & 1u, status, 704);
+            const int pi = (int)(gs & (kPpRing - 1));
+            bool ok = mbar_wait(&s->ppfree[pi], (uint32_t)(((gs >> 2) & 1) ^ 1), status, 709);
+            ok = ok && mbar_wait(&s->full[p0], fc0 & 1u, status, 704);
             ok = ok && mbar_wait(&s->full[p1], fc1 & 1u, status, 704);
             const int R1 = kTile * tau + 64;
-            float* pp = s->pp[gs & 1];
-            span_norms_and_sums(ring, p0, p1, s, pp, R1, N, rb, grp, l);
+            span_norms_and_sums(ring, p0, p1, s, s->pp[pi], R1, N, rb, grp, l);
             if (bar_or(kBarNorm, kNormThreads, !ok)) return;
-            if (t == 0) {   // every thread is done with the two slabs and has written its norms
+            if (t == 0) {   // every thread is done with the two slabs and has written its norms and segment sums
                 mbar_arrive(&s->sfree[p0]);
                 mbar_arrive(&s->sfree[p1]);
                 mbar_arrive(&s->wready[gs & (kWReady - 1)]);
-            }
-            if (t < kD) {
-                // block sums of column t: a block that closes inside this span is written out, the
-                // rest of the span starts the next one (rows outside the head are zeros)
-                float v[16];
-#pragma unroll
-                for (int sg = 0; sg < 16; ++sg) v[sg] = pp[sg * kD + t];
-                int s0 = 0;   // first segment not yet added
-                while (blk < sp.nblocks && blk_end <= R1 + kTile) {
-                    const int s1 = (blk_end - R1 + kSeg - 1) / kSeg;   // segments [s0, s1) close the block
-                    run += segment_range_sum(v, s0, s1);
-                    block_sums[((int64_t)u * sp.nblocks + blk) * kD + t] = run;
-                    run = 0.f;
-                    ++blk;
-                    blk_end = min(blk_end + b, N);
-                    s0 = s1;
-                }
-                run += segment_range_sum(v, s0, 16);
             }
         }
         hb += 2 * T + 2;
@@ -316,71 +298,121 @@ __device__ void norms_role(const unsigned char* ring, Smem* s, ScoreParams sp, i
 }
 
 // ---------------------------------------------------------------------------- band group
-// Band sums of one row of D.  The thread's row has its diagonal at column 64 + r.  side 0 sums the 64
-// columns that end at the diagonal, side 1 the 64 columns that start there; both live in three
-// 32-column chunks starting at column `taddr` points to, of which the first and the last are cut by the
-// diagonal: column o of the first chunk counts when o >= thr, column o of the last when o < thr.
-// Returns the three chunk sums, every column weighted by its key's 1/||k||; row0 is the ring index of
-// the first column's key.
-__device__ __forceinline__ void band_sums(uint32_t taddr, const float* wring, int row0, int thr, float& X, float& Y,
-                                          float& Z) {
-    const float* wA = wring + (row0 & (kWRing - 1));
-    const float* wB = wring + ((row0 + 32) & (kWRing - 1));
-    const float* wC = wring + ((row0 + 64) & (kWRing - 1));
-    // 16 columns of the first chunk and the 16 columns 64 further on share the diagonal test: column o
-    // of the first chunk counts exactly when column o of the last one does not
-    auto cut16 = [&](const float* a, const float* c, const float* wa, const float* wc, int col0, float& xa, float& xb,
-                     float& za, float& zb) {
+// Band sums of the 32 rows of one lane quarter of D.  Row lr of the quarter has its diagonal at column
+// 64 + 32 q + lr.  side 0 sums the 64 columns that end at the diagonal, side 1 the 64 columns that start there;
+// both live in three 32-column chunks starting at the column `taddr` points to, of which the first and the last
+// are cut by the diagonal: column o of the first chunk counts when o >= lr + (side == 0), column o of the last
+// when it does not.  Every column is weighted by its key's 1/||k||; row0 is the ring index of the first column's key.
+//
+// The accumulator is read in the fragment layout (tmem_ld_frag32): a thread holds columns 8 k + b0 + e
+// (b0 = 2 (t % 4), k = 0..3, e = 0, 1) of the four rows lr = 8 J + t / 4.  The weights of its eight columns per
+// chunk are two-float loads that eight lanes share, which costs a twelfth of the shared-memory wavefronts that a
+// thread-per-row walk spends on broadcasting every weight to every row.  With r0 = t / 4 + (side == 0) the cut
+// 8 k + b0 + e >= 8 J + r0 is decided by k alone unless k == J (0 <= b0 + e <= 7, 0 <= r0 <= 8): columns with
+// k > J lie past the cut, columns with k < J before it, and the pair k == J is tested against r0.
+// Afterwards lane t holds the three chunk sums of row 8 (t % 4) + t / 4 of the quarter.
+struct ChunkSums {
+    float x[2][2], y[2][2], z[2][2];   // [row pair j][column parity e] of the half being read
+};
+
+__device__ __forceinline__ void load_w8(const float* wring, int idx, float2* w) {
 #pragma unroll
-        for (int o4 = 0; o4 < 4; ++o4) {
-            const float4 fa = *reinterpret_cast<const float4*>(wa + 4 * o4);
-            const float4 fc = *reinterpret_cast<const float4*>(wc + 4 * o4);
-            const float was[4] = {fa.x, fa.y, fa.z, fa.w}, wcs[4] = {fc.x, fc.y, fc.z, fc.w};
+    for (int k = 0; k < 4; ++k) w[k] = *reinterpret_cast<const float2*>(wring + ((idx + 8 * k) & (kWRing - 1)));
+}
+
+template <int kChunk>
+__device__ __forceinline__ void chunk_fma(const float* v, const float2* w, int half, bool p0, bool p1, ChunkSums& cs) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int o = 4 * o4 + e;
-                float& x = (e & 1) ? xb : xa;
-                float& z = (e & 1) ? zb : za;
-                if (col0 + o >= thr) x = fmaf(a[o], was[e], x);
-                else z = fmaf(c[o], wcs[e], z);
+    for (int j = 0; j < 2; ++j) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float v0 = v[4 * k + 2 * j], v1 = v[4 * k + 2 * j + 1];
+            if (kChunk == 1) {
+                cs.y[j][0] = fmaf(v0, w[k].x, cs.y[j][0]);
+                cs.y[j][1] = fmaf(v1, w[k].y, cs.y[j][1]);
+            } else {
+                // J = 2 half + j is known only at run time as far as `half` goes; both halves are unrolled by the caller
+                const int J = 2 * half + j;
+                const bool past = k > J, at = k == J;
+                if (kChunk == 0) {
+                    if (past || at) {
+                        cs.x[j][0] = fmaf((past || p0) ? v0 : 0.f, w[k].x, cs.x[j][0]);
+                        cs.x[j][1] = fmaf((past || p1) ? v1 : 0.f, w[k].y, cs.x[j][1]);
+                    }
+                } else {
+                    if (k < J || at) {
+                        cs.z[j][0] = fmaf((k < J || !p0) ? v0 : 0.f, w[k].x, cs.z[j][0]);
+                        cs.z[j][1] = fmaf((k < J || !p1) ? v1 : 0.f, w[k].y, cs.z[j][1]);
+                    }
+                }
             }
         }
-    };
-    auto dot16 = [&](const float* v, const float* w, float& s0, float& s1) {
+    }
+}
+
+// X, Y, Z[J]: chunk sums of row 8 J + t / 4 over this thread's columns (to be added up over the four lanes t % 4)
+template <int kSide>
+__device__ __forceinline__ void band_sums(uint32_t taddr, const float* wring, int row0, int t, float* X, float* Y,
+                                          float* Z) {
+    const int b0 = 2 * (t & 3), r0 = (t >> 2) + (kSide == 0 ? 1 : 0);
+    const bool p0 = b0 >= r0, p1 = b0 + 1 >= r0;
+    const int i0 = (row0 + b0) & (kWRing - 1);
+    float a[16], b[16], c[16];
+    float2 w[4];
 #pragma unroll
-        for (int o4 = 0; o4 < 4; ++o4) {
-            const float4 ww = *reinterpret_cast<const float4*>(w + 4 * o4);
-            s0 = fmaf(v[4 * o4], ww.x, s0);
-            s1 = fmaf(v[4 * o4 + 1], ww.y, s1);
-            s0 = fmaf(v[4 * o4 + 2], ww.z, s0);
-            s1 = fmaf(v[4 * o4 + 3], ww.w, s1);
+    for (int half = 0; half < 2; ++half) {
+        const uint32_t ta = taddr + ((uint32_t)(16 * half) << 16);
+        ChunkSums cs;
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) cs.x[j][e] = cs.y[j][e] = cs.z[j][e] = 0.f;
+        tmem_ld_frag32(ta, a);
+        tmem_ld_frag32(ta + 32, b);
+        tmem_wait_ld(a, b);
+        tmem_ld_frag32(ta + 64, c);
+        load_w8(wring, i0, w);
+        chunk_fma<0>(a, w, half, p0, p1, cs);
+        load_w8(wring, i0 + 32, w);
+        chunk_fma<1>(b, w, half, p0, p1, cs);
+        tmem_wait_ld(c);
+        load_w8(wring, i0 + 64, w);
+        chunk_fma<2>(c, w, half, p0, p1, cs);
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            X[2 * half + j] = cs.x[j][0] + cs.x[j][1];
+            Y[2 * half + j] = cs.y[j][0] + cs.y[j][1];
+            Z[2 * half + j] = cs.z[j][0] + cs.z[j][1];
         }
-    };
-    float x0 = 0.f, x1 = 0.f, y0 = 0.f, y1 = 0.f, z0 = 0.f, z1 = 0.f;
-    float p0[16], p1[16], p2[16], p3[16];
-    // the loads of the next pair of 16-column pieces are in flight while the current pair is summed
-    tmem_ld16(taddr, p0);
-    tmem_ld16(taddr + 64, p1);
-    tmem_wait_ld(p0, p1);
-    tmem_ld16(taddr + 16, p2);
-    tmem_ld16(taddr + 80, p3);
-    cut16(p0, p1, wA, wC, 0, x0, x1, z0, z1);
-    tmem_wait_ld(p2, p3);
-    tmem_ld16(taddr + 32, p0);
-    tmem_ld16(taddr + 48, p1);
-    cut16(p2, p3, wA + 16, wC + 16, 16, x0, x1, z0, z1);
-    tmem_wait_ld(p0, p1);
-    dot16(p0, wB, y0, y1);
-    dot16(p1, wB + 16, y0, y1);
-    X = x0 + x1;
-    Y = y0 + y1;
-    Z = z0 + z1;
+    }
+}
+
+template <int kSide>
+__device__ __forceinline__ void band_tile(Smem* s, uint32_t taddr, int wrow0, int wrow_tile, int q, int lane, int cb) {
+    float X[4], Y[4], Z[4];
+    band_sums<kSide>(taddr, s->w, wrow0, lane, X, Y, Z);
+    float tot[4], part[4];
+#pragma unroll
+    for (int J = 0; J < 4; ++J) {
+        tot[J] = X[J] + Y[J] + Z[J];
+        part[J] = q == 2 ? Z[J] : Y[J] + Z[J];
+    }
+    treduce<4, 4>(tot, lane & 3);
+    const int r = 32 * q + 8 * (lane & 3) + (lane >> 2);   // the row whose sums this lane now holds
+    const float wi = s->w[(wrow_tile + r) & (kWRing - 1)];
+    if (kSide == 0) {
+        treduce<4, 4>(part, lane & 3);
+        s->c[cb][r] = wi * tot[0];
+        // Gram block of the tile's last 64 rows: columns 128 .. diagonal of rows 64 .. 127
+        s->bp[cb][r] = q >= 2 ? wi * part[0] : 0.f;
+    } else {
+        s->f[cb][r] = wi * tot[0];
+    }
 }
 
 __device__ void band_role(Smem* s, uint32_t tmem_base, int units, int T, int* status) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int q = warp & 3, side = warp >> 2;   // quarter of the tile's rows, backward / forward band
-    const int r = q * 32 + lane;                // row of the tile
     long long sb = 0, gt = 0;
     int rb = 64;
     for (int u = blockIdx.x; u < units; u += gridDim.x) {
@@ -394,17 +426,9 @@ __device__ void band_role(Smem* s, uint32_t tmem_base, int units, int T, int* st
             const int R0 = kTile * tau;
             const int cA = 32 * q + 64 * side;   // first column of the first chunk
             const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(st * 256 + cA);
-            float X, Y, Z;
-            band_sums(taddr, s->w, rb + R0 - 64 + cA, lane + (side == 0 ? 1 : 0), X, Y, Z);
+            if (side == 0) band_tile<0>(s, taddr, rb + R0 - 64 + cA, rb + R0, q, lane, cb);
+            else band_tile<1>(s, taddr, rb + R0 - 64 + cA, rb + R0, q, lane, cb);
             tc_fence_before();
-            const float wi = s->w[(rb + R0 + r) & (kWRing - 1)];
-            if (side == 0) {
-                s->c[cb][r] = wi * (X + Y + Z);
-                // Gram block of the tile's last 64 rows: columns 128 .. diagonal of rows 64 .. 127
-                s->bp[cb][r] = q == 2 ? wi * Z : q == 3 ? wi * (Y + Z) : 0.f;
-            } else {
-                s->f[cb][r] = wi * (X + Y + Z);
-            }
             if (bar_or(kBarBand, kBandThreads, !ok)) return;
             if (tid == 0) {
                 mbar_arrive(&s->tempty[st]);
@@ -418,14 +442,41 @@ __device__ void band_role(Smem* s, uint32_t tmem_base, int units, int T, int* st
 
 // ---------------------------------------------------------------------------- scan group
 // Thread r owns row r of the tile: T_i = anchor + prefix of (2 c_i - g_ii) - (2 f_{i-64} - g_{i-64,i-64}).
-__device__ void scan_role(Smem* s, int units, int N, int T, float* __restrict__ inv_norm, float* __restrict__ a_raw,
-                          uint32_t* __restrict__ mm, int* status) {
+// Block sums of column `col` over one span (rows [R1, R1 + 128), 16 segment sums in pp): a block that closes
+// inside the span is written out, the rest of the span starts the next one (rows outside the head are zeros).
+struct BlockWalk {
+    float run;     // running sum of the open block
+    int blk;       // the open block
+    int blk_end;   // the row it ends before
+};
+
+__device__ __forceinline__ void span_block_sums(const float* pp, int R1, int col, const ScoreParams& sp, int N, int64_t u,
+                                                float* __restrict__ block_sums, BlockWalk& bw) {
+    float v[16];
+#pragma unroll
+    for (int sg = 0; sg < 16; ++sg) v[sg] = pp[sg * kD + col];
+    int s0 = 0;   // first segment not yet added
+    while (bw.blk < sp.nblocks && bw.blk_end <= R1 + kTile) {
+        const int s1 = (bw.blk_end - R1 + kSeg - 1) / kSeg;   // segments [s0, s1) close the block
+        bw.run += segment_range_sum(v, s0, s1);
+        block_sums[(u * sp.nblocks + bw.blk) * kD + col] = bw.run;
+        bw.run = 0.f;
+        ++bw.blk;
+        bw.blk_end = min(bw.blk_end + sp.block, N);
+        s0 = s1;
+    }
+    bw.run += segment_range_sum(v, s0, 16);
+}
+
+__device__ void scan_role(Smem* s, ScoreParams sp, int units, int N, int T, float* __restrict__ block_sums,
+                          float* __restrict__ inv_norm, float* __restrict__ a_raw, uint32_t* __restrict__ mm, int* status) {
     const int r = threadIdx.x - kScanWarp0 * 32;
     const int q = r >> 5, lane = r & 31;
-    long long gt = 0;
+    long long gt = 0, sb = 0;
     int rb = 64;
     for (int u = blockIdx.x; u < units; u += gridDim.x) {
         float lo = INFINITY, hi = -INFINITY;
+        BlockWalk bw = {0.f, 0, min(sp.block, N)};
         if (r == 0) s->anchor[gt & 1] = 0.f;
         for (int tau = 0; tau < T; ++tau, ++gt) {
             const int cb = (int)(gt & (kCfRing - 1)), pb = (int)((gt - 1) & (kCfRing - 1)), par = (int)(gt & 1);
@@ -446,9 +497,17 @@ __device__ void scan_role(Smem* s, int units, int N, int T, float* __restrict__ 
             const float ap = warp_sum(q >= 2 ? 2.f * s->bp[cb][r] - gi : 0.f);
             if (lane == 31) s->wtot[par][q] = x;
             if (lane == 0) s->apart[par][q] = ap;
+            // the spans whose norms this tile's band sums waited for are complete: column r of their segment sums
+            const long long gs = sb + tau + 1;
+            if (tau == 0) span_block_sums(s->pp[(gs - 1) & (kPpRing - 1)], -64, r, sp, N, u, block_sums, bw);
+            span_block_sums(s->pp[gs & (kPpRing - 1)], R0 + 64, r, sp, N, u, block_sums, bw);
             if (bar_or(kBarScan, kScanThreads, !ok)) return;
-            // the previous tile's forward sums have been read by now
-            if (r == 0 && gt > 0) mbar_arrive(&s->cfree[pb]);
+            // the previous tile's forward sums and this tile's segment sums have been read by now
+            if (r == 0) {
+                if (gt > 0) mbar_arrive(&s->cfree[pb]);
+                if (tau == 0) mbar_arrive(&s->ppfree[(gs - 1) & (kPpRing - 1)]);
+                mbar_arrive(&s->ppfree[gs & (kPpRing - 1)]);
+            }
             float base = s->anchor[par];
             for (int w = 0; w < q; ++w) base += s->wtot[par][w];
             const float Ti = base + x;
@@ -481,6 +540,7 @@ __device__ void scan_role(Smem* s, int units, int N, int T, float* __restrict__ 
             }
         }
         rb = (rb + ring_advance(T)) & (kWRing - 1);
+        sb += T + 1;
     }
 }
 
@@ -510,6 +570,7 @@ gram_pass_kernel(const __grid_constant__ CUtensorMap tmap, ScoreParams sp, int u
             mbar_init(&s->cready[i], 1);
             mbar_init(&s->cfree[i], 1);
         }
+        for (int i = 0; i < kPpRing; ++i) mbar_init(&s->ppfree[i], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kMmaWarp) tmem_alloc(&s->tmem_base, kTmemCols);
@@ -525,9 +586,9 @@ gram_pass_kernel(const __grid_constant__ CUtensorMap tmap, ScoreParams sp, int u
         if (lane == 0) mma_role(ring, s, tmem_base, units, T, status);
         __syncwarp();
     } else if (warp >= kScanWarp0) {
-        scan_role(s, units, N, T, inv_norm, a_raw, mm, status);
+        scan_role(s, sp, units, N, T, block_sums, inv_norm, a_raw, mm, status);
     } else if (warp >= kNormWarp0) {
-        norms_role(ring, s, sp, units, N, T, block_sums, status);
+        norms_role(ring, s, units, N, T, status);
     } else {
         band_role(s, tmem_base, units, T, status);
     }

@@ -138,6 +138,22 @@ __device__ __forceinline__ void tmem_wait_ld(float* a) {   // the same for one g
                  : "memory");
 }
 
+// 16 lanes x 32 fp32 columns in the accumulator-fragment layout: lane base = the lane field of taddr (a multiple
+// of 16 inside the warp's quarter); thread t receives in v[4 k + 2 j + e] the element of row t / 4 + 8 j and column
+// 8 k + 2 (t % 4) + e, so four threads share a row and a thread sees the same eight columns of four rows in two loads.
+__device__ __forceinline__ void tmem_ld_frag32(uint32_t taddr, float* v) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
 // ---------------------------------------------------------------------------- UMMA (tcgen05.mma)
 // Shared-memory operand descriptor for a K-major bf16 tile stored as 8-row x 128-byte swizzle atoms
 // (the layout a 128B-swizzled TMA box of 64 bf16 columns produces): consecutive 8-row groups are
