@@ -49,13 +49,16 @@ FALLBACK_HBM_GBS = 6650.0
 
 
 def source_digest(name):
+    """Digest of a kernel's source file together with the two headers every kernel includes."""
     import hashlib
-    path = os.path.join(ROOT, "paper_2605_26678_b200", "csrc", name)
+    h = hashlib.sha256()
     try:
-        with open(path, "rb") as f:
-            return hashlib.sha256(f.read()).hexdigest()[:16]
+        for f in (name, "nkv_sm100.cuh", "nkv_common.cuh"):
+            with open(os.path.join(ROOT, "paper_2605_26678_b200", "csrc", f), "rb") as fh:
+                h.update(fh.read())
     except OSError:
         return None
+    return h.hexdigest()[:16]
 
 
 def measured_traffic_per_key(kernel, source, storage, head_dim):
