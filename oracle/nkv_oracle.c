@@ -27,9 +27,9 @@
  *   - layer budget is H * floor((1-r)*N); safeguard floor(0.20 * floor((1-r)N)).
  *
  * Pins: tests/test_oracle_*.py (closed forms, invariants, textbook special
- * cases and brute force on tiny inputs).  The numeric value of the final score
- * on realistic data is "parity unpinned" by the paper (it prints no worked
- * example); everything else is pinned.
+ * cases and brute force on tiny inputs).  The paper prints no worked example;
+ * the surprise -> gate -> final-score chain is pinned by a head constructed so
+ * that every quantity has a closed form.
  */
 #include <math.h>
 #include <stdint.h>

@@ -41,9 +41,10 @@ constexpr int kTile = 128;                    // keys per tile (rows of D)
 constexpr int kSlabRows = 64;                 // rows per staged slab
 constexpr int kRing = 8;                      // slabs in the ring
 constexpr int kSlabHalfBytes = kSlabRows * 128;             // one 64-column half of a slab
-constexpr int kHalfBytes = (kRing + 1) * kSlabHalfBytes;    // all slabs of one half are contiguous; position 8 is a
-                                                            // second copy of position 0, so that a pair of slabs
-                                                            // that starts at position 7 is contiguous too
+constexpr int kMirror = 2;                                  // positions 8 and 9 hold second copies of positions 0 and 1,
+                                                            // so that a run of up to four slabs that starts at
+                                                            // position 6 or 7 is contiguous too
+constexpr int kHalfBytes = (kRing + kMirror) * kSlabHalfBytes;   // all slabs of one half are contiguous
 constexpr int kRingBytes = 2 * kHalfBytes;
 constexpr int kBandThreads = 256, kNormThreads = 256, kScanThreads = 128;
 constexpr int kNormWarp0 = 8, kScanWarp0 = 16, kProducerWarp = 20, kMmaWarp = 21;
@@ -79,12 +80,12 @@ struct Smem {
 };
 constexpr size_t kSmemBytes = 1024 + kRingBytes + sizeof(Smem);
 
-// Slab q of a CTA's slab sequence sits at ring position p and is the fc-th use of that position.
-// Positions are handed out so that the two slabs of a tile's own rows are adjacent (even, odd).
+// Slab q of a CTA's slab sequence sits at ring position p and is the fc-th use of that position.  A head
+// starts at an even q, so the four slabs that a tile's product reads as B start at an even position and the
+// two slabs of its own rows (A) at an odd one.
 __device__ __forceinline__ void slab_slot(long long q, int& p, uint32_t& fc) {
-    const long long Q = q + 7;
-    p = (int)(Q & 7);
-    fc = (uint32_t)(Q >> 3) - (p != 7 ? 1u : 0u);
+    p = (int)(q & 7);
+    fc = (uint32_t)(q >> 3);
 }
 
 // The per-row rings (1/||k||, g_ii) are indexed by a row count that keeps running from head to head, so
@@ -140,9 +141,9 @@ __device__ void producer_role(const CUtensorMap* tmap, unsigned char* ring, Smem
                 }
                 return;
             }
-            mbar_expect_tx(&s->full[p], (p == 0 ? 4 : 2) * kSlabHalfBytes);
-            for (int copy = 0; copy < (p == 0 ? 2 : 1); ++copy) {
-                unsigned char* dst = ring + (size_t)(copy ? kRing : p) * kSlabHalfBytes;
+            mbar_expect_tx(&s->full[p], (p < kMirror ? 4 : 2) * kSlabHalfBytes);
+            for (int copy = 0; copy < (p < kMirror ? 2 : 1); ++copy) {
+                unsigned char* dst = ring + (size_t)(copy ? kRing + p : p) * kSlabHalfBytes;
                 tma_load_4d(dst, tmap, 0, kSlabRows * (lam - 1), h, g, &s->full[p]);
                 tma_load_4d(dst + kHalfBytes, tmap, 64, kSlabRows * (lam - 1), h, g, &s->full[p]);
             }
@@ -151,7 +152,8 @@ __device__ void producer_role(const CUtensorMap* tmap, unsigned char* ring, Smem
 }
 
 // MMA issuer (one thread).  Tile tau of a head: A = slabs 2 tau + 1, 2 tau + 2 (the tile's rows),
-// B = slabs 2 tau .. 2 tau + 3 as two pairs, two MMAs of N = 128 per 16-wide K step.
+// B = slabs 2 tau .. 2 tau + 3, one MMA of N = 256 per 16-wide K step (half the operand reads of A and half the
+// instructions of two N = 128 products).
 // Products already issued keep reading shared memory and writing tensor memory: a role that gives up
 // waits (bounded) for them before the CTA frees both.
 __device__ __forceinline__ void drain_products(Smem* s) {
@@ -160,7 +162,7 @@ __device__ __forceinline__ void drain_products(Smem* s) {
 }
 
 __device__ void mma_role(unsigned char* ring, Smem* s, uint32_t tmem_base, int units, int T, int* status) {
-    constexpr uint32_t idesc = umma_idesc_bf16(kTile, 128);
+    constexpr uint32_t idesc = umma_idesc_bf16(kTile, 256);
     const uint32_t ring_addr = smem_addr(ring);
     long long hb = 0, gt = 0;
     for (int u = blockIdx.x; u < units; u += gridDim.x) {
@@ -174,19 +176,15 @@ __device__ void mma_role(unsigned char* ring, Smem* s, uint32_t tmem_base, int u
             const int st = (int)(gt & 1);
             if (!mbar_wait(&s->tempty[st], (uint32_t)(((gt >> 1) & 1) ^ 1), status, 703)) return drain_products(s);
             tc_fence_after();
-            int pa;
+            int pa, pb;   // odd and even; what follows position 7 is read from the copies at positions 8 and 9
             slab_slot(hb + 2 * tau + 1, pa, fc);
+            slab_slot(hb + 2 * tau, pb, fc);
 #pragma unroll
-            for (int n = 0; n < 2; ++n) {
-                int pb;   // odd; the slab after position 7 is read from the copy at position 8
-                slab_slot(hb + 2 * tau + 2 * n, pb, fc);
-#pragma unroll
-                for (int kk = 0; kk < kD / 16; ++kk) {
-                    const uint32_t koff = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
-                    const uint64_t adesc = umma_desc_sw128(ring_addr + (uint32_t)pa * kSlabHalfBytes + koff);
-                    const uint64_t bdesc = umma_desc_sw128(ring_addr + (uint32_t)pb * kSlabHalfBytes + koff);
-                    umma_bf16(tmem_base + (uint32_t)st * 256u + (uint32_t)n * 128u, adesc, bdesc, idesc, kk > 0);
-                }
+            for (int kk = 0; kk < kD / 16; ++kk) {
+                const uint32_t koff = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
+                const uint64_t adesc = umma_desc_sw128(ring_addr + (uint32_t)pa * kSlabHalfBytes + koff);
+                const uint64_t bdesc = umma_desc_sw128(ring_addr + (uint32_t)pb * kSlabHalfBytes + koff);
+                umma_bf16(tmem_base + (uint32_t)st * 256u, adesc, bdesc, idesc, kk > 0);
             }
             umma_commit(&s->tfull[st]);
             for (int lam = 2 * tau; lam <= (tau == T - 1 ? 2 * tau + 3 : 2 * tau + 1); ++lam) {
