@@ -290,6 +290,16 @@ enum { NKV_DEBUG_INJECT_HOST_STATUS = 5 };
 NKV_API int nkv_debug_set(nkv_handle* h, int what, int64_t value);
 
 /*
+ * Test hook (no counterpart in the paper): runs the bounded wait that the tensor-core key passes use for their
+ * hand-overs on a barrier that nothing arrives at.  One warp polls `polls` times (1 .. 65536; a poll takes well
+ * under a microsecond), gives up and records NKV_ERR_TIMEOUT in the status words at the start of `ws` (device,
+ * >= 256 bytes, 256-byte aligned), which nkv_last_device_status then reports.  The kernel touches nothing else,
+ * so the device stays usable: this is how a wait that runs out is tested without a kernel that hangs.
+ * Enqueues on `stream` and returns.
+ */
+NKV_API int nkv_debug_wait_probe(nkv_handle* h, int64_t polls, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * nkv_budget for callers that cannot allocate device memory (the paper has no
  * counterpart: this is a packaging variant of nkv_budget, same arithmetic,
  * same kernel).  A host that runs inside a memory pool fixed at start-up, a

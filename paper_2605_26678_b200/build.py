@@ -11,7 +11,7 @@ CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libnkv.so")
 
-SOURCES = ["nkv_api.cu", "nkv_scan.cu", "nkv_stream.cu", "nkv_gram.cu", "nkv_dots.cu", "nkv_select.cu", "nkv_compact.cu", "nkv_noalloc.cu"]
+SOURCES = ["nkv_api.cu", "nkv_scan.cu", "nkv_stream.cu", "nkv_gram.cu", "nkv_dots.cu", "nkv_select.cu", "nkv_compact.cu", "nkv_noalloc.cu", "nkv_waitprobe.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",

@@ -726,6 +726,16 @@ int nkv_debug_set(nkv_handle* h, int what, int64_t value) {
     }
 }
 
+int nkv_debug_wait_probe(nkv_handle* h, int64_t polls, void* ws, size_t ws_bytes, void* stream) {
+    if (!h || polls < 1 || polls > (1 << 16)) return NKV_ERR_INVALID_ARG;
+    int rc = check_ws(ws, ws_bytes, align_up(kStatusWords * sizeof(int)));
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    CU(cudaMemsetAsync(ws, 0, kStatusWords * sizeof(int), st));
+    CU(launch_wait_probe(static_cast<int*>(ws), (uint32_t)polls, st, &h->launches));
+    return NKV_OK;
+}
+
 int nkv_set_key_passes(nkv_handle* h, int mode) {
     if (!h || mode < NKV_KEY_PASS_AUTO || mode > NKV_KEY_PASS_TENSOR) return NKV_ERR_INVALID_ARG;
     h->key_pass = mode;

@@ -110,6 +110,8 @@ __device__ __forceinline__ void set_status(int* status, int code, int detail) {
 }
 
 // ---- launchers implemented in the .cu files (all enqueue on `stream`, return cudaError_t) ----
+constexpr int kWaitProbeDetail = 799;   // status detail recorded by the wait probe
+cudaError_t launch_wait_probe(int* status, uint32_t limit, cudaStream_t stream, int64_t* launches);
 cudaError_t launch_anchor_sums(const TensorView& K, int dtype, int G, const ScoreParams& sp, float* block_sums,
                                float* inv_norm, cudaStream_t stream, int64_t* launches);
 cudaError_t launch_anchor_means(int units, int N, int d, const ScoreParams& sp, float* mu_e_inout, float* mu_s,

@@ -39,8 +39,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait: false (after recording where) if the phase never completes.  The polling loop is one
 // out-of-line function: the roles of a kernel run side by side and share the instruction cache, and a
 // wait that finds its phase complete at the first look costs one instruction.
-static __device__ __noinline__ bool mbar_wait_poll(uint64_t* bar, uint32_t parity, int* status, int where) {
-    for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+static __device__ __noinline__ bool mbar_wait_poll(uint64_t* bar, uint32_t parity, int* status, int where,
+                                                  uint32_t limit = kSpinLimit) {
+    for (uint32_t spin = 0; spin < limit; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
         if (spin >= 4) __nanosleep(64);   // leave the issue slots to the warps that have work
     }

@@ -37,7 +37,7 @@ EXPORTS = (
     "nkv_workspace_bytes", "nkv_anchors", "nkv_score", "nkv_budget", "nkv_select", "nkv_compact",
     "nkv_compress", "nkv_host_staging_bytes", "nkv_compress_host", "nkv_last_device_status",
     "nkv_set_timing", "nkv_get_stage_ms", "nkv_launch_count", "nkv_budget_static", "nkv_set_key_passes",
-    "nkv_key_scan", "nkv_debug_set",
+    "nkv_key_scan", "nkv_debug_set", "nkv_debug_wait_probe",
 )
 
 
@@ -114,6 +114,7 @@ def load_library():
     L.nkv_launch_count.restype = i64
     L.nkv_key_scan.argtypes = [vp, tp, pp, vp, vp, vp, vp, vp, vp, sz, vp]
     L.nkv_debug_set.argtypes = [vp, ctypes.c_int, i64]
+    L.nkv_debug_wait_probe.argtypes = [vp, i64, vp, sz, vp]
     L.nkv_set_key_passes.argtypes = [vp, ctypes.c_int]
     L.nkv_budget_static.argtypes = [vp, i64, i64, i64, dbl, pp, vp, vp]
     _lib = L
@@ -442,6 +443,13 @@ def nkv_debug_set(what: str, value: int, h: Optional[Handle] = None) -> None:
     """Test hook of the library (see nkv.h)."""
     h = h or handle()
     _check(h.lib.nkv_debug_set(h.h, DEBUG[what], int(value)), "nkv_debug_set")
+
+
+def nkv_debug_wait_probe(polls: int, ws: torch.Tensor, h: Optional[Handle] = None) -> None:
+    """Test hook: a bounded device-side wait that runs out (see nkv.h); read the outcome with nkv_last_device_status."""
+    h = h or handle()
+    _check(h.lib.nkv_debug_wait_probe(h.h, int(polls), _p(ws), ws.numel() * ws.element_size(), _stream()),
+           "nkv_debug_wait_probe")
 
 
 def nkv_key_scan(K: torch.Tensor, params: Optional[Params] = None, ws: Optional[torch.Tensor] = None,

@@ -390,3 +390,23 @@ def test_host_entry_point_reports_a_device_status_of_any_chunk():
         finally:
             nkv.nkv_debug_set("inject_host_status", 0)
     nkv.nkv_compress_host(Kh, Vh, 0.5, out, staging, 2)           # and fine again
+
+
+@pytest.mark.gpu
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_device_usable():
+    """The hand-overs of the tensor-core key passes are bounded mbarrier waits.  The probe runs that same wait on a
+    barrier nothing arrives at: it must end by itself, the status words must say NKV_ERR_TIMEOUT with the probe's
+    detail code, and the next ordinary call on the same workspace must be clean."""
+    cfg = wl.CONFIGS["cfg1_single_layer_fp32_4k"]
+    K, V = wl.make_cache(cfg, "cuda:0")
+    p = nkv.nkv_default_params()
+    ws = nkv.alloc_workspace(K, p)
+    nkv.nkv_debug_wait_probe(2000, ws)
+    assert nkv.nkv_last_device_status(ws) == nkv.NKV_ERR_TIMEOUT
+    words = ws[:16].view(torch.int32).cpu().tolist()
+    assert words[0] == nkv.NKV_ERR_TIMEOUT and 799 in words[:4]
+    with pytest.raises(nkv.NkvError):
+        nkv.nkv_debug_wait_probe(0, ws)
+    out = nkv.nkv_compress(K, V, 0.75, p, ws=ws)
+    assert nkv.nkv_last_device_status(ws) == nkv.NKV_OK
+    assert int(out.budgets.sum()) == K.shape[1] * nkv.nkv_keep_per_head(K.shape[2], 0.75)
