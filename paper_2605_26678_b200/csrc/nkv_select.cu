@@ -265,12 +265,16 @@ struct ScaleSrc {      // values of one scale of one head; `flip` turns bottom-m
     }
 };
 
-__device__ __forceinline__ float norm01(float a, float lo, float range) { return range > 0.f ? (a - lo) / range : 0.f; }
+// Min-max normalisation with the reciprocal of the range taken once per head (0 for a constant sequence): the
+// per-token kernels are bound by instruction issue, and an IEEE division costs ten instructions.
+__device__ __forceinline__ float inv_range(float range) { return range > 0.f ? 1.0f / range : 0.f; }
+__device__ __forceinline__ float norm01(float a, float lo, float inv) { return (a - lo) * inv; }
 
 __device__ __forceinline__ float surprise3(float x0, float x1, float x2) {
-    const float mean = (x0 + x1 + x2) / 3.0f;
+    constexpr float kThird = 1.0f / 3.0f;
+    const float mean = (x0 + x1 + x2) * kThird;
     const float d0 = x0 - mean, d1 = x1 - mean, d2 = x2 - mean;
-    return sqrtf((d0 * d0 + d1 * d1 + d2 * d2) / 3.0f);
+    return sqrtf((d0 * d0 + d1 * d1 + d2 * d2) * kThird);
 }
 
 __device__ __forceinline__ float block_reduce_f(SelectShared& S, float v, int op) {  // 0 sum, 1 min, 2 max
@@ -308,6 +312,12 @@ constexpr int kSampleMin = 1024, kSampleMax = 32768;   // sample positions: n / 
 // The bracket that one sample rank error of 4 sigma spans grows with n / positions: beyond 64k elements a
 // denser sample keeps it inside the candidate buffers.
 __device__ __forceinline__ int sample_positions(int n) { return min(max(n > 65536 ? n / 4 : n / 8, kSampleMin), kSampleMax); }
+// Sample position i of `positions` over n elements is floor(i * step / 2^16) with step = floor(n * 2^16 / positions):
+// one 64-bit division per thread instead of one per sample (positions <= n, so the index stays below n).
+__device__ __forceinline__ unsigned long long sample_step(int n, int positions) {
+    return ((unsigned long long)n << 16) / (unsigned long long)positions;
+}
+__device__ __forceinline__ int sample_index(int i, unsigned long long step) { return (int)(((unsigned long long)i * step) >> 16); }
 constexpr int kCandSmall = 4096;                       // bracket capacity of the per-head kernels
 constexpr int kCandLarge = 12288;                      // ... of the per-group kernel (dynamic shared memory)
 
@@ -342,6 +352,7 @@ __device__ void block_select_bracket(SelectShared& S, BracketShared<CAP>& X, con
     if (use_bracket) {
         // 1. histogram of a strided sample (rejected elements are skipped)
         const int positions = sample_positions(n);
+        const unsigned long long step = sample_step(n, positions);
         for (int b = tid; b < kBins; b += nt) S.hist[b] = 0;
         __syncthreads();
         int mine = 0;
@@ -352,7 +363,7 @@ __device__ void block_select_bracket(SelectShared& S, BracketShared<CAP>& X, con
             for (int k = 0; k < 4; ++k) {
                 const int i = i0 + k * nt + tid;
                 sv[k] = 0.f;
-                sk[k] = i < positions && src.get((int)(((long long)i * n) / positions), sv[k]);
+                sk[k] = i < positions && src.get(sample_index(i, step), sv[k]);
             }
 #pragma unroll
             for (int k = 0; k < 4; ++k)
@@ -547,6 +558,7 @@ __device__ bool two_tail_sums(SelectShared& S, BracketShared<CAP>& X, const floa
     if (n <= CAP || 2 * m >= n) return false;
     // 1. histogram of a strided sample
     const int positions = sample_positions(n);
+    const unsigned long long step = sample_step(n, positions);
     for (int b = tid; b < kBins; b += nt) S.hist[b] = 0;
     __syncthreads();
     for (int i0 = 0; i0 < positions; i0 += 4 * nt) {   // four loads in flight per thread
@@ -554,7 +566,7 @@ __device__ bool two_tail_sums(SelectShared& S, BracketShared<CAP>& X, const floa
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             const int i = i0 + k * nt + tid;
-            sv[k] = i < positions ? a[(int)(((long long)i * n) / positions)] : 0.f;
+            sv[k] = i < positions ? a[sample_index(i, step)] : 0.f;
         }
 #pragma unroll
         for (int k = 0; k < 4; ++k)
@@ -685,11 +697,12 @@ __global__ void __launch_bounds__(kT, kT == 256 ? 4 : 1) scale_stats_kernel(int 
     const int u = blockIdx.x >> 2, task = blockIdx.x & 3;
     const float* a[3] = {a_raw + ((int64_t)u * 3 + 0) * N, a_raw + ((int64_t)u * 3 + 1) * N,
                          a_raw + ((int64_t)u * 3 + 2) * N};
-    float lo[3], range[3];
+    float lo[3], range[3], inv[3];
 #pragma unroll
     for (int k = 0; k < 3; ++k) {
         lo[k] = ord_float(mm[(int64_t)u * 6 + 2 * k]);
         range[k] = ord_float(mm[(int64_t)u * 6 + 2 * k + 1]) - lo[k];
+        inv[k] = inv_range(range[k]);
     }
     if (threadIdx.x == 0) S.ncorr = 0;
     __syncthreads();
@@ -724,7 +737,7 @@ __global__ void __launch_bounds__(kT, kT == 256 ? 4 : 1) scale_stats_kernel(int 
     } else {
         float smin = INFINITY, smax = -INFINITY, ssum = 0.f;
         auto take = [&](float r0, float r1, float r2) {
-            const float s = surprise3(norm01(r0, lo[0], range[0]), norm01(r1, lo[1], range[1]), norm01(r2, lo[2], range[2]));
+            const float s = surprise3(norm01(r0, lo[0], inv[0]), norm01(r1, lo[1], inv[1]), norm01(r2, lo[2], inv[2]));
             smin = fminf(smin, s);
             smax = fmaxf(smax, s);
             ssum += s;
@@ -783,11 +796,12 @@ __global__ void __launch_bounds__(kMixThreads) mix_kernel(int N, ScoreParams sp,
     const float* a0 = a_raw + ((int64_t)u * 3 + 0) * N;
     const float* a1 = a0 + N;
     const float* a2 = a1 + N;
-    float lo[3], range[3];
+    float lo[3], range[3], inv[3];
 #pragma unroll
     for (int k = 0; k < 3; ++k) {
         lo[k] = ord_float(mm[(int64_t)u * 6 + 2 * k]);
         range[k] = ord_float(mm[(int64_t)u * 6 + 2 * k + 1]) - lo[k];
+        inv[k] = inv_range(range[k]);
     }
     const float* hs = hstat + (int64_t)u * kHeadStat;
     float z[3], zmax = -INFINITY, wsum = 0.f, w[3];
@@ -803,24 +817,24 @@ __global__ void __launch_bounds__(kMixThreads) mix_kernel(int N, ScoreParams sp,
     }
 #pragma unroll
     for (int k = 0; k < 3; ++k) w[k] = z[k] / wsum;
-    const float s_lo = hs[3], s_range = hs[4] - hs[3];
-    const float s_mean = s_range > 0.f ? (hs[5] / (float)N - s_lo) / s_range : 0.f;
+    const float s_lo = hs[3], s_inv = inv_range(hs[4] - hs[3]);
+    const float s_mean = norm01(hs[5] / (float)N, s_lo, s_inv);
 
     const int base = blockIdx.x * (kMixThreads * kMixPerThread);
     // one token: min-max normalise, blend, gate, pin the sinks
     auto route = [&](float r0, float r1, float r2, int j) {
-        const float x0 = norm01(r0, lo[0], range[0]);
-        const float x1 = norm01(r1, lo[1], range[1]);
-        const float x2 = norm01(r2, lo[2], range[2]);
+        const float x0 = norm01(r0, lo[0], inv[0]);
+        const float x1 = norm01(r1, lo[1], inv[1]);
+        const float x2 = norm01(r2, lo[2], inv[2]);
         const float blend = w[0] * x0 + w[1] * x1 + w[2] * x2;
         const float win = fmaxf(x0, fmaxf(x1, x2));
         float alpha;
         if (sp.gate_mode == NKV_GATE_AVERAGE) alpha = 0.f;
         else if (sp.gate_mode == NKV_GATE_MAX) alpha = 1.f;
         else {
-            const float sn = norm01(surprise3(x0, x1, x2), s_lo, s_range);
+            const float sn = norm01(surprise3(x0, x1, x2), s_lo, s_inv);
             const float sprime = fmaxf(0.f, sn - s_mean);
-            alpha = 1.0f / (1.0f + expf(-sp.kappa * (sprime - sp.tau)));
+            alpha = __fdividef(1.0f, 1.0f + __expf(-sp.kappa * (sprime - sp.tau)));   // both within 2 ulp here
         }
         const float v = (1.0f - alpha) * blend + alpha * win + 0.f;
         return j < sp.n_sink ? INFINITY : v;
@@ -860,7 +874,7 @@ __global__ void __launch_bounds__(kMixThreads) mix_kernel(int N, ScoreParams sp,
             o[9 + k] = w[k];
         }
         o[12] = s_lo;
-        o[13] = s_lo + s_range;
+        o[13] = hs[4];
         o[14] = s_mean;
         o[15] = (float)sp.top_m;
     }
@@ -887,15 +901,23 @@ struct PoolSrc {       // all (head, token) pairs of a group whose key does not 
     const float* v;    // [H, N]
     const uint32_t* T; // per-head safeguard threshold keys (shared memory)
     int N;
+    float invN;
     static constexpr bool kVec = true;
+    // head of element j without an integer division: the float quotient is off by one at most
+    __device__ __forceinline__ int head_of(int j) const {
+        int h = (int)((float)j * invN);
+        if ((h + 1) * N <= j) ++h;
+        if (h * N > j) --h;
+        return h;
+    }
     __device__ __forceinline__ bool get(int j, float& x) const {
         x = v[j];
-        return ord_key(x) <= T[j / N];
+        return ord_key(x) <= T[head_of(j)];
     }
     __device__ __forceinline__ bool vec_ok() const { return (N & 3) == 0 && (reinterpret_cast<uintptr_t>(v) & 15) == 0; }
     __device__ __forceinline__ unsigned get4(int j4, float4& x) const {
         x = reinterpret_cast<const float4*>(v)[j4];
-        const uint32_t t = T[(4 * j4) / N];   // N is a multiple of 4: the four share a head
+        const uint32_t t = T[head_of(4 * j4)];   // N is a multiple of 4: the four share a head
         return (ord_key(x.x) <= t ? 1u : 0u) | (ord_key(x.y) <= t ? 2u : 0u) | (ord_key(x.z) <= t ? 4u : 0u) |
                (ord_key(x.w) <= t ? 8u : 0u);
     }
@@ -956,7 +978,7 @@ __global__ void __launch_bounds__(kThreads) budget_kernel(int H, int N, int keep
         }
         if (threadIdx.x == 0) S.ncorr = H;
         __syncthreads();
-        PoolSrc src{v, T, N};
+        PoolSrc src{v, T, N, 1.0f / (float)N};
         block_select_bracket(S, X, src, H * N, (long long)H * N - (long long)H * n_safe, rest, 0.f, (float)kBins, status,
                              nullptr);
         tau = S.theta;
