@@ -414,20 +414,17 @@ __device__ void block_select_bracket(SelectShared& S, BracketShared<CAP>& X, con
         __syncthreads();
         int cnt = 0;
         float sum = 0.f;
-        const int lane = tid & 31;
         // one element: counted (and summed) above the bracket, appended to the list inside it
         auto consume = [&](float v, bool in) {
             const bool above = in && v > p_hi;
             const bool inside = in && !above && v >= p_lo;
             cnt += above;
             if (above) sum += v;
-            const unsigned ballot = __ballot_sync(0xffffffffu, inside);
-            if (ballot) {
-                int base = 0;
-                if (lane == 0) base = atomicAdd(&X.cand_n, __popc(ballot));
-                base = __shfl_sync(0xffffffffu, base, 0);
-                const int pos = base + __popc(ballot & ((1u << lane) - 1u));
-                if (inside && pos < kCandCap) X.cand[pos] = v;
+            // a few percent of the elements: every thread appends its own (a warp-wide vote per element would
+            // send nearly every warp down the append path, which is what this pass spent its time on)
+            if (inside) {
+                const int pos = atomicAdd(&X.cand_n, 1);
+                if (pos < kCandCap) X.cand[pos] = v;
             }
         };
         bool vec = false;
@@ -554,7 +551,7 @@ __device__ bool two_tail_sums(SelectShared& S, BracketShared<CAP>& X, const floa
     constexpr int kHalf = CAP / 2;
     __shared__ int sh_n[2], sh_cnt[2], sh_ok;
     __shared__ float sh_piv[4], sh_sum[2], sh_res[2];
-    const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
+    const int tid = threadIdx.x, nt = blockDim.x;
     if (n <= CAP || 2 * m >= n) return false;
     // 1. histogram of a strided sample
     const int positions = sample_positions(n);
@@ -601,34 +598,44 @@ __device__ bool two_tail_sums(SelectShared& S, BracketShared<CAP>& X, const floa
     __syncthreads();
     int cnt_t = 0, cnt_b = 0;
     float sum_t = 0.f, sum_b = 0.f;
-    for (int jb = 0; jb < n; jb += 4 * nt) {   // four loads in flight per thread
-      float vv[4];
-#pragma unroll
-      for (int k = 0; k < 4; ++k) vv[k] = jb + k * nt + tid < n ? a[jb + k * nt + tid] : 0.f;
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const int j = jb + k * nt + tid;
-        const bool in = j < n;
-        const float v = vv[k];
+    auto take = [&](float v, bool in) {
         const bool above = in && v > pt_hi, below = in && v < pb_lo;
         const bool in_t = in && !above && v >= pt_lo, in_b = in && !below && v <= pb_hi;
         cnt_t += above;
         cnt_b += below;
         if (above) sum_t += v;
         if (below) sum_b += v;
+        if (in_t || in_b) {   // a few percent of the values: every thread appends its own
+            const int side = in_t ? 0 : 1;
+            const int pos = atomicAdd(&sh_n[side], 1);
+            if (pos < kHalf) X.cand[side * kHalf + pos] = v;
+        }
+    };
+    if ((n & 3) == 0 && (reinterpret_cast<uintptr_t>(a) & 15) == 0) {
+        // rows are 16-byte aligned: four values per load, four loads in flight per thread
+        const float4* a4 = reinterpret_cast<const float4*>(a);
+        const int n4 = n >> 2;
+        for (int jb = 0; jb < n4; jb += 4 * nt) {
+            float4 q[4];
 #pragma unroll
-        for (int side = 0; side < 2; ++side) {
-            const bool mine = side == 0 ? in_t : in_b;
-            const unsigned ballot = __ballot_sync(0xffffffffu, mine);
-            if (ballot) {
-                int base = 0;
-                if (lane == 0) base = atomicAdd(&sh_n[side], __popc(ballot));
-                base = __shfl_sync(0xffffffffu, base, 0);
-                const int pos = base + __popc(ballot & ((1u << lane) - 1u));
-                if (mine && pos < kHalf) X.cand[side * kHalf + pos] = v;
+            for (int k = 0; k < 4; ++k) q[k] = jb + k * nt + tid < n4 ? a4[jb + k * nt + tid] : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const bool in = jb + k * nt + tid < n4;
+                take(q[k].x, in);
+                take(q[k].y, in);
+                take(q[k].z, in);
+                take(q[k].w, in);
             }
         }
-      }
+    } else {
+        for (int jb = 0; jb < n; jb += 4 * nt) {   // four loads in flight per thread
+            float vv[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) vv[k] = jb + k * nt + tid < n ? a[jb + k * nt + tid] : 0.f;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) take(vv[k], jb + k * nt + tid < n);
+        }
     }
     cnt_t = block_sum_int(S, cnt_t);
     __syncthreads();
