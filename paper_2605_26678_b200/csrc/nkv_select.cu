@@ -1335,10 +1335,13 @@ __global__ void __launch_bounds__(kThreads) select_kernel(int H, int N, int64_t 
             const int jn = j0 + kThreads * 4 + e;
             nxt[e] = jn < N ? v[jn] : 0.f;
         }
-        int t_eq;
-        int tie_rank = run_eq + block_exclusive_scan(eq_cnt, warp_tot, &tot);
-        t_eq = tot;
-        __syncthreads();
+        // ties at the threshold are rare: their ranks need a scan only in rounds that hold one
+        int t_eq = 0, tie_rank = run_eq;
+        if (__syncthreads_or(eq_cnt)) {
+            tie_rank += block_exclusive_scan(eq_cnt, warp_tot, &tot);
+            t_eq = tot;
+            __syncthreads();
+        }
         int sel[4], sel_cnt = 0;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
