@@ -319,6 +319,10 @@ def run_nkv(args, cfg, r):
     if status != nkv.NKV_OK:
         raise SystemExit("device status %d after the timed region" % status)
     value, ms_per_step = whole_job_throughput(ms_total, args.steps, cfg.keys, world, dist, dev)
+    if clocks.get("sm_mhz"):
+        # million SM cycles per step at the clock sampled under load: comparable between runs that the power cap
+        # held at different clocks
+        clocks["sm_mcycles_per_step"] = ms_per_step * clocks["sm_mhz"] / 1000.0
 
     # ---- per-stage device time (events recorded on the launching stream inside the library) --
     nkv.nkv_set_timing(True, h)
