@@ -258,7 +258,7 @@ NKV_API int64_t nkv_launch_count(const nkv_handle* h);
  *   NKV_KEY_PASS_FMA     both passes with fp32 FMAs on staged key tiles (any supported dtype and d).
  *   NKV_KEY_PASS_TENSOR  (bf16 keys) forms on the tensor cores what is a contraction: in the first pass
  *       (d = 128, W = 64, one CTA per head) k_hat_i . S_i and ||S_i||^2 as sums over a band of the keys'
- *       Gram matrix; in the second pass (d = 64 or 128) the dots of the keys with the anchors, the fp32
+ *       Gram matrix, and ||k_i||^2 as its diagonal; in the second pass (d = 64 or 128) the dots of the keys with the anchors, the fp32
  *       anchors split three ways into bf16.  A pass whose inputs do not allow the tensor form runs the
  *       FMA kernel.
  *   NKV_KEY_PASS_AUTO (default) takes the tensor form of the second pass when d = 128, and of the first
