@@ -70,6 +70,7 @@ template <int D>
 __device__ void dots_producer(const CUtensorMap* tmap, unsigned char* tiles, Smem* s, TileRange tr, int H, int* status) {
     using C = Cfg<D>;
     long long n = 0;
+    const uint64_t policy = l2_evict_first_policy();   // keys are read once per pass
     for (long long t = tr.first; t < tr.last; ++t, ++n) {
         const int slot = (int)(n % C::kSlots);
         const long long fill = n / C::kSlots;
@@ -88,7 +89,7 @@ __device__ void dots_producer(const CUtensorMap* tmap, unsigned char* tiles, Sme
         mbar_expect_tx(&s->full[slot], C::kTileBytes);
 #pragma unroll
         for (int half = 0; half < C::kHalves; ++half)
-            tma_load_4d(dst + half * kTileHalfBytes, tmap, 64 * half, i0, h, g, &s->full[slot]);
+            tma_load_4d(dst + half * kTileHalfBytes, tmap, 64 * half, i0, h, g, &s->full[slot], policy);
     }
 }
 

@@ -136,6 +136,7 @@ __device__ __forceinline__ void treduce(float* v, int l) {
 __device__ void producer_role(const CUtensorMap* tmap, unsigned char* ring, Smem* s, int units, int H, int T,
                               int* status) {
     uint32_t q = 0;
+    const uint64_t policy = l2_evict_first_policy();   // keys are read once per pass
 #pragma unroll 1
     for (int u = blockIdx.x; u < units; u += gridDim.x) {
         const int g = u / H, h = u - g * H;
@@ -161,8 +162,8 @@ __device__ void producer_role(const CUtensorMap* tmap, unsigned char* ring, Smem
 #pragma unroll 1
             for (int copy = 0; copy < (p < kMirror ? 2 : 1); ++copy) {
                 unsigned char* dst = ring + (size_t)(copy ? kRing + p : p) * kSlabHalfBytes;
-                tma_load_4d(dst, tmap, 0, kSlabRows * (lam - 1), h, g, &s->full[p]);
-                tma_load_4d(dst + kHalfBytes, tmap, 64, kSlabRows * (lam - 1), h, g, &s->full[p]);
+                tma_load_4d(dst, tmap, 0, kSlabRows * (lam - 1), h, g, &s->full[p], policy);
+                tma_load_4d(dst + kHalfBytes, tmap, 64, kSlabRows * (lam - 1), h, g, &s->full[p], policy);
             }
         }
     }
