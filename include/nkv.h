@@ -176,11 +176,15 @@ NKV_API int nkv_score(nkv_handle* h, const nkv_tensor* K, const float* mu_s, con
  * (a_star descending, head ascending, position ascending).
  *   a_star   f32 [G,H,N] (sinks already +inf)
  *   budgets  out i32 [G,H], sum over H = H*k
+ *   thresholds_opt  out f32 [G,H] or NULL: the head's selection threshold: the head retains every token that
+ *            scores above it and, in position order, as many of the tokens that score exactly it as its
+ *            budget still allows (+inf while the sinks alone fill the head's budget)
  *   ws       at least 256 + 8*G*H bytes (rounded up to 256); with 8192*G*H + 42000*G bytes more, large calls
  *            spread the cross-head competition of a group over many thread blocks (same result)
  */
 NKV_API int nkv_budget(nkv_handle* h, const float* a_star, int64_t G, int64_t H, int64_t N, double r,
-               const nkv_params* params, int32_t* budgets, void* ws, size_t ws_bytes, void* stream);
+               const nkv_params* params, int32_t* budgets, float* thresholds_opt, void* ws, size_t ws_bytes,
+               void* stream);
 
 /*
  * Section 2.5: TopB_h(a_star) per head under (a_star descending, position

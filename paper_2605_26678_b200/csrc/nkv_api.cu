@@ -412,7 +412,8 @@ int nkv_score(nkv_handle* h, const nkv_tensor* K, const float* mu_s, const float
 }
 
 int nkv_budget(nkv_handle* h, const float* a_star, int64_t G, int64_t H, int64_t N, double r,
-               const nkv_params* params, int32_t* budgets, void* ws, size_t ws_bytes, void* stream) {
+               const nkv_params* params, int32_t* budgets, float* thresholds_opt, void* ws, size_t ws_bytes,
+               void* stream) {
     if (!h || !a_star || !budgets || G < 1 || H < 1 || N < 1 || !params_ok(params)) return NKV_ERR_INVALID_ARG;
     if (!(r >= 0.0 && r < 1.0)) return NKV_ERR_INVALID_ARG;
     if (H > 64 || N > (int64_t)1 << 24 || H * N > (int64_t)1 << 30) return NKV_ERR_UNSUPPORTED;
@@ -428,6 +429,8 @@ int nkv_budget(nkv_handle* h, const float* a_star, int64_t G, int64_t H, int64_t
     void* scratch = ws_bytes >= scr_off + budget_scratch_bytes(G, H) ? at<unsigned char>(ws, scr_off) : nullptr;
     CU(launch_budget((int)G, (int)H, (int)N, (int)k, (int)n_safe, a_star, budgets, at<uint32_t>(ws, thr_off),
                      at<int>(ws, 0), scratch, st, &h->launches));
+    if (thresholds_opt)
+        CU(launch_threshold_scores((int)(G * H), at<uint32_t>(ws, thr_off), thresholds_opt, st, &h->launches));
     return NKV_OK;
 }
 

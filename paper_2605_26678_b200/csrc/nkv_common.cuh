@@ -110,6 +110,7 @@ __device__ __forceinline__ void set_status(int* status, int code, int detail) {
 }
 
 // ---- launchers implemented in the .cu files (all enqueue on `stream`, return cudaError_t) ----
+cudaError_t launch_threshold_scores(int units, const uint32_t* thr, float* out, cudaStream_t stream, int64_t* launches);
 constexpr int kWaitProbeDetail = 799;   // status detail recorded by the wait probe
 cudaError_t launch_wait_probe(int* status, uint32_t limit, cudaStream_t stream, int64_t* launches);
 cudaError_t launch_anchor_sums(const TensorView& K, int dtype, int G, const ScoreParams& sp, float* block_sums,

@@ -1422,6 +1422,20 @@ cudaError_t configure_select_kernels() {
     return e;
 }
 
+namespace {
+// the score of a head's last retained token, from the ordered key the budget kernels leave per head
+__global__ void threshold_scores_kernel(int units, const uint32_t* __restrict__ thr, float* __restrict__ out) {
+    const int u = blockIdx.x * blockDim.x + threadIdx.x;
+    if (u < units) out[u] = ord_float(thr[2 * (int64_t)u]);
+}
+}  // namespace
+
+cudaError_t launch_threshold_scores(int units, const uint32_t* thr, float* out, cudaStream_t stream, int64_t* launches) {
+    threshold_scores_kernel<<<(units + 255) / 256, 256, 0, stream>>>(units, thr, out);
+    ++*launches;
+    return cudaGetLastError();
+}
+
 size_t budget_scratch_bytes(int64_t G, int64_t H) {
     return (size_t)G * H * kBins * sizeof(int) + (size_t)G * 256 + (size_t)G * kBudgetCand * 5;
 }

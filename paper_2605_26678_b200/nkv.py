@@ -101,7 +101,7 @@ def load_library():
     L.nkv_workspace_bytes.argtypes = [vp, i64, i64, i64, i64, i32, pp, ctypes.POINTER(sz)]
     L.nkv_anchors.argtypes = [vp, tp, pp, vp, vp, vp, vp, vp, sz, vp]
     L.nkv_score.argtypes = [vp, tp, vp, vp, vp, pp, vp, vp, vp, vp, sz, vp]
-    L.nkv_budget.argtypes = [vp, vp, i64, i64, i64, dbl, pp, vp, vp, sz, vp]
+    L.nkv_budget.argtypes = [vp, vp, i64, i64, i64, dbl, pp, vp, vp, vp, sz, vp]
     L.nkv_select.argtypes = [vp, vp, vp, i64, i64, i64, i64, vp, vp, vp, vp, sz, vp]
     L.nkv_compact.argtypes = [vp, tp, tp, vp, vp, i64, vp, vp, i32, vp, sz, vp]
     L.nkv_compress.argtypes = [vp, tp, tp, dbl, pp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -279,8 +279,9 @@ def _small_ws(device) -> torch.Tensor:
 
 
 def nkv_budget(a_star: torch.Tensor, r: float, params: Optional[Params] = None,
-               ws: Optional[torch.Tensor] = None, h: Optional[Handle] = None) -> torch.Tensor:
-    """a_star [G,H,N] f32 -> budgets [G,H] i32"""
+               ws: Optional[torch.Tensor] = None, h: Optional[Handle] = None, want_thresholds: bool = False):
+    """a_star [G,H,N] f32 -> budgets [G,H] i32 (and, with want_thresholds, each head's selection threshold, f32 [G,H]:
+    the head keeps the tokens scoring above it and as many of those scoring exactly it as the budget allows)"""
     h = h or handle()
     params = params or nkv_default_params()
     a_star = a_star.contiguous()
@@ -289,9 +290,10 @@ def nkv_budget(a_star: torch.Tensor, r: float, params: Optional[Params] = None,
     # status words, thresholds and the scratch of the parallel form of the group competition
     ws = ws if ws is not None else torch.empty(8192 + 16 * G * H + G * H * 8192 + G * (256 + 5 * 8192), dtype=torch.uint8,
                                                device=a_star.device)
-    _check(h.lib.nkv_budget(h.h, _p(a_star), G, H, N, float(r), ctypes.byref(params), _p(budgets), _p(ws),
+    thresholds = torch.empty((G, H), dtype=torch.float32, device=a_star.device) if want_thresholds else None
+    _check(h.lib.nkv_budget(h.h, _p(a_star), G, H, N, float(r), ctypes.byref(params), _p(budgets), _p(thresholds), _p(ws),
                             ws.numel(), _stream()), "nkv_budget")
-    return budgets
+    return (budgets, thresholds) if want_thresholds else budgets
 
 
 def nkv_budget_static(a_star: torch.Tensor, r: float, params: Optional[Params] = None,

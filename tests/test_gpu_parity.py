@@ -410,3 +410,22 @@ def test_a_wait_that_runs_out_is_reported_and_leaves_the_device_usable():
     out = nkv.nkv_compress(K, V, 0.75, p, ws=ws)
     assert nkv.nkv_last_device_status(ws) == nkv.NKV_OK
     assert int(out.budgets.sum()) == K.shape[1] * nkv.nkv_keep_per_head(K.shape[2], 0.75)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("r", [0.5, 0.75, 0.95])
+def test_budget_thresholds_bracket_the_budgets(r):
+    """nkv_budget's optional thresholds: per head, the tokens scoring above the threshold fit into the budget and the
+    tokens scoring at least the threshold fill it (Section 2.6: the threshold is the score of the last slot taken)."""
+    g = torch.Generator(device="cpu").manual_seed(11)
+    G, H, N = 3, 8, 5000
+    a = torch.rand((G, H, N), generator=g, dtype=torch.float32)
+    a[:, :, ::7] = a[:, :, 1::7][:, :, : a[:, :, ::7].shape[2]]   # plant exact ties
+    a[:, :, :4] = float("inf")
+    a_dev = a.cuda()
+    budgets, thr = nkv.nkv_budget(a_dev, r, want_thresholds=True)
+    assert torch.equal(budgets.cpu(), nkv.nkv_budget(a_dev, r).cpu())
+    above = (a_dev > thr[:, :, None]).sum(dim=2)
+    at_least = (a_dev >= thr[:, :, None]).sum(dim=2)
+    assert bool((above <= budgets).all()) and bool((budgets <= at_least).all())
+    assert int(budgets.sum()) == G * H * nkv.nkv_keep_per_head(N, r)
