@@ -794,7 +794,7 @@ __global__ void __launch_bounds__(kT, kT == 256 ? 4 : 1) scale_stats_kernel(int 
 // mix: elementwise.  Every CTA recomputes its head's three weights and surprise constants (a handful of
 // flops) and routes a chunk of tokens: a* = (1 - alpha) * blend + alpha * max, sinks pinned to +inf.
 constexpr int kMixThreads = 256;
-constexpr int kMixPerThread = 8;
+constexpr int kMixPerThread = 16;
 __global__ void __launch_bounds__(kMixThreads) mix_kernel(int N, ScoreParams sp, const float* __restrict__ a_raw,
                                                           const uint32_t* __restrict__ mm,
                                                           const float* __restrict__ hstat, float* __restrict__ a_star,
