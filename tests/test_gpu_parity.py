@@ -429,3 +429,38 @@ def test_budget_thresholds_bracket_the_budgets(r):
     at_least = (a_dev >= thr[:, :, None]).sum(dim=2)
     assert bool((above <= budgets).all()) and bool((budgets <= at_least).all())
     assert int(budgets.sum()) == G * H * nkv.nkv_keep_per_head(N, r)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("seed", [7, 23])
+def test_random_shapes_end_to_end(seed):
+    """Twenty seeded random calls per seed (N from 65 to 12000 with tile-aligned and ragged lengths, d, storage, heads,
+    layers, ratio and key-pass form drawn at random), each compared with the oracle group by group."""
+    import random
+    rng = random.Random(seed)
+    p = nkv.nkv_default_params()
+    swaps = heads = 0
+    for case in range(20):
+        d = rng.choice([64, 128, 128])
+        dtype = rng.choice(["bf16", "bf16", "fp16", "fp32"])
+        N = rng.choice([rng.randint(65, 700), rng.randint(700, 5000), rng.randint(5000, 12000), 128 * rng.randint(1, 40),
+                        256 * rng.randint(1, 20) + rng.choice([0, 1, 127])])
+        H, layers = rng.randint(1, 8), rng.randint(1, 3)
+        r = rng.choice([0.25, 0.5, 0.75, 0.85, 0.95])
+        mode = rng.choice(["auto", "tensor", "tensor", "fma"])
+        if nkv.nkv_keep_per_head(N, r) < 1:
+            continue
+        K, V = _cache(N, d, dtype, H=H, layers=layers, seed=100 * seed + case, seg=(32, rng.choice([96, 400, 2000])))
+        ws = nkv.alloc_workspace(K, p)
+        nkv.nkv_set_key_passes(mode)
+        try:
+            res = nkv.nkv_compress(K, V, r, p, ws=ws, want_a_star=True)
+        finally:
+            nkv.nkv_set_key_passes("auto")
+        assert nkv.nkv_last_device_status(ws) == nkv.NKV_OK, (case, N, d, dtype, H, layers, r, mode)
+        rep = pr.SwapReport()
+        for g in range(K.shape[0]):
+            pr.check_group_against_oracle(K, V, res, g, r, p, rep)
+        swaps += rep.swapped_tokens
+        heads += rep.heads
+    assert swaps <= max(4, heads // 50)
