@@ -32,10 +32,10 @@
 //     sums     (4 warps)   sums of normalised keys per eight-row segment
 //     scan     (4 warps)   prefix sum, a_c, outputs, min/max
 // Groups hand work to each other through mbarriers; every wait is bounded and a group that gives up
-// records where and leaves, which makes the others give up in turn.  What bounds the kernel is the
-// shared-memory data pipe (operand reads of the MMAs, the copies landing, the segment sums' key reads,
-// barrier polls): outer loops are kept rolled and the kernel's code under 48 KB, because with all groups
-// running different code a larger kernel also starves on instruction fetch.
+// records where and leaves, which makes the others give up in turn.  The busiest unit is the shared-memory
+// data pipe (operand reads of the MMAs, the copies landing, the segment sums' key reads, barrier polls).  Outer
+// loops are kept rolled and the kernel's code under 48 KB: with all groups running different code a kernel of
+// 66 KB starved on instruction fetch.
 #include "nkv_sm100.cuh"
 
 namespace nkv {
